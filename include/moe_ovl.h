@@ -1,0 +1,201 @@
+/* moe_ovl -- the expert-side half of a Mixture-of-Experts layer on one NVIDIA B200
+ * (sm_100a), with the return of expert outputs overlapped with the expert GEMMs
+ * through per-tile ready flags.
+ *
+ * Plain C ABI: every pointer is a raw address, marked below as HOST or DEVICE.
+ * The library never allocates device memory: the caller hands it one workspace
+ * (moe_ovl_workspace_bytes) and owns every tensor.  All functions return
+ * MOE_OVL_OK (0) or a negative MOE_OVL_ERR_* code; nothing throws, aborts or
+ * traps, on the host or on the device.
+ *
+ * Problem statement (Section 2.1, steps 3-5; Section 3.1): this GPU ("rank
+ * r_self") holds El local experts.  After the first all-to-all it has received M
+ * routed token copies ("rows"), grouped by local expert, each tagged with the
+ * rank that owns the token, the token's index on that rank, and its gate weight.
+ * It must (a) run every row through its expert's SwiGLU FFN, (b) deliver each
+ * output row to the receive buffer of the owning rank in source-token order, and
+ * (c) the owner forms the gate-weighted sum per token.  Source ranks are
+ * simulated: the receive buffer of rank r is a region of this GPU's HBM.
+ *
+ * How it is computed (Section 3.2 and 3.3):
+ *   plan      remote-owner-aligned row layout and remote-first tile schedule
+ *             (Algorithm 1), combine plan (Section 3.2.3), segments (Section 3.3.2)
+ *   producer  one persistent tcgen05 kernel over all local experts; raises one
+ *             ready flag per finished output tile (Section 3.3.1)
+ *   consumer  persistent kernel on consumer_sm_count dedicated SMs; polls the
+ *             flags and moves each finished segment with one contiguous copy
+ *             (Section 3.3.2, 3.3.3)
+ *   combine   gate-weighted reduction at the owner (Section 2.1 step 5)
+ * MOE_OVL_MODE_NON_OVERLAP is the comparison baseline of Section 4.1: the same
+ * GEMM kernel on every SM runs to completion, then a separate scatter kernel
+ * moves all rows, then the same combine.
+ */
+#ifndef MOE_OVL_H
+#define MOE_OVL_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct moe_ovl_ctx moe_ovl_ctx; /* opaque, owned by the library */
+
+enum {
+    MOE_OVL_OK = 0,
+    MOE_OVL_ERR_INVALID_ARG = -1, /* null pointer, negative size, value out of range */
+    MOE_OVL_ERR_UNSUPPORTED = -2, /* shape the kernels do not cover (see moe_ovl_config) */
+    MOE_OVL_ERR_CUDA = -3,        /* a CUDA runtime/driver call failed (moe_ovl_last_cuda_error) */
+    MOE_OVL_ERR_WORKSPACE = -4,   /* workspace missing, misaligned or too small */
+    MOE_OVL_ERR_TIMEOUT = -5,     /* a bounded device-side wait gave up (asynchronous, see query_status) */
+    MOE_OVL_ERR_BAD_ROUTING = -6  /* routing metadata inconsistent (asynchronous, see query_status) */
+};
+
+enum { MOE_OVL_MODE_OVERLAP = 0, MOE_OVL_MODE_NON_OVERLAP = 1 };
+
+/* tile geometry, fixed by the kernels */
+#define MOE_OVL_TB_M 128  /* rows per band (output tile height, tb_M of Algorithm 1) */
+#define MOE_OVL_TB_N 256  /* output tile width of the second GEMM */
+#define MOE_OVL_H_TILE 128 /* hidden columns produced by one tile of the first GEMM */
+
+typedef struct {
+    uint32_t struct_size;       /* sizeof(moe_ovl_config), for ABI checks */
+    int32_t device;             /* CUDA device ordinal */
+    int32_t num_src_ranks;      /* R >= 1 */
+    int32_t self_rank;          /* r_self in 0..R-1: its rows are "local" and are scheduled last */
+    int32_t tokens_per_rank;    /* T: the output has R*T rows */
+    int32_t num_local_experts;  /* El >= 1, El * R <= 1024 */
+    int32_t top_k;              /* k: a token owns at most min(k, El) rows here */
+    int32_t d_model;            /* d, multiple of 256 */
+    int32_t d_ffn;              /* F, multiple of 128 */
+    int32_t max_rows;           /* capacity for M */
+    int32_t mid_seg_bands;      /* bands per middle segment (x of Figure 3b), >= 1 */
+    int32_t group_bands;        /* bands whose tiles are interleaved so that they share weight tiles in L2; 0 = default */
+    int32_t wait_timeout_us;    /* bound on every device-side wait; 0 = default (2 s) */
+    int32_t producer_sm_limit;  /* NON_OVERLAP only: cap on GEMM CTAs (diagnostic baseline); 0 = all SMs */
+    uint32_t flags;             /* MOE_OVL_FLAG_* */
+} moe_ovl_config;
+
+#define MOE_OVL_FLAG_HOST_STAGING 1u /* reserve workspace for moe_ovl_expert_return_host */
+
+typedef struct {
+    uint32_t struct_size;
+    int32_t num_rows;             /* M (host value), 0 <= M <= max_rows */
+    const void *x;                /* DEVICE [M, d] bf16 row-major: rows grouped by local expert 0..El-1 */
+    const int32_t *expert_counts; /* DEVICE [El]: rows per local expert, sum == M */
+    const int32_t *src_rank;      /* DEVICE [M] in 0..R-1: owner rank of the row's token */
+    const int32_t *src_token;     /* DEVICE [M] in 0..T-1: token index on the owner rank */
+    const float *gate;            /* DEVICE [M] fp32 gate weight of (token, expert) */
+    const void *w1;               /* DEVICE [El, 2F, d] bf16: rows 0..F-1 gate projection, F..2F-1 up projection */
+    const void *w2;               /* DEVICE [El, d, F] bf16 */
+    int32_t consumer_sm_count;    /* SMs dedicated to the consumer (OVERLAP); 1..SMs/2 */
+    int32_t mode;                 /* MOE_OVL_MODE_* */
+    void *ret;                    /* DEVICE [R][ret_rows_per_rank, d] bf16: simulated peer receive buffers.
+                                     Row s of region r is written iff s < rows_per_rank[r]; the rest is untouched. */
+    int64_t ret_rows_per_rank;    /* >= T * min(k, El) */
+    void *out;                    /* DEVICE [R*T, d] bf16, fully overwritten (tokens with no local row get +0) */
+    int32_t *slot_out;            /* DEVICE [M] or NULL: receive-buffer slot of every input row */
+    int32_t *rows_per_rank_out;   /* DEVICE [R] or NULL */
+    int32_t *segs_per_rank_out;   /* DEVICE [R] or NULL: segments sent to each rank */
+    void *stream;                 /* cudaStream_t of the caller (NULL = legacy default stream) */
+} moe_ovl_args;
+
+/* Host-buffer variant: every tensor that changes per call lives in HOST memory
+ * (pinned for asynchronous copies); weights stay resident on the device. */
+typedef struct {
+    uint32_t struct_size;
+    int32_t num_rows;
+    const void *x;                /* HOST [M, d] bf16 */
+    const int32_t *expert_counts; /* HOST [El] */
+    const int32_t *src_rank;      /* HOST [M] */
+    const int32_t *src_token;     /* HOST [M] */
+    const float *gate;            /* HOST [M] */
+    const void *w1;               /* DEVICE, as in moe_ovl_args */
+    const void *w2;               /* DEVICE */
+    int32_t consumer_sm_count;
+    int32_t mode;
+    void *out;                    /* HOST [R*T, d] bf16 */
+    void *stream;
+} moe_ovl_host_args;
+
+/* Sizes of the plan of the last call, and where the time went (milliseconds). */
+typedef struct {
+    int32_t padded_rows;      /* P, multiple of 128 */
+    int32_t num_bands;        /* P / 128 */
+    int32_t num_items;        /* schedule length: tiles of both GEMMs */
+    int32_t num_segments;
+    int32_t producer_ctas;
+    int32_t consumer_ctas;    /* 0 in NON_OVERLAP */
+    int32_t kernel_launches;  /* kernels of this library launched by the call */
+    int32_t reserved;
+    float ms_total;           /* whole call on the caller's stream */
+    float ms_prep;            /* plan + gather into the aligned layout */
+    float ms_expert_return;   /* start of the GEMM to the last row landed in ret */
+    float ms_producer;        /* the GEMM kernel alone */
+    float ms_mover;           /* consumer (OVERLAP: concurrent with the GEMM) or scatter kernel */
+    float ms_combine;
+} moe_ovl_report;
+
+/* Integer plan arrays of the last call, copied to HOST buffers (any pointer may be
+ * NULL).  Capacities: bands -> max_bands, items -> max_items, segments -> max_bands
+ * (moe_ovl_limits). */
+typedef struct {
+    int32_t *group_rows;      /* [El*R]  n[e][r] */
+    int32_t *pos;             /* [M]     aligned position of every input row */
+    int32_t *band_expert;     /* [bands] in band-id order (band id = first position / 128) */
+    int32_t *band_dest;
+    int32_t *band_valid;
+    int32_t *band_slot0;
+    int32_t *sched_band;      /* [bands] band ids in schedule order */
+    int32_t *item;            /* [items][4] = {kind (0 first GEMM, 1 second), band, tile, expert} in issue order */
+    int32_t *seg;             /* [segments][4] = {first band, bands, dest rank, rows} in schedule order */
+    int32_t *tok_slot;        /* [R*T*min(k,El)] slots of each token's rows, ascending expert, -1 = none */
+    float *tok_gate;          /* [R*T*min(k,El)] matching gates */
+} moe_ovl_plan_view;
+
+enum { MOE_OVL_BUF_XA = 0, MOE_OVL_BUF_H = 1, MOE_OVL_BUF_Y = 2 };
+
+/* Bytes of workspace moe_ovl_create needs for this configuration (256-byte aligned base). */
+int moe_ovl_workspace_bytes(const moe_ovl_config *cfg, size_t *bytes);
+
+/* Capacities derived from the configuration. */
+int moe_ovl_limits(const moe_ovl_config *cfg, int32_t *max_bands, int32_t *max_items);
+
+/* Creates a context on cfg->device.  `workspace` is DEVICE memory owned by the caller
+ * and must outlive the context.  Creates two internal streams and their events;
+ * allocates no device memory. */
+int moe_ovl_create(moe_ovl_ctx **ctx, const moe_ovl_config *cfg, void *workspace, size_t workspace_bytes);
+
+/* Enqueues one pass of the path: plan, gather, expert FFN + return, combine.
+ * Asynchronous: ordered after earlier work on args->stream, complete for later work
+ * on it.  One call in flight per context.  Synchronous argument errors are returned
+ * here; device-side errors are reported by moe_ovl_query_status. */
+int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *args);
+
+/* Same pass with per-call tensors in HOST memory: copies inputs to staging buffers
+ * in the workspace, runs the pass, copies `out` back.  Needs MOE_OVL_FLAG_HOST_STAGING.
+ * Asynchronous with respect to the host if the buffers are pinned. */
+int moe_ovl_expert_return_host(moe_ovl_ctx *ctx, const moe_ovl_host_args *args);
+
+/* Waits for the last call and returns its device status: *code is MOE_OVL_OK,
+ * MOE_OVL_ERR_TIMEOUT or MOE_OVL_ERR_BAD_ROUTING; *detail identifies the wait or
+ * the row.  After an error the outputs are unspecified but were written in bounds. */
+int moe_ovl_query_status(moe_ovl_ctx *ctx, int32_t *code, int64_t *detail);
+
+/* Waits for the last call, then fills the report / copies plan arrays / reads back
+ * `bytes` bytes at `offset` of an internal bf16 buffer (MOE_OVL_BUF_*) to HOST memory. */
+int moe_ovl_get_report(moe_ovl_ctx *ctx, moe_ovl_report *report);
+int moe_ovl_get_plan(moe_ovl_ctx *ctx, const moe_ovl_plan_view *view);
+int moe_ovl_read_buffer(moe_ovl_ctx *ctx, int32_t which, size_t offset, size_t bytes, void *host_dst);
+
+int moe_ovl_destroy(moe_ovl_ctx *ctx);
+
+const char *moe_ovl_strerror(int code);
+/* cudaError_t of the last failing CUDA call made through this context (0 if none). */
+int moe_ovl_last_cuda_error(const moe_ovl_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_OVL_H */

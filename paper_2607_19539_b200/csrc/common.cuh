@@ -1,0 +1,139 @@
+// Shared definitions of the moe_ovl kernels: the parameter block every kernel
+// receives, the device status word, and small PTX wrappers for ordered memory
+// access and bounded waiting.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace moe_ovl {
+
+constexpr int TB_M = 128;     // rows per band (tb_M of Algorithm 1)
+constexpr int TB_N = 256;     // accumulator width of one tile (both GEMMs)
+constexpr int TB_K = 64;      // K extent of one pipeline stage: 64 bf16 = one 128-byte swizzle row
+constexpr int H_TILE = 128;   // hidden columns per first-GEMM tile (gate half + up half of the accumulator)
+
+constexpr int KIND_G1 = 0;    // x . W1 (gate | up) -> SiLU * up -> H
+constexpr int KIND_G2 = 1;    // H . W2 -> Y, raises the consumer-visible flag
+
+// meta[] slots written by the plan kernel
+enum { META_P = 0, META_BANDS, META_ITEMS, META_SEGS, META_SUPERBANDS, META_COUNT = 8 };
+// status[] slots
+enum { ST_CODE = 0, ST_ABORT = 1, ST_DETAIL_LO = 2, ST_DETAIL_HI = 3, ST_COUNT = 4 };
+
+constexpr int ERR_TIMEOUT = -5;
+constexpr int ERR_BAD_ROUTING = -6;
+
+// wait sites reported in the high bits of the status detail
+enum : long long {
+    SITE_TMA_EMPTY = 1, SITE_TMA_HCOUNT, SITE_MMA_FULL, SITE_MMA_TEMPTY, SITE_EPI_TFULL, SITE_CONS_FLAG,
+    SITE_MMA_DRAIN, SITE_TMA_DRAIN,
+    SITE_ROW_RANGE = 16, SITE_ROW_DUP, SITE_COUNT_SUM, SITE_TOK_OVERFLOW
+};
+
+struct Params {
+    // problem
+    int R, r_self, T, El, kmax, d, F;
+    int M;
+    int mgb;            // bands per middle segment
+    int group_bands;    // bands interleaved in one super-band
+    int lag_items;      // schedule items between a band's last first-GEMM tile and its first second-GEMM tile
+    int words;          // 32-bit words of one (expert, rank) token bitmap = ceil(T / 32)
+    int n1, n2;         // tiles per band: F / 128 and d / 256
+    int max_bands, max_items;
+    unsigned epoch;
+    unsigned long long timeout_ns;
+    long long ret_rows_per_rank;
+    // inputs
+    const uint16_t *x;
+    const int *expert_counts, *src_rank, *src_token;
+    const float *gate;
+    // outputs
+    uint16_t *ret, *out;
+    int *slot_out, *rows_per_rank_out, *segs_per_rank_out;
+    // workspace
+    uint16_t *Xa, *H, *Y;
+    unsigned *bitmap;     // [El*R][words]
+    int *wordpfx;         // [El*R][words] exclusive popcount prefix inside a group
+    int *group_rows;      // [El*R] n[e][r]
+    int *group_start;     // [El*R] aligned position of the group's first row
+    int *group_slot;      // [El*R] slot of the group's first row in ret[r]
+    int *pos;             // [M]
+    int *slot;            // [M]
+    int *band_expert, *band_dest, *band_valid, *band_slot0;   // [max_bands]
+    int *sched_band;      // [max_bands]
+    int4 *items;          // [max_items] {kind, band, tile, expert}
+    int4 *segs;           // [max_bands] {first band, bands, dest, rows}
+    int *seg_slot0;       // [max_bands]
+    int *tok_slot;        // [R*T*kmax]
+    float *tok_gate;      // [R*T*kmax]
+    unsigned *hcount;     // [max_bands] first-GEMM tiles finished per band
+    unsigned *flags;      // [max_bands*n2] epoch of the call that finished the tile
+    int *meta;            // [META_COUNT]
+    int *status;          // [ST_COUNT]
+};
+
+// ------------------------------------------------------------------ ordered access
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_u32(unsigned *p, unsigned v)
+{
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void red_release_add_u32(unsigned *p, unsigned v)
+{
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_volatile_s32(const int *p)
+{
+    int v;
+    asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// First error wins; every later waiter sees ST_ABORT and gives up at once.
+__device__ __forceinline__ void report_error(int *status, int code, long long site, long long index)
+{
+    if (atomicCAS(&status[ST_CODE], 0, code) == 0) {
+        long long detail = (site << 48) | (index & 0xffffffffffffll);
+        status[ST_DETAIL_LO] = (int)(detail & 0xffffffffll);
+        status[ST_DETAIL_HI] = (int)(detail >> 32);
+    }
+    __threadfence();
+    atomicExch(&status[ST_ABORT], 1);
+}
+
+// Spin until *p == want (exact) or *p >= want (at_least), giving up at the deadline
+// or when another waiter has aborted.  Returns false on give-up.
+__device__ __forceinline__ bool wait_global(const unsigned *p, unsigned want, bool at_least, const Params &prm,
+                                            long long site, long long index)
+{
+    unsigned v = ld_acquire_u32(p);
+    if (at_least ? (v >= want) : (v == want)) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    for (unsigned it = 1;; ++it) {
+        v = ld_acquire_u32(p);
+        if (at_least ? (v >= want) : (v == want)) return true;
+        if ((it & 63u) == 0) {
+            if (ld_volatile_s32(&prm.status[ST_ABORT])) return false;
+            if (globaltimer_ns() - t0 > prm.timeout_ns) {
+                report_error(prm.status, ERR_TIMEOUT, site, index);
+                return false;
+            }
+            __nanosleep(64);
+        }
+    }
+}
+
+}  // namespace moe_ovl

@@ -1,0 +1,547 @@
+// C-ABI entry points of moe_ovl (see include/moe_ovl.h): context, workspace layout,
+// tensor maps, and the launch sequence of one pass.  Host code only orchestrates;
+// every step of the path runs in the kernels of plan.cuh, producer.cuh, mover.cuh.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "../../include/moe_ovl.h"
+#include "common.cuh"
+#include "mover.cuh"
+#include "plan.cuh"
+#include "producer.cuh"
+
+using namespace moe_ovl;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr size_t ALIGN = 1024;
+inline size_t align_up(size_t v, size_t a = ALIGN) { return (v + a - 1) / a * a; }
+
+struct Layout {
+    // offsets into the workspace, in bytes
+    size_t Xa, H, Y;
+    size_t zero_begin, bitmap, hcount, status, zero_end;   // cleared to 0 at the start of every call
+    size_t tok_slot, tok_slot_bytes;                       // filled with -1 at the start of every call
+    size_t wordpfx, group_rows, group_start, group_slot, pos, slot;
+    size_t band_expert, band_dest, band_valid, band_slot0, sched_band, items, segs, seg_slot0;
+    size_t tok_gate, flags, meta;
+    size_t sb[6];
+    // host staging (MOE_OVL_FLAG_HOST_STAGING)
+    size_t st_x, st_counts, st_rank, st_token, st_gate, st_ret, st_out;
+    size_t total;
+    int max_bands, max_items, words, kmax, n1, n2;
+    long long st_ret_rows;
+};
+
+int check_config(const moe_ovl_config *c)
+{
+    if (!c || c->struct_size != sizeof(moe_ovl_config)) return MOE_OVL_ERR_INVALID_ARG;
+    if (c->num_src_ranks < 1 || c->self_rank < 0 || c->self_rank >= c->num_src_ranks) return MOE_OVL_ERR_INVALID_ARG;
+    if (c->tokens_per_rank < 1 || c->num_local_experts < 1 || c->top_k < 1) return MOE_OVL_ERR_INVALID_ARG;
+    if (c->max_rows < 0 || c->mid_seg_bands < 0 || c->group_bands < 0 || c->wait_timeout_us < 0 ||
+        c->producer_sm_limit < 0 || c->d_model < 1 || c->d_ffn < 1)
+        return MOE_OVL_ERR_INVALID_ARG;
+    if (c->d_model % TB_N != 0 || c->d_ffn % H_TILE != 0) return MOE_OVL_ERR_UNSUPPORTED;
+    if (c->num_local_experts > PLAN_MAX_EXPERTS ||
+        (long long)c->num_local_experts * c->num_src_ranks > PLAN_MAX_GROUPS)
+        return MOE_OVL_ERR_UNSUPPORTED;
+    return MOE_OVL_OK;
+}
+
+int make_layout(const moe_ovl_config *c, Layout *L)
+{
+    const int rc = check_config(c);
+    if (rc != MOE_OVL_OK) return rc;
+    const long long G = (long long)c->num_local_experts * c->num_src_ranks;
+    const long long max_bands_ll = ((long long)c->max_rows + TB_M - 1) / TB_M + G;
+    L->n1 = c->d_ffn / H_TILE;
+    L->n2 = c->d_model / TB_N;
+    const long long max_items_ll = max_bands_ll * (L->n1 + L->n2);
+    if (max_bands_ll > (1 << 24) || max_items_ll > (1ll << 30)) return MOE_OVL_ERR_UNSUPPORTED;
+    L->max_bands = (int)max_bands_ll;
+    L->max_items = (int)max_items_ll;
+    L->words = (c->tokens_per_rank + 31) / 32;
+    L->kmax = std::min(c->top_k, c->num_local_experts);
+    const size_t P = (size_t)L->max_bands * TB_M, d = c->d_model, F = c->d_ffn;
+    const size_t ntok = (size_t)c->num_src_ranks * c->tokens_per_rank;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    L->Xa = take(P * d * 2);
+    L->H = take(P * F * 2);
+    L->Y = take(P * d * 2);
+    L->zero_begin = off;
+    L->bitmap = take((size_t)G * L->words * 4);
+    L->hcount = take((size_t)L->max_bands * 4);
+    L->status = take(ST_COUNT * 4);
+    L->zero_end = off;
+    L->tok_slot_bytes = ntok * L->kmax * 4;
+    L->tok_slot = take(L->tok_slot_bytes);
+    L->tok_gate = take(ntok * L->kmax * 4);
+    L->wordpfx = take((size_t)G * L->words * 4);
+    L->group_rows = take((size_t)G * 4);
+    L->group_start = take((size_t)G * 4);
+    L->group_slot = take((size_t)G * 4);
+    L->pos = take((size_t)std::max(c->max_rows, 1) * 4);
+    L->slot = take((size_t)std::max(c->max_rows, 1) * 4);
+    L->band_expert = take((size_t)L->max_bands * 4);
+    L->band_dest = take((size_t)L->max_bands * 4);
+    L->band_valid = take((size_t)L->max_bands * 4);
+    L->band_slot0 = take((size_t)L->max_bands * 4);
+    L->sched_band = take((size_t)L->max_bands * 4);
+    L->items = take((size_t)L->max_items * 16);
+    L->segs = take((size_t)L->max_bands * 16);
+    L->seg_slot0 = take((size_t)L->max_bands * 4);
+    L->flags = take((size_t)L->max_bands * L->n2 * 4);
+    L->meta = take(META_COUNT * 4);
+    for (int i = 0; i < 6; ++i) L->sb[i] = take((size_t)L->max_bands * 4);
+    L->st_ret_rows = (long long)c->tokens_per_rank * L->kmax;
+    if (c->flags & MOE_OVL_FLAG_HOST_STAGING) {
+        L->st_x = take((size_t)std::max(c->max_rows, 1) * d * 2);
+        L->st_counts = take((size_t)c->num_local_experts * 4);
+        L->st_rank = take((size_t)std::max(c->max_rows, 1) * 4);
+        L->st_token = take((size_t)std::max(c->max_rows, 1) * 4);
+        L->st_gate = take((size_t)std::max(c->max_rows, 1) * 4);
+        L->st_ret = take((size_t)c->num_src_ranks * L->st_ret_rows * d * 2);
+        L->st_out = take(ntok * d * 2);
+    }
+    L->total = off;
+    return MOE_OVL_OK;
+}
+
+}  // namespace
+
+struct moe_ovl_ctx {
+    moe_ovl_config cfg;
+    Layout L;
+    uint8_t *ws;
+    int num_sms;
+    unsigned epoch;
+    cudaStream_t s_prod, s_cons;
+    cudaEvent_t ev_fork, ev_prod_done, ev_cons_done;
+    // timing: call start, after prep, GEMM start/end, mover start/end, call end
+    cudaEvent_t t_begin, t_prep, t_p0, t_p1, t_m0, t_m1, t_end;
+    cudaStream_t last_stream;
+    bool ran;
+    int last_mode, last_prod_ctas, last_cons_ctas, last_launches, last_rows;
+    int last_cuda_error;
+    EncodeTiledFn encode;
+    CUtensorMap map_xa, map_h;
+};
+
+namespace {
+
+#define CU_CHECK(ctx, call)                                  \
+    do {                                                     \
+        cudaError_t e_ = (call);                             \
+        if (e_ != cudaSuccess) {                             \
+            (ctx)->last_cuda_error = (int)e_;                \
+            return MOE_OVL_ERR_CUDA;                         \
+        }                                                    \
+    } while (0)
+
+// 2-D bf16 row-major tensor [rows, cols], box = 64 columns x 128 rows, 128-byte swizzle
+int encode_map(moe_ovl_ctx *ctx, CUtensorMap *map, const void *base, size_t rows, size_t cols)
+{
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)std::max<size_t>(rows, 1)};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {TB_K, TB_M};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides,
+                                   box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        ctx->last_cuda_error = (int)r;
+        return MOE_OVL_ERR_CUDA;
+    }
+    return MOE_OVL_OK;
+}
+
+template <typename T>
+T *at(moe_ovl_ctx *ctx, size_t off) { return reinterpret_cast<T *>(ctx->ws + off); }
+
+Params make_params(moe_ovl_ctx *ctx)
+{
+    const moe_ovl_config &c = ctx->cfg;
+    const Layout &L = ctx->L;
+    Params p;
+    std::memset(&p, 0, sizeof(p));
+    p.R = c.num_src_ranks; p.r_self = c.self_rank; p.T = c.tokens_per_rank; p.El = c.num_local_experts;
+    p.kmax = L.kmax; p.d = c.d_model; p.F = c.d_ffn;
+    p.mgb = std::max(1, c.mid_seg_bands);
+    p.group_bands = c.group_bands > 0 ? c.group_bands : 8;
+    p.words = L.words; p.n1 = L.n1; p.n2 = L.n2; p.max_bands = L.max_bands; p.max_items = L.max_items;
+    p.timeout_ns = (unsigned long long)(c.wait_timeout_us > 0 ? c.wait_timeout_us : 2000000) * 1000ull;
+    p.Xa = at<uint16_t>(ctx, L.Xa); p.H = at<uint16_t>(ctx, L.H); p.Y = at<uint16_t>(ctx, L.Y);
+    p.bitmap = at<unsigned>(ctx, L.bitmap); p.wordpfx = at<int>(ctx, L.wordpfx);
+    p.group_rows = at<int>(ctx, L.group_rows); p.group_start = at<int>(ctx, L.group_start);
+    p.group_slot = at<int>(ctx, L.group_slot); p.pos = at<int>(ctx, L.pos); p.slot = at<int>(ctx, L.slot);
+    p.band_expert = at<int>(ctx, L.band_expert); p.band_dest = at<int>(ctx, L.band_dest);
+    p.band_valid = at<int>(ctx, L.band_valid); p.band_slot0 = at<int>(ctx, L.band_slot0);
+    p.sched_band = at<int>(ctx, L.sched_band); p.items = at<int4>(ctx, L.items); p.segs = at<int4>(ctx, L.segs);
+    p.seg_slot0 = at<int>(ctx, L.seg_slot0); p.tok_slot = at<int>(ctx, L.tok_slot);
+    p.tok_gate = at<float>(ctx, L.tok_gate); p.hcount = at<unsigned>(ctx, L.hcount);
+    p.flags = at<unsigned>(ctx, L.flags); p.meta = at<int>(ctx, L.meta); p.status = at<int>(ctx, L.status);
+    return p;
+}
+
+int sync_last(moe_ovl_ctx *ctx)
+{
+    if (ctx->ran) CU_CHECK(ctx, cudaStreamSynchronize(ctx->last_stream));
+    return MOE_OVL_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *moe_ovl_strerror(int code)
+{
+    switch (code) {
+    case MOE_OVL_OK: return "ok";
+    case MOE_OVL_ERR_INVALID_ARG: return "invalid argument";
+    case MOE_OVL_ERR_UNSUPPORTED: return "unsupported shape";
+    case MOE_OVL_ERR_CUDA: return "CUDA call failed";
+    case MOE_OVL_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case MOE_OVL_ERR_TIMEOUT: return "a device-side wait timed out";
+    case MOE_OVL_ERR_BAD_ROUTING: return "inconsistent routing metadata";
+    default: return "unknown error";
+    }
+}
+
+int moe_ovl_workspace_bytes(const moe_ovl_config *cfg, size_t *bytes)
+{
+    if (!bytes) return MOE_OVL_ERR_INVALID_ARG;
+    Layout L;
+    const int rc = make_layout(cfg, &L);
+    if (rc != MOE_OVL_OK) return rc;
+    *bytes = L.total + ALIGN;     // slack to round the base up to the alignment TMA-read buffers need
+    return MOE_OVL_OK;
+}
+
+int moe_ovl_limits(const moe_ovl_config *cfg, int32_t *max_bands, int32_t *max_items)
+{
+    Layout L;
+    const int rc = make_layout(cfg, &L);
+    if (rc != MOE_OVL_OK) return rc;
+    if (max_bands) *max_bands = L.max_bands;
+    if (max_items) *max_items = L.max_items;
+    return MOE_OVL_OK;
+}
+
+int moe_ovl_last_cuda_error(const moe_ovl_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+int moe_ovl_create(moe_ovl_ctx **out, const moe_ovl_config *cfg, void *workspace, size_t workspace_bytes)
+{
+    if (!out) return MOE_OVL_ERR_INVALID_ARG;
+    *out = nullptr;
+    Layout L;
+    int rc = make_layout(cfg, &L);
+    if (rc != MOE_OVL_OK) return rc;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < L.total + ALIGN)
+        return MOE_OVL_ERR_WORKSPACE;
+    moe_ovl_ctx *ctx = new (std::nothrow) moe_ovl_ctx();
+    if (!ctx) return MOE_OVL_ERR_INVALID_ARG;
+    std::memset(ctx, 0, sizeof(*ctx));
+    ctx->cfg = *cfg;
+    ctx->L = L;
+    // the layout assumes a 1024-byte aligned base; round up inside the slack
+    ctx->ws = reinterpret_cast<uint8_t *>(align_up(reinterpret_cast<uintptr_t>(workspace)));
+
+    auto fail = [&](int code) { moe_ovl_destroy(ctx); return code; };
+#define CREATE_CHECK(call)                                         \
+    do {                                                           \
+        if ((call) != cudaSuccess) return fail(MOE_OVL_ERR_CUDA);  \
+    } while (0)
+    CREATE_CHECK(cudaSetDevice(cfg->device));
+    CREATE_CHECK(cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, cfg->device));
+    int lo = 0, hi = 0;
+    CREATE_CHECK(cudaDeviceGetStreamPriorityRange(&lo, &hi));
+    // the consumer stream gets the higher priority (Section 3.3.3)
+    CREATE_CHECK(cudaStreamCreateWithPriority(&ctx->s_cons, cudaStreamNonBlocking, hi));
+    CREATE_CHECK(cudaStreamCreateWithPriority(&ctx->s_prod, cudaStreamNonBlocking, lo));
+    cudaEvent_t *plain[] = {&ctx->ev_fork, &ctx->ev_prod_done, &ctx->ev_cons_done};
+    for (auto e : plain) CREATE_CHECK(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
+    cudaEvent_t *timed[] = {&ctx->t_begin, &ctx->t_prep, &ctx->t_p0, &ctx->t_p1, &ctx->t_m0, &ctx->t_m1, &ctx->t_end};
+    for (auto e : timed) CREATE_CHECK(cudaEventCreate(e));
+    CREATE_CHECK(cudaFuncSetAttribute(producer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PROD_SMEM_BYTES));
+    CREATE_CHECK(cudaFuncSetAttribute(consumer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      CONSUMER_SMEM_BYTES));
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    CREATE_CHECK(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) return fail(MOE_OVL_ERR_CUDA);
+    ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    const size_t P = (size_t)L.max_bands * TB_M;
+    rc = encode_map(ctx, &ctx->map_xa, ctx->ws + L.Xa, P, cfg->d_model);
+    if (rc == MOE_OVL_OK) rc = encode_map(ctx, &ctx->map_h, ctx->ws + L.H, P, cfg->d_ffn);
+    if (rc != MOE_OVL_OK) return fail(rc);
+    // flags hold the epoch of the call that finished the tile: clear them once, never again
+    CREATE_CHECK(cudaMemset(ctx->ws + L.flags, 0, (size_t)L.max_bands * L.n2 * 4));
+    CREATE_CHECK(cudaMemset(ctx->ws + L.meta, 0, META_COUNT * 4));
+    CREATE_CHECK(cudaMemset(ctx->ws + L.status, 0, ST_COUNT * 4));
+#undef CREATE_CHECK
+    *out = ctx;
+    return MOE_OVL_OK;
+}
+
+int moe_ovl_destroy(moe_ovl_ctx *ctx)
+{
+    if (!ctx) return MOE_OVL_OK;
+    if (ctx->ran) cudaStreamSynchronize(ctx->last_stream);
+    if (ctx->s_prod) { cudaStreamSynchronize(ctx->s_prod); cudaStreamDestroy(ctx->s_prod); }
+    if (ctx->s_cons) { cudaStreamSynchronize(ctx->s_cons); cudaStreamDestroy(ctx->s_cons); }
+    cudaEvent_t evs[] = {ctx->ev_fork, ctx->ev_prod_done, ctx->ev_cons_done, ctx->t_begin, ctx->t_prep, ctx->t_p0,
+                         ctx->t_p1, ctx->t_m0, ctx->t_m1, ctx->t_end};
+    for (auto e : evs)
+        if (e) cudaEventDestroy(e);
+    delete ctx;
+    return MOE_OVL_OK;
+}
+
+int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
+{
+    if (!ctx || !a || a->struct_size != sizeof(moe_ovl_args)) return MOE_OVL_ERR_INVALID_ARG;
+    const moe_ovl_config &c = ctx->cfg;
+    const Layout &L = ctx->L;
+    if (a->num_rows < 0 || a->num_rows > c.max_rows) return MOE_OVL_ERR_INVALID_ARG;
+    if (!a->expert_counts || !a->w1 || !a->w2 || !a->ret || !a->out) return MOE_OVL_ERR_INVALID_ARG;
+    if (a->num_rows > 0 && (!a->x || !a->src_rank || !a->src_token || !a->gate)) return MOE_OVL_ERR_INVALID_ARG;
+    if (a->ret_rows_per_rank < (int64_t)c.tokens_per_rank * L.kmax) return MOE_OVL_ERR_INVALID_ARG;
+    if (a->mode != MOE_OVL_MODE_OVERLAP && a->mode != MOE_OVL_MODE_NON_OVERLAP) return MOE_OVL_ERR_INVALID_ARG;
+    const uintptr_t align16 = reinterpret_cast<uintptr_t>(a->x) | reinterpret_cast<uintptr_t>(a->w1) |
+                              reinterpret_cast<uintptr_t>(a->w2) | reinterpret_cast<uintptr_t>(a->ret) |
+                              reinterpret_cast<uintptr_t>(a->out);
+    if (align16 & 15u) return MOE_OVL_ERR_INVALID_ARG;
+    const bool overlap = a->mode == MOE_OVL_MODE_OVERLAP;
+    int prod_ctas, cons_ctas = 0;
+    if (overlap) {
+        if (a->consumer_sm_count < 1 || a->consumer_sm_count > ctx->num_sms / 2) return MOE_OVL_ERR_INVALID_ARG;
+        cons_ctas = a->consumer_sm_count;
+        prod_ctas = ctx->num_sms - cons_ctas;       // disjoint SM sets: grids sum to the SM count
+    } else {
+        prod_ctas = c.producer_sm_limit > 0 ? std::min(c.producer_sm_limit, ctx->num_sms) : ctx->num_sms;
+    }
+    CU_CHECK(ctx, cudaSetDevice(c.device));
+    cudaStream_t st = static_cast<cudaStream_t>(a->stream);
+
+    Params p = make_params(ctx);
+    p.M = a->num_rows;
+    p.epoch = ++ctx->epoch;
+    p.lag_items = 2 * prod_ctas;
+    p.ret_rows_per_rank = a->ret_rows_per_rank;
+    p.x = static_cast<const uint16_t *>(a->x);
+    p.expert_counts = a->expert_counts; p.src_rank = a->src_rank; p.src_token = a->src_token; p.gate = a->gate;
+    p.ret = static_cast<uint16_t *>(a->ret); p.out = static_cast<uint16_t *>(a->out);
+    p.slot_out = a->slot_out; p.rows_per_rank_out = a->rows_per_rank_out; p.segs_per_rank_out = a->segs_per_rank_out;
+
+    ProducerMaps maps;
+    maps.xa = ctx->map_xa;
+    maps.h = ctx->map_h;
+    int rc = encode_map(ctx, &maps.w1, a->w1, (size_t)c.num_local_experts * 2 * c.d_ffn, c.d_model);
+    if (rc == MOE_OVL_OK) rc = encode_map(ctx, &maps.w2, a->w2, (size_t)c.num_local_experts * c.d_model, c.d_ffn);
+    if (rc != MOE_OVL_OK) return rc;
+
+    PlanScratch sc;
+    sc.sb_start = at<int>(ctx, L.sb[0]); sc.sb_nb = at<int>(ctx, L.sb[1]); sc.sb_expert = at<int>(ctx, L.sb[2]);
+    sc.sb_g1off = at<int>(ctx, L.sb[3]); sc.sb_g2off = at<int>(ctx, L.sb[4]); sc.sb_g1end = at<int>(ctx, L.sb[5]);
+
+    int launches = 0;
+    CU_CHECK(ctx, cudaEventRecord(ctx->t_begin, st));
+    // ---- plan + gather (8a-1 .. 8a-3): integer kernels on the caller's stream
+    CU_CHECK(ctx, cudaMemsetAsync(ctx->ws + L.zero_begin, 0, L.zero_end - L.zero_begin, st));
+    CU_CHECK(ctx, cudaMemsetAsync(ctx->ws + L.tok_slot, 0xff, L.tok_slot_bytes, st));
+    if (p.M > 0) {
+        plan_mark_kernel<<<(p.M + 255) / 256, 256, 0, st>>>(p);
+        ++launches;
+    }
+    plan_build_kernel<<<1, PLAN_THREADS, 0, st>>>(p, sc);
+    ++launches;
+    if (p.M > 0) {
+        plan_rows_kernel<<<(p.M + 7) / 8, 256, 0, st>>>(p);
+        plan_zero_pad_kernel<<<std::min(L.max_bands, 4 * ctx->num_sms), 256, 0, st>>>(p);
+        launches += 2;
+    }
+    CU_CHECK(ctx, cudaGetLastError());
+    CU_CHECK(ctx, cudaEventRecord(ctx->t_prep, st));
+
+    if (overlap) {
+        // ---- two persistent kernels on two streams, disjoint SM sets (Section 3.3.3)
+        CU_CHECK(ctx, cudaEventRecord(ctx->ev_fork, st));
+        CU_CHECK(ctx, cudaStreamWaitEvent(ctx->s_cons, ctx->ev_fork, 0));
+        CU_CHECK(ctx, cudaStreamWaitEvent(ctx->s_prod, ctx->ev_fork, 0));
+        CU_CHECK(ctx, cudaEventRecord(ctx->t_m0, ctx->s_cons));
+        consumer_kernel<<<cons_ctas, MOVER_THREADS, CONSUMER_SMEM_BYTES, ctx->s_cons>>>(p);
+        CU_CHECK(ctx, cudaEventRecord(ctx->t_m1, ctx->s_cons));
+        CU_CHECK(ctx, cudaEventRecord(ctx->ev_cons_done, ctx->s_cons));
+        CU_CHECK(ctx, cudaEventRecord(ctx->t_p0, ctx->s_prod));
+        producer_kernel<<<prod_ctas, PROD_THREADS, PROD_SMEM_BYTES, ctx->s_prod>>>(maps, p, 1);
+        CU_CHECK(ctx, cudaEventRecord(ctx->t_p1, ctx->s_prod));
+        CU_CHECK(ctx, cudaEventRecord(ctx->ev_prod_done, ctx->s_prod));
+        CU_CHECK(ctx, cudaStreamWaitEvent(st, ctx->ev_cons_done, 0));
+        CU_CHECK(ctx, cudaStreamWaitEvent(st, ctx->ev_prod_done, 0));
+    } else {
+        // ---- comparison baseline: the GEMM runs to completion, then a separate scatter kernel
+        CU_CHECK(ctx, cudaEventRecord(ctx->t_p0, st));
+        producer_kernel<<<prod_ctas, PROD_THREADS, PROD_SMEM_BYTES, st>>>(maps, p, 0);
+        CU_CHECK(ctx, cudaEventRecord(ctx->t_p1, st));
+        CU_CHECK(ctx, cudaEventRecord(ctx->t_m0, st));
+        scatter_kernel<<<8 * ctx->num_sms, 256, 0, st>>>(p);
+        CU_CHECK(ctx, cudaEventRecord(ctx->t_m1, st));
+    }
+    launches += 2;
+    combine_kernel<<<8 * ctx->num_sms, 256, 0, st>>>(p);
+    ++launches;
+    CU_CHECK(ctx, cudaGetLastError());
+    CU_CHECK(ctx, cudaEventRecord(ctx->t_end, st));
+
+    ctx->last_stream = st;
+    ctx->ran = true;
+    ctx->last_mode = a->mode;
+    ctx->last_prod_ctas = prod_ctas;
+    ctx->last_cons_ctas = cons_ctas;
+    ctx->last_launches = launches;
+    ctx->last_rows = p.M;
+    return MOE_OVL_OK;
+}
+
+int moe_ovl_expert_return_host(moe_ovl_ctx *ctx, const moe_ovl_host_args *h)
+{
+    if (!ctx || !h || h->struct_size != sizeof(moe_ovl_host_args)) return MOE_OVL_ERR_INVALID_ARG;
+    const moe_ovl_config &c = ctx->cfg;
+    const Layout &L = ctx->L;
+    if (!(c.flags & MOE_OVL_FLAG_HOST_STAGING)) return MOE_OVL_ERR_WORKSPACE;
+    if (h->num_rows < 0 || h->num_rows > c.max_rows || !h->expert_counts || !h->out) return MOE_OVL_ERR_INVALID_ARG;
+    if (h->num_rows > 0 && (!h->x || !h->src_rank || !h->src_token || !h->gate)) return MOE_OVL_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(h->stream);
+    const size_t M = (size_t)h->num_rows, d = c.d_model;
+    CU_CHECK(ctx, cudaSetDevice(c.device));
+    CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_counts, h->expert_counts, (size_t)c.num_local_experts * 4,
+                                  cudaMemcpyHostToDevice, st));
+    if (M > 0) {
+        CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_x, h->x, M * d * 2, cudaMemcpyHostToDevice, st));
+        CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_rank, h->src_rank, M * 4, cudaMemcpyHostToDevice, st));
+        CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_token, h->src_token, M * 4, cudaMemcpyHostToDevice, st));
+        CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_gate, h->gate, M * 4, cudaMemcpyHostToDevice, st));
+    }
+    moe_ovl_args a;
+    std::memset(&a, 0, sizeof(a));
+    a.struct_size = sizeof(a);
+    a.num_rows = h->num_rows;
+    a.x = ctx->ws + L.st_x;
+    a.expert_counts = at<int32_t>(ctx, L.st_counts);
+    a.src_rank = at<int32_t>(ctx, L.st_rank);
+    a.src_token = at<int32_t>(ctx, L.st_token);
+    a.gate = at<float>(ctx, L.st_gate);
+    a.w1 = h->w1; a.w2 = h->w2;
+    a.consumer_sm_count = h->consumer_sm_count;
+    a.mode = h->mode;
+    a.ret = ctx->ws + L.st_ret;
+    a.ret_rows_per_rank = L.st_ret_rows;
+    a.out = ctx->ws + L.st_out;
+    a.stream = h->stream;
+    const int rc = moe_ovl_expert_return(ctx, &a);
+    if (rc != MOE_OVL_OK) return rc;
+    CU_CHECK(ctx, cudaMemcpyAsync(h->out, ctx->ws + L.st_out, (size_t)c.num_src_ranks * c.tokens_per_rank * d * 2,
+                                  cudaMemcpyDeviceToHost, st));
+    return MOE_OVL_OK;
+}
+
+int moe_ovl_query_status(moe_ovl_ctx *ctx, int32_t *code, int64_t *detail)
+{
+    if (!ctx) return MOE_OVL_ERR_INVALID_ARG;
+    int rc = sync_last(ctx);
+    if (rc != MOE_OVL_OK) return rc;
+    int st[ST_COUNT] = {0, 0, 0, 0};
+    CU_CHECK(ctx, cudaMemcpy(st, ctx->ws + ctx->L.status, sizeof(st), cudaMemcpyDeviceToHost));
+    if (code) *code = st[ST_CODE];
+    if (detail) *detail = ((int64_t)st[ST_DETAIL_HI] << 32) | (uint32_t)st[ST_DETAIL_LO];
+    return MOE_OVL_OK;
+}
+
+int moe_ovl_get_report(moe_ovl_ctx *ctx, moe_ovl_report *r)
+{
+    if (!ctx || !r) return MOE_OVL_ERR_INVALID_ARG;
+    std::memset(r, 0, sizeof(*r));
+    if (!ctx->ran) return MOE_OVL_OK;
+    int rc = sync_last(ctx);
+    if (rc != MOE_OVL_OK) return rc;
+    int meta[META_COUNT];
+    CU_CHECK(ctx, cudaMemcpy(meta, ctx->ws + ctx->L.meta, sizeof(meta), cudaMemcpyDeviceToHost));
+    r->padded_rows = meta[META_P];
+    r->num_bands = meta[META_BANDS];
+    r->num_items = meta[META_ITEMS];
+    r->num_segments = meta[META_SEGS];
+    r->producer_ctas = ctx->last_prod_ctas;
+    r->consumer_ctas = ctx->last_cons_ctas;
+    r->kernel_launches = ctx->last_launches;
+    float prod_end = 0.f, mover_end = 0.f;
+    CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_total, ctx->t_begin, ctx->t_end));
+    CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_prep, ctx->t_begin, ctx->t_prep));
+    CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_producer, ctx->t_p0, ctx->t_p1));
+    CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_mover, ctx->t_m0, ctx->t_m1));
+    CU_CHECK(ctx, cudaEventElapsedTime(&prod_end, ctx->t_prep, ctx->t_p1));
+    CU_CHECK(ctx, cudaEventElapsedTime(&mover_end, ctx->t_prep, ctx->t_m1));
+    r->ms_expert_return = std::max(prod_end, mover_end);
+    r->ms_combine = r->ms_total - r->ms_prep - r->ms_expert_return;
+    return MOE_OVL_OK;
+}
+
+int moe_ovl_get_plan(moe_ovl_ctx *ctx, const moe_ovl_plan_view *v)
+{
+    if (!ctx || !v) return MOE_OVL_ERR_INVALID_ARG;
+    if (!ctx->ran) return MOE_OVL_ERR_INVALID_ARG;
+    int rc = sync_last(ctx);
+    if (rc != MOE_OVL_OK) return rc;
+    const Layout &L = ctx->L;
+    const moe_ovl_config &c = ctx->cfg;
+    int meta[META_COUNT];
+    CU_CHECK(ctx, cudaMemcpy(meta, ctx->ws + L.meta, sizeof(meta), cudaMemcpyDeviceToHost));
+    const size_t B = (size_t)meta[META_BANDS], M = (size_t)ctx->last_rows;
+    const size_t ntokk = (size_t)c.num_src_ranks * c.tokens_per_rank * L.kmax;
+    struct { void *dst; size_t off, bytes; } cp[] = {
+        {v->group_rows, L.group_rows, (size_t)c.num_local_experts * c.num_src_ranks * 4},
+        {v->pos, L.pos, M * 4},
+        {v->band_expert, L.band_expert, B * 4},
+        {v->band_dest, L.band_dest, B * 4},
+        {v->band_valid, L.band_valid, B * 4},
+        {v->band_slot0, L.band_slot0, B * 4},
+        {v->sched_band, L.sched_band, B * 4},
+        {v->item, L.items, (size_t)meta[META_ITEMS] * 16},
+        {v->seg, L.segs, (size_t)meta[META_SEGS] * 16},
+        {v->tok_slot, L.tok_slot, ntokk * 4},
+        {v->tok_gate, L.tok_gate, ntokk * 4},
+    };
+    for (auto &e : cp)
+        if (e.dst && e.bytes) CU_CHECK(ctx, cudaMemcpy(e.dst, ctx->ws + e.off, e.bytes, cudaMemcpyDeviceToHost));
+    return MOE_OVL_OK;
+}
+
+int moe_ovl_read_buffer(moe_ovl_ctx *ctx, int32_t which, size_t offset, size_t bytes, void *host_dst)
+{
+    if (!ctx || !host_dst) return MOE_OVL_ERR_INVALID_ARG;
+    const Layout &L = ctx->L;
+    const size_t P = (size_t)L.max_bands * TB_M;
+    size_t base, cap;
+    switch (which) {
+    case MOE_OVL_BUF_XA: base = L.Xa; cap = P * ctx->cfg.d_model * 2; break;
+    case MOE_OVL_BUF_H: base = L.H; cap = P * ctx->cfg.d_ffn * 2; break;
+    case MOE_OVL_BUF_Y: base = L.Y; cap = P * ctx->cfg.d_model * 2; break;
+    default: return MOE_OVL_ERR_INVALID_ARG;
+    }
+    if (offset > cap || bytes > cap - offset) return MOE_OVL_ERR_INVALID_ARG;
+    int rc = sync_last(ctx);
+    if (rc != MOE_OVL_OK) return rc;
+    if (bytes) CU_CHECK(ctx, cudaMemcpy(host_dst, ctx->ws + base + offset, bytes, cudaMemcpyDeviceToHost));
+    return MOE_OVL_OK;
+}
+
+}  // extern "C"

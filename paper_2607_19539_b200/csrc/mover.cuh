@@ -1,0 +1,118 @@
+// Return path and weighted reduction.
+//   consumer_kernel  persistent, one CTA per dedicated SM: polls the ready flags of its
+//                    next segment and moves the segment's valid rows into the owner
+//                    rank's receive buffer with one contiguous copy (Section 3.3.2-3.3.3)
+//   scatter_kernel   the non-overlap comparison: all bands, whole GPU, after the GEMM
+//   combine_kernel   out[r,t] = sum_j gate_j * ret[r][slot_j]  (Section 2.1 step 5)
+// All three are HBM/L2-bandwidth work: 16-byte coalesced loads and stores.
+#pragma once
+
+#include "common.cuh"
+
+namespace moe_ovl {
+
+constexpr int MOVER_THREADS = 1024;
+// Dynamic shared memory the consumer asks for but never touches: large enough that neither a
+// second consumer CTA nor a GEMM CTA fits on the same SM, which gives the consumer SMs of its own.
+constexpr int CONSUMER_SMEM_BYTES = 120 * 1024;
+
+__device__ __forceinline__ void copy_rows_16B(const uint16_t *src, uint16_t *dst, size_t nvec, int tid, int nthr)
+{
+    const uint4 *s = reinterpret_cast<const uint4 *>(src);
+    uint4 *d = reinterpret_cast<uint4 *>(dst);
+    size_t v = tid;
+    for (; v + 3 * (size_t)nthr < nvec; v += 4 * (size_t)nthr) {
+        const uint4 a = __ldcg(s + v), b = __ldcg(s + v + nthr), c = __ldcg(s + v + 2 * (size_t)nthr),
+                    e = __ldcg(s + v + 3 * (size_t)nthr);
+        __stcs(d + v, a);
+        __stcs(d + v + nthr, b);
+        __stcs(d + v + 2 * (size_t)nthr, c);
+        __stcs(d + v + 3 * (size_t)nthr, e);
+    }
+    for (; v < nvec; v += nthr) __stcs(d + v, __ldcg(s + v));
+}
+
+__global__ void __launch_bounds__(MOVER_THREADS, 1) consumer_kernel(const Params p)
+{
+    extern __shared__ uint8_t unused_smem[];
+    __shared__ int s_ok;
+    const int nseg = p.meta[META_SEGS];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // segments are listed in schedule order; CTA c takes segments c, c + cSM, ...
+    for (int s = blockIdx.x; s < nseg; s += gridDim.x) {
+        const int4 seg = p.segs[s];                  // {first band, bands, dest, rows}
+        if (warp == 0) {
+            // a segment is ready when every tile of every one of its bands is flagged (acquire)
+            const int nflags = seg.y * p.n2;
+            const unsigned *f = p.flags + (size_t)seg.x * p.n2;
+            bool ok = true;
+            for (int i = lane; i < nflags && ok; i += 32)
+                ok = wait_global(f + i, p.epoch, false, p, SITE_CONS_FLAG, (long long)seg.x * p.n2 + i);
+            ok = __all_sync(0xffffffffu, ok);
+            if (lane == 0) s_ok = ok ? 1 : 0;
+        }
+        __syncthreads();
+        if (!s_ok) return;
+        const uint16_t *src = p.Y + (size_t)seg.x * TB_M * p.d;
+        uint16_t *dst = p.ret + ((size_t)seg.z * p.ret_rows_per_rank + p.seg_slot0[s]) * p.d;
+        copy_rows_16B(src, dst, (size_t)seg.w * p.d / 8, threadIdx.x, blockDim.x);
+        __syncthreads();
+    }
+}
+
+// One CTA per (band, chunk of rows): grid-stride over bands x chunks.
+constexpr int SCATTER_CHUNKS = 8;     // 16 rows each
+__global__ void __launch_bounds__(256) scatter_kernel(const Params p)
+{
+    const int nbands = p.meta[META_BANDS];
+    const int rows_per_chunk = TB_M / SCATTER_CHUNKS;
+    for (int u = blockIdx.x; u < nbands * SCATTER_CHUNKS; u += gridDim.x) {
+        const int band = u / SCATTER_CHUNKS, chunk = u % SCATTER_CHUNKS;
+        const int valid = p.band_valid[band];
+        const int r0 = chunk * rows_per_chunk;
+        if (r0 >= valid) continue;
+        const int rows = min(rows_per_chunk, valid - r0);
+        const uint16_t *src = p.Y + ((size_t)band * TB_M + r0) * p.d;
+        uint16_t *dst = p.ret + ((size_t)p.band_dest[band] * p.ret_rows_per_rank + p.band_slot0[band] + r0) * p.d;
+        copy_rows_16B(src, dst, (size_t)rows * p.d / 8, threadIdx.x, blockDim.x);
+    }
+}
+
+// One CTA per token at a time; thread v handles 8 consecutive features.
+__global__ void __launch_bounds__(256) combine_kernel(const Params p)
+{
+    const int ntok = p.R * p.T;
+    const int nv = p.d / 8;
+    for (int tok = blockIdx.x; tok < ntok; tok += gridDim.x) {
+        const int r = tok / p.T;
+        const int *ts = p.tok_slot + (size_t)tok * p.kmax;
+        const float *tg = p.tok_gate + (size_t)tok * p.kmax;
+        const uint16_t *base = p.ret + (size_t)r * p.ret_rows_per_rank * p.d;
+        uint4 *o = reinterpret_cast<uint4 *>(p.out + (size_t)tok * p.d);
+        for (int v = threadIdx.x; v < nv; v += blockDim.x) {
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            for (int j = 0; j < p.kmax; ++j) {           // ascending local expert
+                const int slot = ts[j];
+                if (slot < 0) break;
+                const float g = tg[j];
+                const uint4 q = __ldcs(reinterpret_cast<const uint4 *>(base + (size_t)slot * p.d) + v);
+                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    acc[2 * i] += g * __uint_as_float(w[i] << 16);
+                    acc[2 * i + 1] += g * __uint_as_float(w[i] & 0xffff0000u);
+                }
+            }
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t r2;
+                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r2) : "f"(acc[2 * i + 1]), "f"(acc[2 * i]));
+                w[i] = r2;
+            }
+            o[v] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
+}
+
+}  // namespace moe_ovl

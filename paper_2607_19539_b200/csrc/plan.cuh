@@ -1,0 +1,310 @@
+// Plan kernels: remote-owner-aligned row layout and remote-first tile schedule
+// (Algorithm 1), combine plan (Section 3.2.3), segments (Section 3.3.2, Figure 3b),
+// and the gather of the dispatched rows into the aligned layout.
+//
+// All integer work.  Rank-in-group is found without sorting: a routed copy is
+// identified by (expert, owner rank, token), so every (expert, rank) group gets a
+// bitmap over the T tokens of that rank; the rank of a row inside its group (rows
+// in source-token order) is the number of set bits below its token.
+#pragma once
+
+#include "common.cuh"
+
+namespace moe_ovl {
+
+constexpr int PLAN_MAX_GROUPS = 1024;   // El * R
+constexpr int PLAN_MAX_EXPERTS = 256;   // El
+constexpr int PLAN_THREADS = 1024;
+
+// Scratch arrays of the plan kernel, one entry per super-band.
+struct PlanScratch {
+    int *sb_start;   // first schedule position
+    int *sb_nb;      // bands
+    int *sb_expert;
+    int *sb_g1off;   // item index of the super-band's first-GEMM block
+    int *sb_g2off;   // item index of its second-GEMM block
+    int *sb_g1end;
+};
+
+__device__ __forceinline__ int expert_of_row(const int *pre, int El, int i)
+{
+    // pre[e] = first row of expert e, pre[El] = total; largest e with pre[e] <= i
+    int lo = 0, hi = El;
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (pre[mid] <= i) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ void load_expert_prefix(const Params &p, int *pre)
+{
+    if (threadIdx.x == 0) {
+        int acc = 0;
+        for (int e = 0; e < p.El; ++e) {
+            pre[e] = acc;
+            acc += p.expert_counts[e];
+        }
+        pre[p.El] = acc;
+    }
+    __syncthreads();
+}
+
+// ---- step 1: mark (expert, rank, token) of every row ---------------------------------------
+__global__ void __launch_bounds__(256) plan_mark_kernel(Params p)
+{
+    __shared__ int pre[PLAN_MAX_EXPERTS + 1];
+    load_expert_prefix(p, pre);
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= p.M) return;
+    if (i >= pre[p.El]) {
+        report_error(p.status, ERR_BAD_ROUTING, SITE_COUNT_SUM, i);
+        return;
+    }
+    const int e = expert_of_row(pre, p.El, i);
+    const int r = p.src_rank[i], t = p.src_token[i];
+    if (r < 0 || r >= p.R || t < 0 || t >= p.T) {
+        report_error(p.status, ERR_BAD_ROUTING, SITE_ROW_RANGE, i);
+        return;
+    }
+    const unsigned bit = 1u << (t & 31);
+    const unsigned old = atomicOr(&p.bitmap[(size_t)(e * p.R + r) * p.words + (t >> 5)], bit);
+    if (old & bit) report_error(p.status, ERR_BAD_ROUTING, SITE_ROW_DUP, i);
+}
+
+__device__ __forceinline__ int num_segments(int nb, int mgb)
+{
+    return nb <= 2 ? nb : 2 + (nb - 2 + mgb - 1) / mgb;
+}
+
+// ---- step 2: everything that is per group / band / segment / schedule item -------------------
+__global__ void __launch_bounds__(PLAN_THREADS, 1) plan_build_kernel(Params p, PlanScratch sc)
+{
+    __shared__ int n[PLAN_MAX_GROUPS], nb[PLAN_MAX_GROUPS], gstart[PLAN_MAX_GROUPS], gslot[PLAN_MAX_GROUPS];
+    __shared__ int gsched[PLAN_MAX_GROUPS], gsegoff[PLAN_MAX_GROUPS];
+    __shared__ int key[PLAN_MAX_EXPERTS], eorder[PLAN_MAX_EXPERTS];
+    __shared__ int run_start[2 * PLAN_MAX_EXPERTS], run_nb[2 * PLAN_MAX_EXPERTS], run_sb0[2 * PLAN_MAX_EXPERTS + 1];
+    __shared__ int run_exp[2 * PLAN_MAX_EXPERTS];
+    __shared__ int segs_per_rank[PLAN_MAX_GROUPS];
+    __shared__ int s_nsb, s_items;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    const int G = p.El * p.R;
+    const int R = p.R, El = p.El, self = p.r_self;
+
+    // A: per group, exclusive popcount prefix over its bitmap words, and n[e][r]
+    for (int g = warp; g < G; g += nwarps) {
+        const unsigned *bm = p.bitmap + (size_t)g * p.words;
+        int *wp = p.wordpfx + (size_t)g * p.words;
+        int run = 0;
+        for (int w0 = 0; w0 < p.words; w0 += 32) {
+            const int w = w0 + lane;
+            const int c = w < p.words ? __popc(bm[w]) : 0;
+            int inc = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += v;
+            }
+            if (w < p.words) wp[w] = run + inc - c;
+            run += __shfl_sync(0xffffffffu, inc, 31);
+        }
+        if (lane == 0) n[g] = run;
+    }
+    for (int r = tid; r < R; r += blockDim.x) segs_per_rank[r] = 0;
+    __syncthreads();
+
+    // B: row layout (Algorithm 1): per expert, remote owner groups in ascending rank, local group last,
+    //    every group rounded up to a multiple of tb_M; receive-buffer slots expert-major and dense
+    if (tid == 0) {
+        int total = 0, cursor = 0;
+        for (int e = 0; e < El; ++e) {
+            int remote_bands = 0;
+            for (int q = 0; q < R; ++q) {
+                const int r = q < R - 1 ? (q < self ? q : q + 1) : self;   // remote ranks ascending, then self
+                const int g = e * R + r;
+                gstart[g] = cursor;
+                nb[g] = (n[g] + TB_M - 1) / TB_M;
+                cursor += nb[g] * TB_M;
+                total += n[g];
+                if (r != self) remote_bands += nb[g];
+            }
+            key[e] = remote_bands;
+        }
+        for (int r = 0; r < R; ++r) {
+            int acc = 0;
+            for (int e = 0; e < El; ++e) {
+                gslot[e * R + r] = acc;
+                acc += n[e * R + r];
+            }
+            if (p.rows_per_rank_out) p.rows_per_rank_out[r] = acc;
+        }
+        p.meta[META_P] = cursor;
+        p.meta[META_BANDS] = cursor / TB_M;
+        if (total != p.M) report_error(p.status, ERR_BAD_ROUTING, SITE_COUNT_SUM, total);
+    }
+    __syncthreads();
+
+    // C: experts by remote band count, descending; ties to the lower index (Algorithm 1, rule (ii))
+    for (int e = tid; e < El; e += blockDim.x) {
+        int rank = 0;
+        for (int o = 0; o < El; ++o) rank += (key[o] > key[e]) || (key[o] == key[e] && o < e);
+        eorder[rank] = e;
+    }
+    __syncthreads();
+
+    // D: schedule positions of groups.  Runs: the remote bands of each expert in sorted order (rule (i):
+    //    all remote tiles first), then the local bands of each expert in natural order.
+    if (tid == 0) {
+        int spos = 0, segoff = 0, sbcount = 0;
+        for (int run = 0; run < 2 * El; ++run) {
+            const bool remote = run < El;
+            const int e = remote ? eorder[run] : run - El;
+            run_start[run] = spos;
+            run_exp[run] = e;
+            for (int q = remote ? 0 : R - 1; q < (remote ? R - 1 : R); ++q) {
+                const int r = q < R - 1 ? (q < self ? q : q + 1) : self;
+                const int g = e * R + r;
+                gsched[g] = spos;
+                spos += nb[g];
+                gsegoff[g] = segoff;
+                const int ns = num_segments(nb[g], p.mgb);
+                segoff += ns;
+                segs_per_rank[r] += ns;
+            }
+            run_nb[run] = spos - run_start[run];
+            run_sb0[run] = sbcount;
+            sbcount += (run_nb[run] + p.group_bands - 1) / p.group_bands;
+        }
+        run_sb0[2 * El] = sbcount;
+        s_nsb = sbcount;
+        p.meta[META_SEGS] = segoff;
+        p.meta[META_SUPERBANDS] = sbcount;
+    }
+    __syncthreads();
+
+    // E: band table, schedule order of bands, segments, super-bands
+    for (int g = warp; g < G; g += nwarps) {
+        const int e = g / R, r = g % R;
+        for (int b = lane; b < nb[g]; b += 32) {
+            const int band = gstart[g] / TB_M + b;
+            p.band_expert[band] = e;
+            p.band_dest[band] = r;
+            p.band_valid[band] = min(TB_M, n[g] - b * TB_M);
+            p.band_slot0[band] = gslot[g] + b * TB_M;
+            p.sched_band[gsched[g] + b] = band;
+            p.hcount[band] = 0;
+        }
+        const int ns = num_segments(nb[g], p.mgb);
+        for (int q = lane; q < ns; q += 32) {
+            int first, cnt;
+            if (nb[g] <= 2 || q == 0) { first = q; cnt = 1; }
+            else if (q == ns - 1) { first = nb[g] - 1; cnt = 1; }
+            else { first = 1 + (q - 1) * p.mgb; cnt = min(p.mgb, nb[g] - 1 - first); }
+            const int rows = min(n[g] - first * TB_M, cnt * TB_M);
+            p.segs[gsegoff[g] + q] = make_int4(gstart[g] / TB_M + first, cnt, r, rows);
+            p.seg_slot0[gsegoff[g] + q] = gslot[g] + first * TB_M;
+        }
+        if (lane == 0) p.group_rows[g] = n[g];
+        if (lane == 1) p.group_start[g] = gstart[g];
+        if (lane == 2) p.group_slot[g] = gslot[g];
+    }
+    for (int r = tid; r < R; r += blockDim.x)
+        if (p.segs_per_rank_out) p.segs_per_rank_out[r] = segs_per_rank[r];
+    for (int run = tid; run < 2 * El; run += blockDim.x) {
+        const int nsb = run_sb0[run + 1] - run_sb0[run];
+        for (int q = 0; q < nsb; ++q) {
+            const int base = run_nb[run] / nsb, rem = run_nb[run] % nsb;
+            const int sb = run_sb0[run] + q;
+            sc.sb_start[sb] = run_start[run] + q * base + min(q, rem);
+            sc.sb_nb[sb] = base + (q < rem ? 1 : 0);
+            sc.sb_expert[sb] = run_exp[run];
+        }
+    }
+    __syncthreads();
+
+    // F: issue order of tile blocks.  Inside a super-band the tile index is the outer loop and the band the
+    //    inner one, so that the CTAs working side by side share a weight tile.  The second-GEMM block of a
+    //    super-band is issued lag_items items after its first-GEMM block, so that its input is normally
+    //    complete when a CTA reaches it.
+    if (tid == 0) {
+        const int nsb = s_nsb;
+        int ng1 = 0, off = 0;
+        for (int ng2 = 0; ng2 < nsb; ++ng2) {
+            while (ng1 < nsb && (ng1 <= ng2 || off - sc.sb_g1end[ng2] < p.lag_items)) {
+                sc.sb_g1off[ng1] = off;
+                off += sc.sb_nb[ng1] * p.n1;
+                sc.sb_g1end[ng1] = off;
+                ++ng1;
+            }
+            sc.sb_g2off[ng2] = off;
+            off += sc.sb_nb[ng2] * p.n2;
+        }
+        s_items = off;
+        p.meta[META_ITEMS] = off;
+    }
+    __syncthreads();
+
+    // G: the item list
+    for (int sb = 0; sb < s_nsb; ++sb) {
+        const int start = sc.sb_start[sb], cnt = sc.sb_nb[sb], e = sc.sb_expert[sb];
+        const int o1 = sc.sb_g1off[sb], o2 = sc.sb_g2off[sb];
+        for (int idx = tid; idx < cnt * p.n1; idx += blockDim.x)
+            p.items[o1 + idx] = make_int4(KIND_G1, p.sched_band[start + idx % cnt], idx / cnt, e);
+        for (int idx = tid; idx < cnt * p.n2; idx += blockDim.x)
+            p.items[o2 + idx] = make_int4(KIND_G2, p.sched_band[start + idx % cnt], idx / cnt, e);
+    }
+}
+
+// ---- step 3: per row: aligned position, return slot, per-token list entry, copy into the layout ---
+__global__ void __launch_bounds__(256) plan_rows_kernel(Params p)
+{
+    __shared__ int pre[PLAN_MAX_EXPERTS + 1];
+    load_expert_prefix(p, pre);
+    const int lane = threadIdx.x & 31;
+    const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (i >= p.M || i >= pre[p.El]) return;
+    const int e = expert_of_row(pre, p.El, i);
+    const int r = p.src_rank[i], t = p.src_token[i];
+    if (r < 0 || r >= p.R || t < 0 || t >= p.T) return;
+    const int g = e * p.R + r;
+    const size_t w = (size_t)g * p.words + (t >> 5);
+    const int q = p.wordpfx[w] + __popc(p.bitmap[w] & ((1u << (t & 31)) - 1u));
+    const int pos = p.group_start[g] + q;
+    const int slot = p.group_slot[g] + q;
+    // entry of this row in its token's list: number of lower-indexed local experts the token also selected
+    int j = 0;
+    for (int o = lane; o < e; o += 32)
+        j += (p.bitmap[(size_t)(o * p.R + r) * p.words + (t >> 5)] >> (t & 31)) & 1u;
+    j = __reduce_add_sync(0xffffffffu, j);
+    if (lane == 0) {
+        p.pos[i] = pos;
+        p.slot[i] = slot;
+        if (p.slot_out) p.slot_out[i] = slot;
+        if (j < p.kmax) {
+            const size_t at = ((size_t)r * p.T + t) * p.kmax + j;
+            p.tok_slot[at] = slot;
+            p.tok_gate[at] = p.gate[i];
+        } else {
+            report_error(p.status, ERR_BAD_ROUTING, SITE_TOK_OVERFLOW, i);
+        }
+    }
+    const uint4 *src = reinterpret_cast<const uint4 *>(p.x + (size_t)i * p.d);
+    uint4 *dst = reinterpret_cast<uint4 *>(p.Xa + (size_t)pos * p.d);
+    const int nv = p.d / 8;
+    for (int v = lane; v < nv; v += 32) dst[v] = __ldg(src + v);
+}
+
+// ---- step 4: zero the padding rows of every band (Section 3.2.1: zero-filled rows) -----------
+__global__ void __launch_bounds__(256) plan_zero_pad_kernel(Params p)
+{
+    const int nbands = p.meta[META_BANDS];
+    for (int band = blockIdx.x; band < nbands; band += gridDim.x) {
+        const int valid = p.band_valid[band];
+        uint4 *dst = reinterpret_cast<uint4 *>(p.Xa + ((size_t)band * TB_M + valid) * p.d);
+        const size_t nv = (size_t)(TB_M - valid) * p.d / 8;
+        for (size_t v = threadIdx.x; v < nv; v += blockDim.x) dst[v] = make_uint4(0, 0, 0, 0);
+    }
+}
+
+}  // namespace moe_ovl

@@ -1,0 +1,392 @@
+// Producer: one persistent kernel that runs the grouped SwiGLU FFN of all local
+// experts from a single launch, following the plan's item list, and raises a ready
+// flag per finished output tile (Section 3.3.1: rank-wide persistent GEMM with
+// tile-level signalling in the epilogue).
+//
+// sm_100a design (the paper's is CUTLASS on A100): warp-specialised CTA, one per SM.
+//   warp 0     TMA loads (cp.async.bulk.tensor, 128-byte swizzle) into a 4-stage ring
+//   warp 1     one thread issues tcgen05.mma (bf16 x bf16 -> fp32, M=128 N=256 K=16),
+//              accumulators in tensor memory, double buffered (2 x 256 columns)
+//   warps 2-5  epilogue: tcgen05.ld -> fp32 math -> bf16 -> global, then publish
+// A schedule item is one 128-row band times one tile:
+//   first GEMM   A = Xa[band], B = 128 gate rows and 128 up rows of W1 -> one N=256
+//                accumulator; the epilogue pairs column c with c+128: h = silu(g) * u,
+//                128 columns of H; then hcount[band] += 1 (release)
+//   second GEMM  waits until hcount[band] == F/128, A = H[band], B = 256 rows of W2,
+//                writes 256 columns of Y; then flag[band][tile] = epoch (release)
+// Every wait is bounded; on a give-up the CTA records a status, drains its copies,
+// frees its tensor memory and returns.
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace moe_ovl {
+
+constexpr int PROD_STAGES = 4;
+constexpr int PROD_A_BYTES = TB_M * TB_K * 2;          // 16 KiB
+constexpr int PROD_B_BYTES = TB_N * TB_K * 2;          // 32 KiB
+constexpr int PROD_STAGE_BYTES = PROD_A_BYTES + PROD_B_BYTES;
+constexpr int PROD_THREADS = 192;
+constexpr int PROD_TMEM_COLS = 512;
+constexpr int PROD_SMEM_BYTES = PROD_STAGES * PROD_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+// ------------------------------------------------------------------ PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait on an mbarrier phase.  False = gave up (deadline, or another waiter aborted).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Params &prm, long long site,
+                                          long long index)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    for (unsigned it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 0) {
+            if (ld_volatile_s32(&prm.status[ST_ABORT])) return false;
+            if (globaltimer_ns() - t0 > prm.timeout_ns) {
+                report_error(prm.status, ERR_TIMEOUT, site, index);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap *map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]; bf16 inputs, fp32 accumulate
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The mbarrier gets one arrival when every MMA issued so far by this thread has finished.
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+// 32 lanes x 32 columns of fp32: thread t of the warp gets lane (base lane + t), 32 consecutive columns
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory operand descriptor: K-major tile, 128-byte swizzle, rows of 128 bytes packed in groups of
+// eight (stride between groups 1024 bytes), descriptor version 1.
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3ffffu) >> 4);          // start address
+    d |= (uint64_t)1 << 16;                            // leading byte offset (unused with swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset
+    d |= (uint64_t)1 << 46;                            // version
+    d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
+    return d;
+}
+// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N=256, M=128.
+constexpr uint32_t UMMA_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TB_N >> 3) << 17) |
+                                ((uint32_t)(TB_M >> 4) << 24);
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
+
+__device__ __forceinline__ void bar_sync_epilogue() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// AND over the 128 epilogue threads, so that they leave the tile loop together
+__device__ __forceinline__ bool epilogue_all(bool ok)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, 2, 128, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)ok)
+        : "memory");
+    return r != 0;
+}
+
+// ------------------------------------------------------------------ kernel
+
+struct ProducerMaps {
+    CUtensorMap xa, h, w1, w2;   // all 2-D bf16 row-major, box 64 x 128, 128-byte swizzle
+};
+
+__global__ void __launch_bounds__(PROD_THREADS, 1)
+producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const int raise_flags)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bars = smem_base + PROD_STAGES * PROD_STAGE_BYTES;
+    // barrier slots, 8 bytes each
+    const uint32_t bar_full = bars, bar_empty = bars + 8 * PROD_STAGES;
+    const uint32_t bar_tfull = bars + 16 * PROD_STAGES, bar_tempty = bar_tfull + 16, bar_drain = bar_tempty + 16;
+    const uint32_t tmem_slot = bar_drain + 8;
+    uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    volatile uint32_t *tmem_slot_gen = reinterpret_cast<volatile uint32_t *>(
+        smem_gen + PROD_STAGES * PROD_STAGE_BYTES + 16 * PROD_STAGES + 16 + 16 + 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < PROD_STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(bar_tfull + 8 * a, 1);
+            mbar_init(bar_tempty + 8 * a, 4);     // one arrival per epilogue warp
+        }
+        mbar_init(bar_drain, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async;" ::: "memory");
+        prefetch_tmap(&maps.xa);
+        prefetch_tmap(&maps.h);
+        prefetch_tmap(&maps.w1);
+        prefetch_tmap(&maps.w2);
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, PROD_TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot_gen;
+
+    const int n_items = p.meta[META_ITEMS];
+    const int grid = gridDim.x;
+
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            long long fills = 0;
+            bool ok = true;
+            for (int it = blockIdx.x; it < n_items && ok; it += grid) {
+                const int4 item = p.items[it];
+                const int kind = item.x, band = item.y, tile = item.z, e = item.w;
+                const CUtensorMap *amap, *bmap;
+                int b_row0, b_row1, ksteps;
+                if (kind == KIND_G1) {
+                    amap = &maps.xa; bmap = &maps.w1;
+                    b_row0 = e * 2 * p.F + tile * H_TILE;      // gate projection rows
+                    b_row1 = b_row0 + p.F;                     // matching up projection rows
+                    ksteps = p.d / TB_K;
+                } else {
+                    amap = &maps.h; bmap = &maps.w2;
+                    b_row0 = e * p.d + tile * TB_N;
+                    b_row1 = b_row0 + TB_N / 2;
+                    ksteps = p.F / TB_K;
+                    // every first-GEMM tile of this band must have landed in H
+                    ok = wait_global(&p.hcount[band], (unsigned)p.n1, true, p, SITE_TMA_HCOUNT, band);
+                    if (!ok) break;
+                    asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
+                }
+                const int a_row = band * TB_M;
+                for (int ks = 0; ks < ksteps; ++ks) {
+                    ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, p, SITE_TMA_EMPTY, it);
+                    if (!ok) break;
+                    const uint32_t sa = smem_base + stage * PROD_STAGE_BYTES, sb = sa + PROD_A_BYTES;
+                    const uint32_t full = bar_full + 8 * stage;
+                    mbar_arrive_expect_tx(full, PROD_STAGE_BYTES);
+                    tma_load_2d(sa, amap, full, ks * TB_K, a_row);
+                    tma_load_2d(sb, bmap, full, ks * TB_K, b_row0);
+                    tma_load_2d(sb + PROD_B_BYTES / 2, bmap, full, ks * TB_K, b_row1);
+                    ++fills;
+                    if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // give-up path: let the copies already issued land before the shared memory goes away
+                const long long pending = fills < PROD_STAGES ? fills : PROD_STAGES;
+                for (long long q = 1; q <= pending; ++q) {
+                    const long long f = fills - q;                       // index of an issued fill
+                    const int s = (int)(f % PROD_STAGES);
+                    const uint32_t par = (uint32_t)((f / PROD_STAGES) & 1);
+                    const unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(bar_full + 8 * s, par) && globaltimer_ns() - t0 < p.timeout_ns) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer
+        if (lane == 0) {
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int it = blockIdx.x; it < n_items && ok; it += grid) {
+                const int kind = p.items[it].x;
+                const int ksteps = (kind == KIND_G1 ? p.d : p.F) / TB_K;
+                ok = mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, p, SITE_MMA_TEMPTY, it);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * TB_N;
+                for (int ks = 0; ks < ksteps; ++ks) {
+                    ok = mbar_wait(bar_full + 8 * stage, phase, p, SITE_MMA_FULL, it);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sa = smem_base + stage * PROD_STAGE_BYTES, sb = sa + PROD_A_BYTES;
+                    const uint64_t adesc = umma_smem_desc(sa), bdesc = umma_smem_desc(sb);
+#pragma unroll
+                    for (int k = 0; k < TB_K / 16; ++k)      // 16 bf16 = 32 bytes per MMA along K
+                        umma_bf16(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), UMMA_IDESC,
+                                  (ks | k) != 0 ? 1u : 0u);
+                    umma_commit(bar_empty + 8 * stage);       // stage reusable once these MMAs have read it
+                    if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(bar_tfull + 8 * acc);             // accumulator complete
+                acc ^= 1;
+                if (acc == 0) acc_phase ^= 1u;
+            }
+            // all MMAs issued by this thread must have finished before tensor memory is freed
+            umma_commit(bar_drain);
+            const unsigned long long t0 = globaltimer_ns();
+            while (!mbar_try_wait(bar_drain, 0) && globaltimer_ns() - t0 < p.timeout_ns) {}
+        }
+    } else {
+        // ---------------- epilogue: warps 2..5 own tensor-memory lanes 32*(warp % 4) .. +31
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const bool leader = (threadIdx.x == 64);
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int it = blockIdx.x; it < n_items && ok; it += grid) {
+            const int4 item = p.items[it];
+            const int kind = item.x, band = item.y, tile = item.z;
+            ok = mbar_wait(bar_tfull + 8 * acc, acc_phase, p, SITE_EPI_TFULL, it);
+            ok = epilogue_all(ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + (uint32_t)acc * TB_N + ((uint32_t)(q * 32) << 16);
+            const size_t grow = (size_t)band * TB_M + row;
+            if (kind == KIND_G1) {
+                uint16_t *dst = p.H + grow * p.F + (size_t)tile * H_TILE;
+#pragma unroll 1
+                for (int c = 0; c < H_TILE; c += 32) {
+                    uint32_t g[32], u[32];
+                    tmem_ld32(taddr + c, g);
+                    tmem_ld32(taddr + H_TILE + c, u);
+                    tmem_ld_wait();
+                    uint32_t o[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        o[j] = pack_bf16x2(silu_mul(__uint_as_float(g[2 * j]), __uint_as_float(u[2 * j])),
+                                           silu_mul(__uint_as_float(g[2 * j + 1]), __uint_as_float(u[2 * j + 1])));
+                    uint4 *d4 = reinterpret_cast<uint4 *>(dst + c);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) d4[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                }
+            } else {
+                uint16_t *dst = p.Y + grow * p.d + (size_t)tile * TB_N;
+#pragma unroll 1
+                for (int c = 0; c < TB_N; c += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + c, v);
+                    tmem_ld_wait();
+                    uint32_t o[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        o[j] = pack_bf16x2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                    uint4 *d4 = reinterpret_cast<uint4 *>(dst + c);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) d4[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                }
+            }
+            // accumulator buffer can be overwritten by the tile after next
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+            // publish (Section 3.3.1): stores, fence, then one release per tile
+            __threadfence();
+            if (kind == KIND_G1) asm volatile("fence.proxy.async;" ::: "memory");   // H is re-read through TMA
+            bar_sync_epilogue();
+            if (leader) {
+                if (kind == KIND_G1) red_release_add_u32(&p.hcount[band], 1u);
+                else if (raise_flags) st_release_u32(&p.flags[(size_t)band * p.n2 + tile], p.epoch);
+            }
+            acc ^= 1;
+            if (acc == 0) acc_phase ^= 1u;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, PROD_TMEM_COLS);
+    }
+}
+
+}  // namespace moe_ovl
