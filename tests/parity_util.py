@@ -1,0 +1,103 @@
+"""Helpers of the GPU parity tests: run the oracle on the same seeded inputs and compare."""
+import numpy as np
+
+from oracle import value_oracle as VO
+from oracle.index_oracle import build_plan
+from paper_2607_19539_b200 import inputs as I
+
+TOL_REL = 2e-2   # max relative distance on values (bf16 output, fp32 accumulate), stated by the benchmark spec
+
+
+def rel_dist(a, b):
+    """Per-token ||a-b||_2 / max(||b||_2, 1e-6 sqrt(d)) (the 'relative distance' of Section 4.4)."""
+    a = a.astype(np.float64)
+    b = b.astype(np.float64)
+    den = np.maximum(np.linalg.norm(b, axis=-1), 1e-6 * np.sqrt(b.shape[-1]))
+    return np.linalg.norm(a - b, axis=-1) / den
+
+
+def oracle_plan(shape, dsp, mgb=1):
+    return build_plan(dsp.expert_counts.tolist(), dsp.src_rank.tolist(), dsp.src_token.tolist(), shape.R,
+                      shape.self_rank, 128, mgb, shape.d // 256, gate=dsp.gate.tolist(), T=shape.T)
+
+
+def check_indices(shape, dsp, plan, gpu_plan, slot_out, rows_per_rank, segs_per_rank, report):
+    """Bit-exact integer parity: layout, slots, counts, bands, segments, schedule rules."""
+    M = dsp.M
+    assert report.padded_rows == plan.P and report.num_bands == len(plan.bands)
+    assert slot_out[:M].tolist() == plan.slot
+    assert rows_per_rank.tolist() == plan.rows_per_rank
+    assert segs_per_rank.tolist() == plan.segs_per_rank
+    assert gpu_plan["pos"].tolist() == plan.pos
+    assert gpu_plan["group_rows"].reshape(shape.El, shape.R).tolist() == plan.n
+    assert gpu_plan["band_expert"].tolist() == [b.expert for b in plan.bands]
+    assert gpu_plan["band_dest"].tolist() == [b.dest for b in plan.bands]
+    assert gpu_plan["band_valid"].tolist() == [b.valid for b in plan.bands]
+    assert gpu_plan["band_slot0"].tolist() == [b.slot0 for b in plan.bands]
+    assert gpu_plan["sched_band"].tolist() == plan.band_order
+    segs = [[s.first_band, s.nbands, s.dest, s.rows] for s in plan.segments]
+    assert gpu_plan["seg"].tolist() == segs
+    # per-token lists for the weighted reduction
+    kmax = shape.kmax
+    want_slot = np.full((shape.R * shape.T, kmax), -1, np.int32)
+    want_gate = np.zeros((shape.R * shape.T, kmax), np.float32)
+    for tok, (ss, gs) in enumerate(zip(plan.tok_slot, plan.tok_gate)):
+        want_slot[tok, :len(ss)] = ss
+        want_gate[tok, :len(gs)] = gs
+    assert (gpu_plan["tok_slot"] == want_slot).all()
+    assert (gpu_plan["tok_gate"][want_slot >= 0] == want_gate[want_slot >= 0]).all()
+    # issue order: the library interleaves the tiles of neighbouring bands (so that they share weight tiles in
+    # L2) and adds the first-GEMM tiles, so the list is not Algorithm 1's literally; what is unique must hold:
+    items = gpu_plan["item"]
+    n1, n2 = shape.F // 128, shape.d // 256
+    g2 = items[items[:, 0] == 1]
+    g1 = items[items[:, 0] == 0]
+    expect = sorted((b.band, j) for b in plan.bands for j in range(n2))
+    assert sorted(map(tuple, g2[:, 1:3].tolist())) == expect                       # every output tile once
+    assert sorted(map(tuple, g1[:, 1:3].tolist())) == sorted((b.band, j) for b in plan.bands for j in range(n1))
+    band = {b.band: b for b in plan.bands}
+    assert all(band[b].expert == e for _, b, _, e in items.tolist())
+    first_seen = list(dict.fromkeys(g2[:, 1].tolist()))
+    assert first_seen == plan.band_order                                           # bands start in schedule order
+    local = [band[b].local for b in g2[:, 1].tolist()]
+    k = local.index(True) if True in local else len(local)
+    assert not any(local[:k]) and all(local[k:])                                   # rule (i): remote tiles first
+    ex = [e for e in g2[:k, 3].tolist()]
+    runs = [e for i, e in enumerate(ex) if i == 0 or ex[i - 1] != e]
+    assert runs == [e for e in plan.expert_order if any(b.expert == e and not b.local for b in plan.bands)]
+    # a second-GEMM tile is issued after every first-GEMM tile of its band
+    last_g1 = {}
+    for idx, (kind, b, j, e) in enumerate(items.tolist()):
+        if kind == 0:
+            last_g1[b] = idx
+        else:
+            assert idx > last_g1[b]
+
+
+def oracle_values(inp, tokens):
+    sh = inp.shape
+    return VO.forward_tokens(inp.x, inp.expert, inp.gate, inp.w1, inp.w2, sh.El, sh.first_local,
+                             np.asarray(tokens, np.int32))
+
+
+def check_values(shape, dsp, plan, tokens, o_out, o_y, o_yexp, gpu_out_bits, gpu_ret_bits):
+    """out and the returned rows of the given tokens against the oracle, within TOL_REL."""
+    tokens = np.asarray(tokens)
+    got = I.bf16_bits_to_f32(gpu_out_bits[tokens])
+    ref = I.bf16_bits_to_f32(o_out)
+    none = (o_yexp < 0).all(axis=1)
+    assert (gpu_out_bits[tokens][none] == 0).all()                 # no local expert: +0
+    worst = float(rel_dist(got[~none], ref[~none]).max()) if (~none).any() else 0.0
+    assert worst <= TOL_REL, worst
+    # returned rows: ret[r][slot] holds the unscaled expert output of that (token, expert)
+    worst_y = 0.0
+    for s, tok in enumerate(tokens.tolist()):
+        r = tok // shape.T
+        slots = plan.tok_slot[tok]
+        assert len(slots) == int((o_yexp[s] >= 0).sum())
+        for j, slot in enumerate(slots):
+            a = I.bf16_bits_to_f32(gpu_ret_bits[r, slot])[None]
+            b = I.bf16_bits_to_f32(o_y[s, j])[None]
+            worst_y = max(worst_y, float(rel_dist(a, b)[0]))
+    assert worst_y <= TOL_REL, worst_y
+    return worst, worst_y

@@ -1,0 +1,73 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times: indices bit-exact in
+full; values on a seeded sample of tokens the oracle can compute one by one; and properties that hold for
+every row without a CPU FFN."""
+import numpy as np
+import pytest
+
+from paper_2607_19539_b200 import inputs as I
+
+from . import parity_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def sample_tokens(shape, dsp, per_rank, seed=0):
+    """per_rank tokens of every source rank that own at least one local row, plus the tokens owning the
+    first and the last row of every (expert, rank) group."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    tok = dsp.src_rank.astype(np.int64) * shape.T + dsp.src_token
+    picks = []
+    for r in range(shape.R):
+        mine = np.unique(tok[dsp.src_rank == r])
+        picks.append(rng.choice(mine, size=min(per_rank, mine.size), replace=False))
+        for e in range(shape.El):
+            g = tok[(dsp.src_rank == r) & (dsp.row_expert == e)]
+            if g.size:
+                picks.append(np.array([g.min(), g.max()]))
+    return np.unique(np.concatenate(picks)).astype(np.int32)
+
+
+@pytest.mark.parametrize("name,csm,per_rank", [("mixtral", 8, 16), ("fine", 8, 24), ("mixtral_zipf", 8, 8)])
+def test_full_size_parity(name, csm, per_rank):
+    import torch
+    from paper_2607_19539_b200 import binding as B, harness as Hn
+    shape = I.SHAPES[name]
+    inp = I.make_inputs(shape)
+    dsp = I.dispatch(inp)
+    ctx = Hn.make_context(shape, max_rows=dsp.M)
+    prob = Hn.upload(inp, dsp)
+    Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=csm)
+    torch.cuda.synchronize()
+    assert ctx.moe_ovl_query_status()[0] == 0
+    plan = U.oracle_plan(shape, dsp)
+    rep = ctx.moe_ovl_get_report()
+    U.check_indices(shape, dsp, plan, ctx.moe_ovl_get_plan(), prob.slot_out.cpu().numpy(),
+                    prob.rows_per_rank_out.cpu().numpy(), prob.segs_per_rank_out.cpu().numpy(), rep)
+    out = Hn.device_to_bits(prob.out)
+    ret = Hn.device_to_bits(prob.ret)
+    # (1) sampled tokens against the oracle
+    toks = sample_tokens(shape, dsp, per_rank)
+    o = U.oracle_values(inp, toks)
+    worst, worst_y = U.check_values(shape, dsp, plan, toks, *o, out, ret)
+    print(f"{name}: {len(toks)} sampled tokens, max rel dist out {worst:.2e}, returned rows {worst_y:.2e}")
+    # (2) every row: the receive buffer holds exactly the GEMM's output row
+    Y = ctx.moe_ovl_read_buffer(B.BUF_Y, 0, rep.padded_rows)
+    pos, slot = np.asarray(plan.pos), np.asarray(plan.slot)
+    assert (ret[dsp.src_rank, slot] == Y[pos]).all()
+    # (3) every token: out is the gate-weighted sum of its returned rows (recomputed here from the GPU's ret)
+    acc = np.zeros((shape.R * shape.T, shape.d), np.float32)
+    tok = dsp.src_rank.astype(np.int64) * shape.T + dsp.src_token
+    for e in range(shape.El):                                  # ascending expert = accumulation order
+        rows = np.nonzero(dsp.row_expert == e)[0]
+        acc[tok[rows]] += dsp.gate[rows, None] * I.bf16_bits_to_f32(ret[dsp.src_rank[rows], slot[rows]])
+    touched = np.zeros(shape.R * shape.T, bool)
+    touched[tok] = True
+    assert (out[~touched] == 0).all()
+    assert U.rel_dist(I.bf16_bits_to_f32(out[touched]), acc[touched]).max() < 5e-3
+    # (4) the non-overlap baseline gives the same bits
+    prob2 = Hn.upload(inp, dsp, w1=prob.w1, w2=prob.w2)
+    Hn.run(ctx, prob2, mode=B.MODE_NON_OVERLAP)
+    torch.cuda.synchronize()
+    assert ctx.moe_ovl_query_status()[0] == 0
+    assert torch.equal(prob2.out.view(torch.int16), prob.out.view(torch.int16))
+    assert torch.equal(prob2.ret.view(torch.int16), prob.ret.view(torch.int16))

@@ -1,0 +1,213 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded inputs.
+Indices bit-exact; values within 2e-2 max relative distance (bf16 output, fp32 accumulate)."""
+import numpy as np
+import pytest
+
+from paper_2607_19539_b200 import inputs as I
+
+from . import parity_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def _gpu():
+    import torch
+    from paper_2607_19539_b200 import binding as B, harness as Hn
+    return torch, B, Hn
+
+
+def _run_case(shape, mode, csm, shuffle=None, mgb=1, group_bands=0, inp=None, dsp=None):
+    torch, B, Hn = _gpu()
+    inp = inp or I.make_inputs(shape)
+    dsp = dsp or I.dispatch(inp, shuffle_seed=shuffle)
+    ctx = Hn.make_context(shape, max_rows=max(dsp.M, 1), mid_seg_bands=mgb, group_bands=group_bands,
+                          wait_timeout_us=2_000_000)
+    prob = Hn.upload(inp, dsp)
+    Hn.run(ctx, prob, mode=mode, consumer_sm_count=csm)
+    torch.cuda.synchronize()
+    code, detail = ctx.moe_ovl_query_status()
+    assert code == 0, (code, hex(detail))
+    return inp, dsp, ctx, prob
+
+
+SMALL = ["tiny", "tiny_zipf", "small", "small_zipf_rot"]
+
+
+@pytest.mark.parametrize("name", SMALL)
+@pytest.mark.parametrize("mode,csm", [(0, 2), (0, 8), (0, 32), (1, 0)])
+def test_small_shapes_full_parity(name, mode, csm):
+    torch, B, Hn = _gpu()
+    shape = I.SHAPES[name]
+    inp, dsp, ctx, prob = _run_case(shape, mode, csm, shuffle=None if mode else 17)
+    plan = U.oracle_plan(shape, dsp)
+    U.check_indices(shape, dsp, plan, ctx.moe_ovl_get_plan(), prob.slot_out.cpu().numpy(),
+                    prob.rows_per_rank_out.cpu().numpy(), prob.segs_per_rank_out.cpu().numpy(),
+                    ctx.moe_ovl_get_report())
+    toks = np.arange(shape.R * shape.T)
+    o_out, o_y, o_yexp = U.oracle_values(inp, toks)
+    U.check_values(shape, dsp, plan, toks, o_out, o_y, o_yexp, Hn.device_to_bits(prob.out),
+                   Hn.device_to_bits(prob.ret))
+    # rows of ret beyond rows_per_rank are untouched (still the NaN fill of the harness)
+    ret = prob.ret.float().cpu().numpy()
+    for r in range(shape.R):
+        assert not np.isnan(ret[r, :plan.rows_per_rank[r]]).any()
+        assert np.isnan(ret[r, plan.rows_per_rank[r]:]).all()
+
+
+@pytest.mark.parametrize("name,mgb,gb", [("small", 2, 0), ("small_zipf_rot", 3, 2), ("small_zipf_rot", 1, 1)])
+def test_segment_and_group_knobs(name, mgb, gb):
+    torch, B, Hn = _gpu()
+    shape = I.SHAPES[name]
+    inp, dsp, ctx, prob = _run_case(shape, 0, 4, mgb=mgb, group_bands=gb)
+    plan = U.oracle_plan(shape, dsp, mgb=mgb)
+    U.check_indices(shape, dsp, plan, ctx.moe_ovl_get_plan(), prob.slot_out.cpu().numpy(),
+                    prob.rows_per_rank_out.cpu().numpy(), prob.segs_per_rank_out.cpu().numpy(),
+                    ctx.moe_ovl_get_report())
+    toks = np.arange(0, shape.R * shape.T, 7)
+    o = U.oracle_values(inp, toks)
+    U.check_values(shape, dsp, plan, toks, *o, Hn.device_to_bits(prob.out), Hn.device_to_bits(prob.ret))
+
+
+@pytest.mark.parametrize("name", ["tiny", "small_zipf_rot"])
+def test_overlap_equals_non_overlap_bitwise(name):
+    """Both modes run the same GEMM code on the same tiles: any difference is a protocol bug, not rounding."""
+    torch, B, Hn = _gpu()
+    shape = I.SHAPES[name]
+    inp = I.make_inputs(shape)
+    dsp = I.dispatch(inp)
+    ctx = Hn.make_context(shape, max_rows=dsp.M)
+    base = Hn.upload(inp, dsp)
+    Hn.run(ctx, base, mode=B.MODE_NON_OVERLAP)
+    torch.cuda.synchronize()
+    ref_out, ref_ret = base.out.clone(), base.ret.clone()
+    for it in range(20):
+        csm = (2, 4, 8, 16, 32)[it % 5]
+        prob = Hn.upload(inp, dsp, w1=base.w1, w2=base.w2)
+        Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=csm)
+        torch.cuda.synchronize()
+        assert ctx.moe_ovl_query_status()[0] == 0
+        assert torch.equal(prob.out.view(torch.int16), ref_out.view(torch.int16))
+        assert torch.equal(prob.ret.view(torch.int16), ref_ret.view(torch.int16))
+
+
+def test_identity_experts_reproduce_x_bit_exactly():
+    torch, B, Hn = _gpu()
+    shape = I.MoEShape("id", R=3, T=300, Eg=4, k=2, El=2, d=256, F=256, seed=7, self_rank=1)
+    inp = I.make_inputs(shape)
+    d = shape.d
+    w1 = np.zeros((shape.El, 2 * d, d), np.float32)
+    w1[:, :d, d - 1] = 32.0                                  # gate pre-activation = 32: silu(32) = 32 in fp32
+    w1[:, d:, :] = np.eye(d, dtype=np.float32) / 32.0
+    inp.w1 = I.f32_to_bf16_bits(w1)
+    inp.w2 = I.f32_to_bf16_bits(np.broadcast_to(np.eye(d, dtype=np.float32), (shape.El, d, d)).copy())
+    inp.gate[:] = 1.0
+    xf = I.bf16_bits_to_f32(inp.x)
+    xf[..., -1] = 1.0
+    inp.x = I.f32_to_bf16_bits(xf)
+    inp, dsp, ctx, prob = _run_case(shape, 0, 8, inp=inp)
+    out = Hn.device_to_bits(prob.out)
+    m = np.zeros(shape.R * shape.T, int)
+    np.add.at(m, dsp.src_rank * shape.T + dsp.src_token, 1)
+    x_flat = inp.x.reshape(-1, d)
+    assert set(m.tolist()) == {0, 1, 2}
+    assert (out[m == 1] == x_flat[m == 1]).all()
+    assert (out[m == 0] == 0).all()
+    assert (out[m == 2] == I.f32_to_bf16_bits(2.0 * I.bf16_bits_to_f32(x_flat[m == 2]))).all()
+    # the receive buffers hold the dispatched rows themselves, in (expert, source-token) order
+    ret = Hn.device_to_bits(prob.ret)
+    slot = prob.slot_out.cpu().numpy()
+    assert (ret[dsp.src_rank, slot[:dsp.M]] == dsp.x_rows).all()
+
+
+def test_edge_cases_empty_and_degenerate():
+    torch, B, Hn = _gpu()
+    shape = I.MoEShape("edge", R=2, T=64, Eg=4, k=2, El=3, d=256, F=128, seed=3)
+    inp = I.make_inputs(shape)
+    # (a) no rows at all: out is all +0, nothing else written
+    dsp = I.dispatch(inp)
+    empty = I.Dispatched(dsp.x_rows[:0], np.zeros(3, np.int32), dsp.src_rank[:0], dsp.src_token[:0], dsp.gate[:0],
+                         dsp.row_expert[:0])
+    for mode in (0, 1):
+        _, _, ctx, prob = _run_case(shape, mode, 2, inp=inp, dsp=empty)
+        assert (Hn.device_to_bits(prob.out) == 0).all()
+        assert prob.rows_per_rank_out.tolist() == [0, 0] and prob.segs_per_rank_out.tolist() == [0, 0]
+        assert torch.isnan(prob.ret.float()).all()
+        rep = ctx.moe_ovl_get_report()
+        assert rep.num_bands == 0 and rep.num_items == 0 and rep.num_segments == 0
+    # (b) a single row; (c) an expert with no rows between two loaded ones
+    keep_one = np.zeros(dsp.M, bool)
+    keep_one[5] = True
+    keep_gap = dsp.row_expert != 1
+    for keep in (keep_one, keep_gap):
+        sub = I.Dispatched(dsp.x_rows[keep], np.bincount(dsp.row_expert[keep], minlength=3).astype(np.int32),
+                           dsp.src_rank[keep], dsp.src_token[keep], dsp.gate[keep], dsp.row_expert[keep])
+        _, _, ctx, prob = _run_case(shape, 0, 4, inp=inp, dsp=sub)
+        plan = U.oracle_plan(shape, sub)
+        U.check_indices(shape, sub, plan, ctx.moe_ovl_get_plan(), prob.slot_out.cpu().numpy(),
+                        prob.rows_per_rank_out.cpu().numpy(), prob.segs_per_rank_out.cpu().numpy(),
+                        ctx.moe_ovl_get_report())
+        # oracle on routing restricted to the kept rows: drop the other selections by pointing them off-GPU
+        inp2 = I.MoEInputs(shape, inp.x, inp.w1, inp.w2, inp.expert.copy(), inp.gate)
+        kept = set(zip(sub.row_expert.tolist(), sub.src_rank.tolist(), sub.src_token.tolist()))
+        for r in range(shape.R):
+            for t in range(shape.T):
+                for q in range(shape.k):
+                    e = inp2.expert[r, t, q]
+                    if e < shape.El and (int(e), r, t) not in kept:
+                        inp2.expert[r, t, q] = shape.Eg + 5
+        toks = np.arange(shape.R * shape.T)
+        o = U.oracle_values(inp2, toks)
+        U.check_values(shape, sub, plan, toks, *o, Hn.device_to_bits(prob.out), Hn.device_to_bits(prob.ret))
+
+
+def test_bad_routing_is_reported_not_fatal():
+    torch, B, Hn = _gpu()
+    shape = I.SHAPES["tiny"]
+    inp = I.make_inputs(shape)
+    dsp = I.dispatch(inp)
+    ctx = Hn.make_context(shape, max_rows=dsp.M)
+    for kind in ("rank", "dup", "sum"):
+        bad = I.Dispatched(dsp.x_rows, dsp.expert_counts.copy(), dsp.src_rank.copy(), dsp.src_token.copy(), dsp.gate,
+                           dsp.row_expert)
+        if kind == "rank":
+            bad.src_rank[3] = shape.R
+        elif kind == "dup":
+            bad.src_rank[1], bad.src_token[1] = bad.src_rank[0], bad.src_token[0]
+        else:
+            bad.expert_counts[0] -= 1
+        prob = Hn.upload(inp, bad)
+        Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=4)
+        torch.cuda.synchronize()
+        code, detail = ctx.moe_ovl_query_status()
+        assert code == B.ERR_BAD_ROUTING, (kind, code)
+    # the context stays usable
+    prob = Hn.upload(inp, dsp)
+    Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=4)
+    torch.cuda.synchronize()
+    assert ctx.moe_ovl_query_status()[0] == 0
+    # synchronous argument errors
+    with pytest.raises(B.MoeOvlError) as e:
+        Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=0)
+    assert e.value.code == B.ERR_INVALID_ARG
+    with pytest.raises(B.MoeOvlError):
+        Hn.run(ctx, prob, mode=7)
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    torch, B, Hn = _gpu()
+    shape = I.SHAPES["small"]
+    inp = I.make_inputs(shape)
+    dsp = I.dispatch(inp)
+    ctx = Hn.make_context(shape, max_rows=dsp.M, flags=B.FLAG_HOST_STAGING)
+    prob = Hn.upload(inp, dsp)
+    Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=8)
+    torch.cuda.synchronize()
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    hx = pin(dsp.x_rows.view(np.int16))
+    hc, hr, ht, hg = pin(dsp.expert_counts), pin(dsp.src_rank), pin(dsp.src_token), pin(dsp.gate)
+    hout = torch.zeros((shape.R * shape.T, shape.d), dtype=torch.int16).pin_memory()
+    ctx.moe_ovl_expert_return_host(x=hx, expert_counts=hc, src_rank=hr, src_token=ht, gate=hg, w1=prob.w1,
+                                   w2=prob.w2, out=hout, consumer_sm_count=8, mode=B.MODE_OVERLAP)
+    torch.cuda.synchronize()
+    assert ctx.moe_ovl_query_status()[0] == 0
+    assert torch.equal(hout, prob.out.view(torch.int16).cpu())
