@@ -174,7 +174,7 @@ def run_reference(args, shape):
 def workload_config(shape, args):
     return {"workload": f"{shape.name}: {shape.R} simulated ranks x {shape.T} tokens, {shape.Eg} experts "
                         f"top-{shape.k}, {shape.El} local, d={shape.d}, ffn={shape.F}, {shape.router} router",
-            "consumer_sms": args.consumer_sms, "mode": "overlap", "seed": shape.seed,
+            "consumer_sms": args.consumer_sms, "mode": getattr(args, "mode", "overlap"), "seed": shape.seed,
             "l2": "inputs larger than L2 (weights + activations >> 126 MB), no flush",
             "parallelism": f"replicas x{args.gpus}" if args.gpus > 1 else "single GPU"}
 
@@ -189,6 +189,10 @@ def main():
     ap.add_argument("--consumer-sms", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--mode", default="overlap", choices=["overlap", "non_overlap"],
+                    help="non_overlap times the comparison baseline alone (the only mode a profiler that "
+                         "serialises kernels can run: the consumer would wait for a GEMM that is not running)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -240,11 +244,12 @@ def main():
         reports.append(ctx.moe_ovl_get_report())
         return total_ms, per, reports[-1], (t0, t1)
 
-    # ---- headline: overlap mode, K steps
+    # ---- headline: K steps in the chosen mode (overlap unless asked otherwise)
+    head_mode = B.MODE_OVERLAP if args.mode == "overlap" else B.MODE_NON_OVERLAP
     sampler = ClockSampler(local_rank if os.environ.get("CUDA_VISIBLE_DEVICES") is None else 0)
     sampler.start()
     time.sleep(0.3)
-    total_ms, per, rep, (t0, t1) = timed(B.MODE_OVERLAP, args.consumer_sms, args.steps, args.warmup)
+    total_ms, per, rep, (t0, t1) = timed(head_mode, args.consumer_sms, args.steps, args.warmup)
     clocks = sampler.stop(t0, t1)
     secs = D.max_over_ranks(total_ms / 1e3, dev)
     value = step_flops * args.steps * world / secs / 1e12
@@ -253,7 +258,7 @@ def main():
     # is launched on; averaged over a few extra steps
     prod_ms, mover_ms, er_ms, prep_ms, comb_ms = [], [], [], [], []
     for _ in range(min(args.steps, 10)):
-        Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=args.consumer_sms)
+        Hn.run(ctx, prob, mode=head_mode, consumer_sm_count=args.consumer_sms)
         r = ctx.moe_ovl_get_report()
         prod_ms.append(r.ms_producer); mover_ms.append(r.ms_mover); er_ms.append(r.ms_expert_return)
         prep_ms.append(r.ms_prep); comb_ms.append(r.ms_combine)
@@ -267,20 +272,22 @@ def main():
                 "traffic": NCU_PRODUCER_TRAFFIC_BYTES.get(shape.name)}
 
     # ---- comparison: the in-build non-overlap baseline, same steps
-    nov_ms, nov_per, nov_rep, _ = timed(B.MODE_NON_OVERLAP, 0, args.steps, 3)
-    nov_secs = D.max_over_ranks(nov_ms / 1e3, dev)
-    nov_er = []
-    for _ in range(min(args.steps, 10)):
-        Hn.run(ctx, prob, mode=B.MODE_NON_OVERLAP)
-        nov_er.append(ctx.moe_ovl_get_report())
-    non_overlap = {"ms_per_step": nov_secs / args.steps * 1e3,
-                   "tflops": step_flops * args.steps * world / nov_secs / 1e12,
-                   "expert_return_us": statistics.mean(r.ms_expert_return for r in nov_er) * 1e3,
-                   "gemm_us": statistics.mean(r.ms_producer for r in nov_er) * 1e3,
-                   "scatter_us": statistics.mean(r.ms_mover for r in nov_er) * 1e3}
+    non_overlap = None
+    if args.mode == "overlap":
+        nov_ms, nov_per, nov_rep, _ = timed(B.MODE_NON_OVERLAP, 0, args.steps, 3)
+        nov_secs = D.max_over_ranks(nov_ms / 1e3, dev)
+        nov_er = []
+        for _ in range(min(args.steps, 10)):
+            Hn.run(ctx, prob, mode=B.MODE_NON_OVERLAP)
+            nov_er.append(ctx.moe_ovl_get_report())
+        non_overlap = {"ms_per_step": nov_secs / args.steps * 1e3,
+                       "tflops": step_flops * args.steps * world / nov_secs / 1e12,
+                       "expert_return_us": statistics.mean(r.ms_expert_return for r in nov_er) * 1e3,
+                       "gemm_us": statistics.mean(r.ms_producer for r in nov_er) * 1e3,
+                       "scatter_us": statistics.mean(r.ms_mover for r in nov_er) * 1e3}
 
     sweep = []
-    if not args.no_sweep and world == 1:
+    if not args.no_sweep and world == 1 and args.mode == "overlap":
         for csm in (2, 4, 8, 16, 32):
             ms, _, _, _ = timed(B.MODE_OVERLAP, csm, max(3, args.steps // 4), 2)
             ers = []
@@ -298,22 +305,22 @@ def main():
 
     def host_step():
         ctx.moe_ovl_expert_return_host(x=hx, expert_counts=hc, src_rank=hr, src_token=ht, gate=hg, w1=prob.w1,
-                                       w2=prob.w2, out=hout, consumer_sm_count=args.consumer_sms,
-                                       mode=B.MODE_OVERLAP)
-    for _ in range(3):
+                                       w2=prob.w2, out=hout, consumer_sm_count=args.consumer_sms, mode=head_mode)
+    e2e_steps = 0 if args.no_e2e else args.steps
+    for _ in range(3 if e2e_steps else 0):
         host_step()
     torch.cuda.synchronize()
     D.barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for _ in range(args.steps):
+    for _ in range(e2e_steps):
         host_step()
     e1.record()
     torch.cuda.synchronize()
     e2e_secs = D.max_over_ranks(e0.elapsed_time(e1) / 1e3, dev)
     h2d = hx.numel() * 2 + (hc.numel() + hr.numel() + ht.numel()) * 4 + hg.numel() * 4
     d2h = hout.numel() * 2
-    e2e = {"value": step_flops * args.steps * world / e2e_secs / 1e12, "unit": UNIT,
+    e2e = None if args.no_e2e else {"value": step_flops * args.steps * world / e2e_secs / 1e12, "unit": UNIT,
            "ms_per_step": e2e_secs / args.steps * 1e3, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
            "note": "weights stay resident on the device; x, routing metadata in, out back, every step"}
 

@@ -60,6 +60,8 @@ SHAPES: Dict[str, MoEShape] = {
     "mixtral_zipf": MoEShape("mixtral_zipf", R=4, T=4096, Eg=8, k=2, El=2, d=4096, F=14336, router="zipf"),
     "tiny_zipf": MoEShape("tiny_zipf", R=4, T=256, Eg=8, k=2, El=2, d=256, F=512, router="zipf"),
     "fine": MoEShape("fine", R=8, T=8192, Eg=64, k=6, El=8, d=2048, F=1408),
+    # a quarter of the Mixtral-shaped layer's tokens, same weights: small enough for a full profiler capture
+    "mixtral_quarter": MoEShape("mixtral_quarter", R=4, T=1024, Eg=8, k=2, El=2, d=4096, F=14336),
     # mid-size shapes for parity tests (several bands per group, ragged tails)
     "small": MoEShape("small", R=3, T=700, Eg=6, k=2, El=3, d=512, F=384, self_rank=1),
     "small_zipf_rot": MoEShape("small_zipf_rot", R=4, T=900, Eg=8, k=3, El=2, d=256, F=640,
