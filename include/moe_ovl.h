@@ -191,6 +191,40 @@ int moe_ovl_read_buffer(moe_ovl_ctx *ctx, int32_t which, size_t offset, size_t b
 
 int moe_ovl_destroy(moe_ovl_ctx *ctx);
 
+/* Return slots without any allocation (the paper has no counterpart: this entry point
+ * exists for one class of callers of this library, not for the method).
+ *
+ * Some callers can neither call cudaMalloc nor give the library a workspace: code that
+ * runs after the host application has handed every byte of device memory to its own
+ * pool (a cudaMalloc then fails, or forces that pool to give memory back), and code in
+ * latency-critical loops where cudaMalloc's implicit device-wide synchronisation stalls
+ * every stream.  For them this call computes what the plan step of
+ * moe_ovl_expert_return computes for the return path -- slot_out[i], the row of the
+ * owner rank's receive buffer that input row i is delivered to (expert-major, source-
+ * token order), and rows_per_rank_out -- using scratch that is a fixed array inside the
+ * library image instead of a workspace.  It calls no cudaMalloc, cudaFree or any other
+ * allocating routine.
+ *
+ *   expert_counts DEVICE [El], src_rank / src_token DEVICE [M]: as in moe_ovl_args
+ *   slot_out DEVICE [M] (rows with out-of-range metadata get -1), rows_per_rank_out
+ *   DEVICE [R] or NULL; stream: cudaStream_t of the caller.  Asynchronous.
+ *
+ * Limits: El * R <= MOE_OVL_STATIC_MAX_GROUPS and El * R * ceil(T / 32) <=
+ * MOE_OVL_STATIC_MAX_WORDS (the array is 512 KiB, and every GPU that loads the library
+ * holds it until the process exits); larger problems return MOE_OVL_ERR_UNSUPPORTED and
+ * belong to moe_ovl_expert_return with a workspace.
+ * The first call on a device resolves the array's device address (one runtime query,
+ * with that device made current) and should therefore be made before any stream capture
+ * begins on that device.  Every call uses the same array: the kernel clears what it needs
+ * at its start, but two calls that overlap on one GPU (different streams) race on it and
+ * give wrong slots -- keep calls on a device ordered. */
+#define MOE_OVL_STATIC_MAX_GROUPS 1024
+#define MOE_OVL_STATIC_MAX_WORDS 65536
+int moe_ovl_return_slots_static(int32_t device, int32_t num_src_ranks, int32_t tokens_per_rank,
+                                int32_t num_local_experts, int32_t num_rows, const int32_t *expert_counts,
+                                const int32_t *src_rank, const int32_t *src_token, int32_t *slot_out,
+                                int32_t *rows_per_rank_out, void *stream);
+
 const char *moe_ovl_strerror(int code);
 /* cudaError_t of the last failing CUDA call made through this context (0 if none). */
 int moe_ovl_last_cuda_error(const moe_ovl_ctx *ctx);

@@ -26,6 +26,7 @@ EXPORTS = [
     "moe_ovl_workspace_bytes", "moe_ovl_limits", "moe_ovl_create", "moe_ovl_expert_return",
     "moe_ovl_expert_return_host", "moe_ovl_query_status", "moe_ovl_get_report", "moe_ovl_get_plan",
     "moe_ovl_read_buffer", "moe_ovl_destroy", "moe_ovl_strerror", "moe_ovl_last_cuda_error",
+    "moe_ovl_return_slots_static",
 ]
 
 
@@ -106,6 +107,7 @@ def load(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moe_ovl_read_buffer.argtypes = [C.c_void_p, C.c_int32, C.c_size_t, C.c_size_t, C.c_void_p]
     lib.moe_ovl_destroy.argtypes = [C.c_void_p]
     lib.moe_ovl_last_cuda_error.argtypes = [C.c_void_p]
+    lib.moe_ovl_return_slots_static.argtypes = [C.c_int32] * 5 + [C.c_void_p] * 6
     _lib = lib
     return lib
 
@@ -135,6 +137,21 @@ def moe_ovl_limits(cfg: Config):
     if rc != OK:
         raise MoeOvlError(rc, "moe_ovl_limits")
     return int(b.value), int(i.value)
+
+
+def moe_ovl_return_slots_static(*, device: int, num_src_ranks: int, tokens_per_rank: int, num_local_experts: int,
+                                expert_counts, src_rank, src_token, slot_out, rows_per_rank_out=None,
+                                stream=None) -> None:
+    """Return slots computed with the library's built-in scratch array: for callers that cannot allocate
+    device memory (their application owns all of it, or cudaMalloc's synchronisation is unaffordable) and
+    have no workspace to give.  Nothing is allocated here either: outputs are the caller's tensors."""
+    import torch
+    st = torch.cuda.current_stream(device) if stream is None else stream
+    rc = load().moe_ovl_return_slots_static(device, num_src_ranks, tokens_per_rank, num_local_experts,
+                                            int(src_rank.shape[0]), _ptr(expert_counts), _ptr(src_rank),
+                                            _ptr(src_token), _ptr(slot_out), _ptr(rows_per_rank_out), st.cuda_stream)
+    if rc != OK:
+        raise MoeOvlError(rc, "moe_ovl_return_slots_static")
 
 
 def _ptr(t) -> Optional[int]:

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmoe_ovl.so")
-SOURCES = ["moe_ovl.cu"]
+SOURCES = ["moe_ovl.cu", "noalloc.cu"]
 HEADERS = ["common.cuh", "plan.cuh", "producer.cuh", "mover.cuh", os.path.join("..", "..", "include", "moe_ovl.h")]
 
 
