@@ -89,7 +89,7 @@ typedef struct {
     const float *gate;            /* DEVICE [M] fp32 gate weight of (token, expert) */
     const void *w1;               /* DEVICE [El, 2F, d] bf16: rows 0..F-1 gate projection, F..2F-1 up projection */
     const void *w2;               /* DEVICE [El, d, F] bf16 */
-    int32_t consumer_sm_count;    /* SMs dedicated to the consumer (OVERLAP); 1..SMs/2 */
+    int32_t consumer_sm_count;    /* SMs dedicated to the consumer (OVERLAP); 1..SMs/2, rounded up to a whole SM pair */
     int32_t mode;                 /* MOE_OVL_MODE_* */
     void *ret;                    /* DEVICE [R][ret_rows_per_rank, d] bf16: simulated peer receive buffers.
                                      Row s of region r is written iff s < rows_per_rank[r]; the rest is untouched. */
@@ -148,7 +148,8 @@ typedef struct {
     int32_t *band_valid;
     int32_t *band_slot0;
     int32_t *sched_band;      /* [bands] band ids in schedule order */
-    int32_t *item;            /* [items][4] = {kind (0 first GEMM, 1 second), band, tile, expert} in issue order */
+    int32_t *item;            /* [items][4] = {kind (0 first GEMM, 1 second) | expert << 8, band, second band of the
+                                 pair or -1, tile} in issue order */
     int32_t *seg;             /* [segments][4] = {first band, bands, dest rank, rows} in schedule order */
     int32_t *tok_slot;        /* [R*T*min(k,El)] slots of each token's rows, ascending expert, -1 = none */
     float *tok_gate;          /* [R*T*min(k,El)] matching gates */

@@ -62,7 +62,7 @@ struct Params {
     int *slot;            // [M]
     int *band_expert, *band_dest, *band_valid, *band_slot0;   // [max_bands]
     int *sched_band;      // [max_bands]
-    int4 *items;          // [max_items] {kind, band, tile, expert}
+    int4 *items;          // [max_items] {kind | expert << 8, band 0, band 1 or -1, tile}
     int4 *segs;           // [max_bands] {first band, bands, dest, rows}
     int *seg_slot0;       // [max_bands]
     int *tok_slot;        // [R*T*kmax]

@@ -325,10 +325,11 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     int prod_ctas, cons_ctas = 0;
     if (overlap) {
         if (a->consumer_sm_count < 1 || a->consumer_sm_count > ctx->num_sms / 2) return MOE_OVL_ERR_INVALID_ARG;
-        cons_ctas = a->consumer_sm_count;
-        prod_ctas = ctx->num_sms - cons_ctas;       // disjoint SM sets: grids sum to the SM count
+        cons_ctas = (a->consumer_sm_count + 1) & ~1;        // whole SM pairs: the GEMM's CTAs work in pairs
+        prod_ctas = (ctx->num_sms - cons_ctas) & ~1;        // disjoint SM sets: grids sum to the SM count
     } else {
-        prod_ctas = c.producer_sm_limit > 0 ? std::min(c.producer_sm_limit, ctx->num_sms) : ctx->num_sms;
+        prod_ctas = (c.producer_sm_limit > 0 ? std::min(c.producer_sm_limit, ctx->num_sms) : ctx->num_sms) & ~1;
+        if (prod_ctas < 2) return MOE_OVL_ERR_INVALID_ARG;
     }
     CU_CHECK(ctx, cudaSetDevice(c.device));
     cudaStream_t st = static_cast<cudaStream_t>(a->stream);
@@ -336,7 +337,7 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     Params p = make_params(ctx);
     p.M = a->num_rows;
     p.epoch = ++ctx->epoch;
-    p.lag_items = 2 * prod_ctas;
+    p.lag_items = prod_ctas;                        // two rounds of the prod_ctas / 2 CTA pairs
     p.ret_rows_per_rank = a->ret_rows_per_rank;
     p.x = static_cast<const uint16_t *>(a->x);
     p.expert_counts = a->expert_counts; p.src_rank = a->src_rank; p.src_token = a->src_token; p.gate = a->gate;

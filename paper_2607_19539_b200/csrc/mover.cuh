@@ -32,7 +32,9 @@ __device__ __forceinline__ void copy_rows_16B(const uint16_t *src, uint16_t *dst
     for (; v < nvec; v += nthr) __stcs(d + v, __ldcg(s + v));
 }
 
-__global__ void __launch_bounds__(MOVER_THREADS, 1) consumer_kernel(const Params p)
+// Launched as clusters of two so that the consumer takes whole SM pairs and leaves whole pairs to the GEMM,
+// whose CTAs work in pairs.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MOVER_THREADS, 1) consumer_kernel(const Params p)
 {
     extern __shared__ uint8_t unused_smem[];
     __shared__ int s_ok;

@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_build_kernel(Params p, P
     __shared__ int run_start[2 * PLAN_MAX_EXPERTS], run_nb[2 * PLAN_MAX_EXPERTS], run_sb0[2 * PLAN_MAX_EXPERTS + 1];
     __shared__ int run_exp[2 * PLAN_MAX_EXPERTS];
     __shared__ int segs_per_rank[PLAN_MAX_GROUPS];
-    __shared__ int s_nsb, s_items;
+    __shared__ int s_nsb;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
     const int G = p.El * p.R;
@@ -174,7 +174,9 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_build_kernel(Params p, P
             }
             run_nb[run] = spos - run_start[run];
             run_sb0[run] = sbcount;
-            sbcount += (run_nb[run] + p.group_bands - 1) / p.group_bands;
+            // super-bands are made of whole band pairs (the GEMM works on two bands at a time)
+            const int pairs = (run_nb[run] + 1) / 2, pairs_per_sb = max(1, p.group_bands / 2);
+            sbcount += (pairs + pairs_per_sb - 1) / pairs_per_sb;
         }
         run_sb0[2 * El] = sbcount;
         s_nsb = sbcount;
@@ -213,34 +215,36 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_build_kernel(Params p, P
         if (p.segs_per_rank_out) p.segs_per_rank_out[r] = segs_per_rank[r];
     for (int run = tid; run < 2 * El; run += blockDim.x) {
         const int nsb = run_sb0[run + 1] - run_sb0[run];
+        const int pairs = (run_nb[run] + 1) / 2;
         for (int q = 0; q < nsb; ++q) {
-            const int base = run_nb[run] / nsb, rem = run_nb[run] % nsb;
+            // spread the run's band pairs evenly; only the run's last super-band can end on a single band
+            const int base = pairs / nsb, rem = pairs % nsb;
             const int sb = run_sb0[run] + q;
-            sc.sb_start[sb] = run_start[run] + q * base + min(q, rem);
-            sc.sb_nb[sb] = base + (q < rem ? 1 : 0);
+            const int pair0 = q * base + min(q, rem), npairs = base + (q < rem ? 1 : 0);
+            sc.sb_start[sb] = run_start[run] + 2 * pair0;
+            sc.sb_nb[sb] = min(2 * npairs, run_nb[run] - 2 * pair0);
             sc.sb_expert[sb] = run_exp[run];
         }
     }
     __syncthreads();
 
-    // F: issue order of tile blocks.  Inside a super-band the tile index is the outer loop and the band the
-    //    inner one, so that the CTAs working side by side share a weight tile.  The second-GEMM block of a
-    //    super-band is issued lag_items items after its first-GEMM block, so that its input is normally
-    //    complete when a CTA reaches it.
+    // F: issue order of tile blocks.  An item is a pair of bands times one tile.  Inside a super-band the tile
+    //    index is the outer loop and the band pair the inner one, so that the CTA pairs working side by side
+    //    share a weight tile.  The second-GEMM block of a super-band is issued lag_items items after its
+    //    first-GEMM block, so that its input is normally complete when a CTA pair reaches it.
     if (tid == 0) {
         const int nsb = s_nsb;
         int ng1 = 0, off = 0;
         for (int ng2 = 0; ng2 < nsb; ++ng2) {
             while (ng1 < nsb && (ng1 <= ng2 || off - sc.sb_g1end[ng2] < p.lag_items)) {
                 sc.sb_g1off[ng1] = off;
-                off += sc.sb_nb[ng1] * p.n1;
+                off += ((sc.sb_nb[ng1] + 1) / 2) * p.n1;
                 sc.sb_g1end[ng1] = off;
                 ++ng1;
             }
             sc.sb_g2off[ng2] = off;
-            off += sc.sb_nb[ng2] * p.n2;
+            off += ((sc.sb_nb[ng2] + 1) / 2) * p.n2;
         }
-        s_items = off;
         p.meta[META_ITEMS] = off;
     }
     __syncthreads();
@@ -248,11 +252,16 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_build_kernel(Params p, P
     // G: the item list
     for (int sb = 0; sb < s_nsb; ++sb) {
         const int start = sc.sb_start[sb], cnt = sc.sb_nb[sb], e = sc.sb_expert[sb];
+        const int np = (cnt + 1) / 2;
         const int o1 = sc.sb_g1off[sb], o2 = sc.sb_g2off[sb];
-        for (int idx = tid; idx < cnt * p.n1; idx += blockDim.x)
-            p.items[o1 + idx] = make_int4(KIND_G1, p.sched_band[start + idx % cnt], idx / cnt, e);
-        for (int idx = tid; idx < cnt * p.n2; idx += blockDim.x)
-            p.items[o2 + idx] = make_int4(KIND_G2, p.sched_band[start + idx % cnt], idx / cnt, e);
+        for (int idx = tid; idx < np * (p.n1 + p.n2); idx += blockDim.x) {
+            const bool g1 = idx < np * p.n1;
+            const int k = g1 ? idx : idx - np * p.n1;
+            const int pair = k % np, tile = k / np;
+            const int b0 = p.sched_band[start + 2 * pair];
+            const int b1 = 2 * pair + 1 < cnt ? p.sched_band[start + 2 * pair + 1] : -1;
+            p.items[(g1 ? o1 : o2) + k] = make_int4((g1 ? KIND_G1 : KIND_G2) | (e << 8), b0, b1, tile);
+        }
     }
 }
 

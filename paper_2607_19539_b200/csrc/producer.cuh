@@ -3,17 +3,22 @@
 // flag per finished output tile (Section 3.3.1: rank-wide persistent GEMM with
 // tile-level signalling in the epilogue).
 //
-// sm_100a design (the paper's is CUTLASS on A100): warp-specialised CTA, one per SM.
-//   warp 0     TMA loads (cp.async.bulk.tensor, 128-byte swizzle) into a 4-stage ring
-//   warp 1     one thread issues tcgen05.mma (bf16 x bf16 -> fp32, M=128 N=256 K=16),
-//              accumulators in tensor memory, double buffered (2 x 256 columns)
+// sm_100a design (the paper's is CUTLASS on A100): warp-specialised CTAs, one per SM, launched
+// as clusters of two that share every MMA (cta_group::2): the pair computes a 256 x 256 tile,
+// each CTA holding its own 128 rows of A and only HALF of the B tile, which cuts the operand
+// traffic from L2 per SM by a third against a single-CTA 128 x 256 tile.
+//   warp 0     TMA loads (cp.async.bulk.tensor, 128-byte swizzle) into a 6-stage ring; both
+//              CTAs' loads complete on the leader CTA's mbarrier
+//   warp 1     in the leader CTA one thread issues tcgen05.mma (bf16 x bf16 -> fp32, M=256
+//              N=256 K=16); accumulators in tensor memory, double buffered (2 x 256 columns)
 //   warps 2-5  epilogue: tcgen05.ld -> fp32 math -> bf16 -> global, then publish
-// A schedule item is one 128-row band times one tile:
-//   first GEMM   A = Xa[band], B = 128 gate rows and 128 up rows of W1 -> one N=256
-//                accumulator; the epilogue pairs column c with c+128: h = silu(g) * u,
-//                128 columns of H; then hcount[band] += 1 (release)
-//   second GEMM  waits until hcount[band] == F/128, A = H[band], B = 256 rows of W2,
-//                writes 256 columns of Y; then flag[band][tile] = epoch (release)
+// A schedule item is a pair of 128-row bands of one expert (the second may be absent) times
+// one tile; CTA rank r of the cluster owns band r of the pair:
+//   first GEMM   A = Xa[band]; B = 128 gate rows of W1 (held by rank 0) and the matching 128
+//                up rows (rank 1) -> one N=256 accumulator; the epilogue pairs column c with
+//                c+128: h = silu(g) * u, 128 columns of H; then hcount[band] += 1 (release)
+//   second GEMM  waits until hcount[band] == F/128, A = H[band], B = 256 rows of W2 (128 per
+//                rank), writes 256 columns of Y; then flag[band][tile] = epoch (release)
 // Every wait is bounded; on a give-up the CTA records a status, drains its copies,
 // frees its tensor memory and returns.
 #pragma once
@@ -24,9 +29,9 @@
 
 namespace moe_ovl {
 
-constexpr int PROD_STAGES = 4;
-constexpr int PROD_A_BYTES = TB_M * TB_K * 2;          // 16 KiB
-constexpr int PROD_B_BYTES = TB_N * TB_K * 2;          // 32 KiB
+constexpr int PROD_STAGES = 6;
+constexpr int PROD_A_BYTES = TB_M * TB_K * 2;          // 16 KiB: this CTA's 128 rows of A
+constexpr int PROD_B_BYTES = (TB_N / 2) * TB_K * 2;    // 16 KiB: this CTA's half of the B tile
 constexpr int PROD_STAGE_BYTES = PROD_A_BYTES + PROD_B_BYTES;
 constexpr int PROD_THREADS = 192;
 constexpr int PROD_TMEM_COLS = 512;
@@ -78,11 +83,36 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const P
     }
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrivals on a barrier that may live in the peer CTA (shared::cluster address)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+// Tile load into this CTA's shared memory; the bytes are counted on a barrier that may be the peer CTA's.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t cluster_bar, int x, int y)
 {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(cluster_bar), "r"(x), "r"(y)
         : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap *map)
@@ -95,29 +125,38 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
 {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
                  : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
 {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]; bf16 inputs, fp32 accumulate
+// D[tmem] (+)= A[smem] * B[smem] over the CTA pair; bf16 inputs, fp32 accumulate
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                           uint32_t accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// The mbarrier gets one arrival when every MMA issued so far by this thread has finished.
-__device__ __forceinline__ void umma_commit(uint32_t bar)
+// The mbarrier at this offset gets one arrival in BOTH CTAs of the pair when every MMA issued so far by this
+// thread has finished.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"((uint16_t)3)
+        : "memory");
+}
+// Same, this CTA's barrier only.
+__device__ __forceinline__ void umma_commit_self(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                  : "memory");
 }
 // 32 lanes x 32 columns of fp32: thread t of the warp gets lane (base lane + t), 32 consecutive columns
@@ -148,9 +187,9 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr)
     d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
     return d;
 }
-// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N=256, M=128.
+// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N=256, M=256 over the CTA pair.
 constexpr uint32_t UMMA_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TB_N >> 3) << 17) |
-                                ((uint32_t)(TB_M >> 4) << 24);
+                                ((uint32_t)((2 * TB_M) >> 4) << 24);
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
@@ -182,7 +221,7 @@ struct ProducerMaps {
     CUtensorMap xa, h, w1, w2;   // all 2-D bf16 row-major, box 64 x 128, 128-byte swizzle
 };
 
-__global__ void __launch_bounds__(PROD_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PROD_THREADS, 1)
 producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const int raise_flags)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -197,15 +236,18 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
         smem_gen + PROD_STAGES * PROD_STAGE_BYTES + 16 * PROD_STAGES + 16 + 16 + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();          // 0 = leader: owns the barriers the pair synchronises on
+    // shared::cluster addresses of the leader's barriers (for rank 0 these are its own)
+    const uint32_t lead_full = map_to_cta(bar_full, 0), lead_tempty = map_to_cta(bar_tempty, 0);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < PROD_STAGES; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_full + 8 * s, 1);       // the leader's TMA thread arrives, expecting both CTAs' bytes
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tfull + 8 * a, 1);
-            mbar_init(bar_tempty + 8 * a, 4);     // one arrival per epilogue warp
+            mbar_init(bar_tempty + 8 * a, 8);     // one arrival per epilogue warp of both CTAs
         }
         mbar_init(bar_drain, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -218,33 +260,34 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
     if (warp == 1) tmem_alloc(tmem_slot, PROD_TMEM_COLS);
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();                           // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_gen;
 
     const int n_items = p.meta[META_ITEMS];
-    const int grid = gridDim.x;
+    const int first = blockIdx.x >> 1, stride = gridDim.x >> 1;     // items are dealt to clusters
 
     if (warp == 0) {
-        // ---------------- TMA producer
+        // ---------------- TMA producer (both CTAs)
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
             long long fills = 0;
             bool ok = true;
-            for (int it = blockIdx.x; it < n_items && ok; it += grid) {
-                const int4 item = p.items[it];
-                const int kind = item.x, band = item.y, tile = item.z, e = item.w;
+            for (int it = first; it < n_items && ok; it += stride) {
+                const int4 item = p.items[it];       // {kind | expert << 8, band 0, band 1 or -1, tile}
+                const int kind = item.x & 0xff, e = item.x >> 8, tile = item.w;
+                const int band = (rank == 0 || item.z < 0) ? item.y : item.z;
                 const CUtensorMap *amap, *bmap;
-                int b_row0, b_row1, ksteps;
+                int b_row, ksteps;
                 if (kind == KIND_G1) {
                     amap = &maps.xa; bmap = &maps.w1;
-                    b_row0 = e * 2 * p.F + tile * H_TILE;      // gate projection rows
-                    b_row1 = b_row0 + p.F;                     // matching up projection rows
+                    // rank 0 holds the gate-projection rows of the tile, rank 1 the matching up-projection rows
+                    b_row = e * 2 * p.F + tile * H_TILE + (int)rank * p.F;
                     ksteps = p.d / TB_K;
                 } else {
                     amap = &maps.h; bmap = &maps.w2;
-                    b_row0 = e * p.d + tile * TB_N;
-                    b_row1 = b_row0 + TB_N / 2;
+                    b_row = e * p.d + tile * TB_N + (int)rank * (TB_N / 2);
                     ksteps = p.F / TB_K;
                     // every first-GEMM tile of this band must have landed in H
                     ok = wait_global(&p.hcount[band], (unsigned)p.n1, true, p, SITE_TMA_HCOUNT, band);
@@ -256,16 +299,19 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, p, SITE_TMA_EMPTY, it);
                     if (!ok) break;
                     const uint32_t sa = smem_base + stage * PROD_STAGE_BYTES, sb = sa + PROD_A_BYTES;
-                    const uint32_t full = bar_full + 8 * stage;
-                    mbar_arrive_expect_tx(full, PROD_STAGE_BYTES);
+                    const uint32_t full = lead_full + 8 * stage;
+                    // The leader announces the bytes of both CTAs.  The peer's bytes may land before this
+                    // arrival; the phase still cannot complete early because the arrival itself is pending.
+                    // The peer can only refill a stage after the leader's MMAs have consumed (hence completed)
+                    // its previous phase, so bytes never leak into the wrong phase.
+                    if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * PROD_STAGE_BYTES);
                     tma_load_2d(sa, amap, full, ks * TB_K, a_row);
-                    tma_load_2d(sb, bmap, full, ks * TB_K, b_row0);
-                    tma_load_2d(sb + PROD_B_BYTES / 2, bmap, full, ks * TB_K, b_row1);
+                    tma_load_2d(sb, bmap, full, ks * TB_K, b_row);
                     ++fills;
                     if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
-            if (!ok) {
+            if (!ok && rank == 0) {
                 // give-up path: let the copies already issued land before the shared memory goes away
                 const long long pending = fills < PROD_STAGES ? fills : PROD_STAGES;
                 for (long long q = 1; q <= pending; ++q) {
@@ -278,13 +324,13 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer
-        if (lane == 0) {
+        // ---------------- MMA issuer (leader CTA only; its MMAs run on both SMs of the pair)
+        if (lane == 0 && rank == 0) {
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            for (int it = blockIdx.x; it < n_items && ok; it += grid) {
-                const int kind = p.items[it].x;
+            for (int it = first; it < n_items && ok; it += stride) {
+                const int kind = p.items[it].x & 0xff;
                 const int ksteps = (kind == KIND_G1 ? p.d : p.F) / TB_K;
                 ok = mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, p, SITE_MMA_TEMPTY, it);
                 if (!ok) break;
@@ -300,16 +346,16 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     for (int k = 0; k < TB_K / 16; ++k)      // 16 bf16 = 32 bytes per MMA along K
                         umma_bf16(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), UMMA_IDESC,
                                   (ks | k) != 0 ? 1u : 0u);
-                    umma_commit(bar_empty + 8 * stage);       // stage reusable once these MMAs have read it
+                    umma_commit_pair(bar_empty + 8 * stage);  // both CTAs may refill the stage once it has been read
                     if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit(bar_tfull + 8 * acc);             // accumulator complete
+                umma_commit_pair(bar_tfull + 8 * acc);        // accumulator complete, in both CTAs
                 acc ^= 1;
                 if (acc == 0) acc_phase ^= 1u;
             }
             // all MMAs issued by this thread must have finished before tensor memory is freed
-            umma_commit(bar_drain);
+            umma_commit_self(bar_drain);
             const unsigned long long t0 = globaltimer_ns();
             while (!mbar_try_wait(bar_drain, 0) && globaltimer_ns() - t0 < p.timeout_ns) {}
         }
@@ -321,16 +367,20 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int it = blockIdx.x; it < n_items && ok; it += grid) {
+        for (int it = first; it < n_items && ok; it += stride) {
             const int4 item = p.items[it];
-            const int kind = item.x, band = item.y, tile = item.z;
+            const int kind = item.x & 0xff, tile = item.w;
+            const bool present = (rank == 0) || item.z >= 0;        // the pair's second band may be absent
+            const int band = rank == 0 ? item.y : item.z;
             ok = mbar_wait(bar_tfull + 8 * acc, acc_phase, p, SITE_EPI_TFULL, it);
             ok = epilogue_all(ok);
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + (uint32_t)acc * TB_N + ((uint32_t)(q * 32) << 16);
-            const size_t grow = (size_t)band * TB_M + row;
-            if (kind == KIND_G1) {
+            const size_t grow = (size_t)(present ? band : 0) * TB_M + row;
+            if (!present) {
+                // nothing to store: the accumulator of an absent band is discarded
+            } else if (kind == KIND_G1) {
                 uint16_t *dst = p.H + grow * p.F + (size_t)tile * H_TILE;
 #pragma unroll 1
                 for (int c = 0; c < H_TILE; c += 32) {
@@ -363,15 +413,18 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     for (int j = 0; j < 4; ++j) d4[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
                 }
             }
-            // accumulator buffer can be overwritten by the tile after next
+            // accumulator buffer can be overwritten by the tile after next: tell the leader's MMA thread
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+            if (lane == 0) {
+                if (rank == 0) mbar_arrive(bar_tempty + 8 * acc);
+                else mbar_arrive_cluster(lead_tempty + 8 * acc);
+            }
             // publish (Section 3.3.1): stores, fence, then one release per tile
             __threadfence();
             if (kind == KIND_G1) asm volatile("fence.proxy.async;" ::: "memory");   // H is re-read through TMA
             bar_sync_epilogue();
-            if (leader) {
+            if (leader && present) {
                 if (kind == KIND_G1) red_release_add_u32(&p.hcount[band], 1u);
                 else if (raise_flags) st_release_u32(&p.flags[(size_t)band * p.n2 + tile], p.epoch);
             }
@@ -382,6 +435,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
 
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();       // the peer no longer reads this CTA's shared memory or signals its barriers
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();

@@ -48,7 +48,14 @@ def check_indices(shape, dsp, plan, gpu_plan, slot_out, rows_per_rank, segs_per_
     assert (gpu_plan["tok_gate"][want_slot >= 0] == want_gate[want_slot >= 0]).all()
     # issue order: the library interleaves the tiles of neighbouring bands (so that they share weight tiles in
     # L2) and adds the first-GEMM tiles, so the list is not Algorithm 1's literally; what is unique must hold:
-    items = gpu_plan["item"]
+    # an item is {kind | expert << 8, band, second band of the pair or -1, tile}: expand pairs to single bands
+    raw = gpu_plan["item"]
+    rows = []
+    for x, b0, b1, tile in raw.tolist():
+        rows.append((x & 0xff, b0, tile, x >> 8))
+        if b1 >= 0:
+            rows.append((x & 0xff, b1, tile, x >> 8))
+    items = np.asarray(rows, np.int64).reshape(-1, 4)
     n1, n2 = shape.F // 128, shape.d // 256
     g2 = items[items[:, 0] == 1]
     g1 = items[items[:, 0] == 0]
