@@ -27,7 +27,7 @@ constexpr int ERR_BAD_ROUTING = -6;
 // wait sites reported in the high bits of the status detail
 enum : long long {
     SITE_TMA_EMPTY = 1, SITE_TMA_HCOUNT, SITE_MMA_FULL, SITE_MMA_TEMPTY, SITE_EPI_TFULL, SITE_CONS_FLAG,
-    SITE_MMA_DRAIN, SITE_TMA_DRAIN,
+    SITE_MMA_DRAIN, SITE_TMA_DRAIN, SITE_CLAIM, SITE_SCHED_GO,
     SITE_ROW_RANGE = 16, SITE_ROW_DUP, SITE_COUNT_SUM, SITE_TOK_OVERFLOW
 };
 
@@ -67,6 +67,7 @@ struct Params {
     int *seg_slot0;       // [max_bands]
     int *tok_slot;        // [R*T*kmax]
     float *tok_gate;      // [R*T*kmax]
+    int *next_item;       // schedule items claimed so far (GEMM CTA pairs take them in order)
     unsigned *hcount;     // [max_bands] first-GEMM tiles finished per band
     unsigned *flags;      // [max_bands*n2] epoch of the call that finished the tile
     int *meta;            // [META_COUNT]
@@ -114,24 +115,27 @@ __device__ __forceinline__ void report_error(int *status, int code, long long si
     atomicExch(&status[ST_ABORT], 1);
 }
 
-// Spin until *p == want (exact) or *p >= want (at_least), giving up at the deadline
-// or when another waiter has aborted.  Returns false on give-up.
+// Poll until *p == want (exact) or *p >= want (at_least), giving up at the deadline or when another waiter
+// has aborted.  Returns false on give-up.  Between polls the thread sleeps, backing off up to max_sleep_ns:
+// a waiter that spins hot takes power and L2 bandwidth from the GEMM it is waiting for.
 __device__ __forceinline__ bool wait_global(const unsigned *p, unsigned want, bool at_least, const Params &prm,
-                                            long long site, long long index)
+                                            long long site, long long index, unsigned max_sleep_ns = 256)
 {
     unsigned v = ld_acquire_u32(p);
     if (at_least ? (v >= want) : (v == want)) return true;
     const unsigned long long t0 = globaltimer_ns();
+    unsigned sleep_ns = 32;
     for (unsigned it = 1;; ++it) {
+        __nanosleep(sleep_ns);
+        if (sleep_ns < max_sleep_ns) sleep_ns *= 2;
         v = ld_acquire_u32(p);
         if (at_least ? (v >= want) : (v == want)) return true;
-        if ((it & 63u) == 0) {
+        if ((it & 15u) == 0) {
             if (ld_volatile_s32(&prm.status[ST_ABORT])) return false;
             if (globaltimer_ns() - t0 > prm.timeout_ns) {
                 report_error(prm.status, ERR_TIMEOUT, site, index);
                 return false;
             }
-            __nanosleep(64);
         }
     }
 }

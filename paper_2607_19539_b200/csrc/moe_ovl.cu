@@ -29,7 +29,7 @@ inline size_t align_up(size_t v, size_t a = ALIGN) { return (v + a - 1) / a * a;
 struct Layout {
     // offsets into the workspace, in bytes
     size_t Xa, H, Y;
-    size_t zero_begin, bitmap, hcount, status, zero_end;   // cleared to 0 at the start of every call
+    size_t zero_begin, bitmap, hcount, status, next_item, zero_end;   // cleared to 0 at the start of every call
     size_t tok_slot, tok_slot_bytes;                       // filled with -1 at the start of every call
     size_t wordpfx, group_rows, group_start, group_slot, pos, slot;
     size_t band_expert, band_dest, band_valid, band_slot0, sched_band, items, segs, seg_slot0;
@@ -82,6 +82,7 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->bitmap = take((size_t)G * L->words * 4);
     L->hcount = take((size_t)L->max_bands * 4);
     L->status = take(ST_COUNT * 4);
+    L->next_item = take(4);
     L->zero_end = off;
     L->tok_slot_bytes = ntok * L->kmax * 4;
     L->tok_slot = take(L->tok_slot_bytes);
@@ -189,6 +190,7 @@ Params make_params(moe_ovl_ctx *ctx)
     p.sched_band = at<int>(ctx, L.sched_band); p.items = at<int4>(ctx, L.items); p.segs = at<int4>(ctx, L.segs);
     p.seg_slot0 = at<int>(ctx, L.seg_slot0); p.tok_slot = at<int>(ctx, L.tok_slot);
     p.tok_gate = at<float>(ctx, L.tok_gate); p.hcount = at<unsigned>(ctx, L.hcount);
+    p.next_item = at<int>(ctx, L.next_item);
     p.flags = at<unsigned>(ctx, L.flags); p.meta = at<int>(ctx, L.meta); p.status = at<int>(ctx, L.status);
     return p;
 }

@@ -49,7 +49,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MOVER_THREADS, 1) co
             const unsigned *f = p.flags + (size_t)seg.x * p.n2;
             bool ok = true;
             for (int i = lane; i < nflags && ok; i += 32)
-                ok = wait_global(f + i, p.epoch, false, p, SITE_CONS_FLAG, (long long)seg.x * p.n2 + i);
+                ok = wait_global(f + i, p.epoch, false, p, SITE_CONS_FLAG, (long long)seg.x * p.n2 + i, 2048);
             ok = __all_sync(0xffffffffu, ok);
             if (lane == 0) s_ok = ok ? 1 : 0;
         }

@@ -12,6 +12,10 @@
 //   warp 1     in the leader CTA one thread issues tcgen05.mma (bf16 x bf16 -> fp32, M=256
 //              N=256 K=16); accumulators in tensor memory, double buffered (2 x 256 columns)
 //   warps 2-5  epilogue: tcgen05.ld -> fp32 math -> bf16 -> global, then publish
+//   warp 6     scheduler (leader CTA): claims the next schedule item with an atomic counter, one
+//              item ahead of the TMA warp, and hands it to every role of both CTAs through a
+//              small ring in shared memory.  Items are claimed in schedule order, so the
+//              remote-first order holds and every dependency still points to an earlier claim.
 // A schedule item is a pair of 128-row bands of one expert (the second may be absent) times
 // one tile; CTA rank r of the cluster owns band r of the pair:
 //   first GEMM   A = Xa[band]; B = 128 gate rows of W1 (held by rank 0) and the matching 128
@@ -33,9 +37,10 @@ constexpr int PROD_STAGES = 6;
 constexpr int PROD_A_BYTES = TB_M * TB_K * 2;          // 16 KiB: this CTA's 128 rows of A
 constexpr int PROD_B_BYTES = (TB_N / 2) * TB_K * 2;    // 16 KiB: this CTA's half of the B tile
 constexpr int PROD_STAGE_BYTES = PROD_A_BYTES + PROD_B_BYTES;
-constexpr int PROD_THREADS = 192;
+constexpr int PROD_THREADS = 224;                      // TMA, MMA, 4 epilogue warps, scheduler
+constexpr int PROD_RING = 16;                          // claimed-item ring; roles are never more than 5 items apart
 constexpr int PROD_TMEM_COLS = 512;
-constexpr int PROD_SMEM_BYTES = PROD_STAGES * PROD_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int PROD_SMEM_BYTES = PROD_STAGES * PROD_STAGE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers, ring*/;
 
 // ------------------------------------------------------------------ PTX wrappers
 
@@ -65,14 +70,29 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
+// Same test with acquire semantics at cluster scope: for barriers the peer CTA arrives on.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // Bounded wait on an mbarrier phase.  False = gave up (deadline, or another waiter aborted).
+template <bool kClusterScope = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Params &prm, long long site,
                                           long long index)
 {
-    if (mbar_try_wait(bar, parity)) return true;
+    auto test = [&]() { return kClusterScope ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
+    if (test()) return true;
     const unsigned long long t0 = globaltimer_ns();
     for (unsigned it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (test()) return true;
         if ((it & 255u) == 0) {
             if (ld_volatile_s32(&prm.status[ST_ABORT])) return false;
             if (globaltimer_ns() - t0 > prm.timeout_ns) {
@@ -231,9 +251,14 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
     const uint32_t bar_full = bars, bar_empty = bars + 8 * PROD_STAGES;
     const uint32_t bar_tfull = bars + 16 * PROD_STAGES, bar_tempty = bar_tfull + 16, bar_drain = bar_tempty + 16;
     const uint32_t tmem_slot = bar_drain + 8;
+    const uint32_t bar_go = tmem_slot + 8;                         // TMA thread -> scheduler: "started an item"
+    const uint32_t bar_ring = bar_go + 8;                          // PROD_RING barriers: slot filled
+    const uint32_t ring = bar_ring + 8 * PROD_RING;                // PROD_RING claimed item indices
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    volatile uint32_t *tmem_slot_gen = reinterpret_cast<volatile uint32_t *>(
-        smem_gen + PROD_STAGES * PROD_STAGE_BYTES + 16 * PROD_STAGES + 16 + 16 + 8);
+    const uint32_t bars_off = PROD_STAGES * PROD_STAGE_BYTES;
+    volatile uint32_t *tmem_slot_gen = reinterpret_cast<volatile uint32_t *>(smem_gen + (tmem_slot - smem_base));
+    volatile int *ring_gen = reinterpret_cast<volatile int *>(smem_gen + (ring - smem_base));
+    (void)bars_off;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();          // 0 = leader: owns the barriers the pair synchronises on
@@ -250,6 +275,8 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             mbar_init(bar_tempty + 8 * a, 8);     // one arrival per epilogue warp of both CTAs
         }
         mbar_init(bar_drain, 1);
+        mbar_init(bar_go, 1);
+        for (int s = 0; s < PROD_RING; ++s) mbar_init(bar_ring + 8 * s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async;" ::: "memory");
         prefetch_tmap(&maps.xa);
@@ -265,7 +292,13 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
     const uint32_t tmem_base = *tmem_slot_gen;
 
     const int n_items = p.meta[META_ITEMS];
-    const int first = blockIdx.x >> 1, stride = gridDim.x >> 1;     // items are dealt to clusters
+    // n-th item of this cluster: wait until the scheduler has filled ring slot n % PROD_RING, then read it.
+    // Returns n_items (or more) when the schedule is exhausted, -1 on a give-up.
+    auto claimed = [&](int n) -> int {
+        const int slot = n % PROD_RING;
+        if (!mbar_wait<true>(bar_ring + 8 * slot, (uint32_t)(n / PROD_RING) & 1u, p, SITE_CLAIM, n)) return -1;
+        return ring_gen[slot];
+    };
 
     if (warp == 0) {
         // ---------------- TMA producer (both CTAs)
@@ -274,7 +307,10 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             uint32_t phase = 0;
             long long fills = 0;
             bool ok = true;
-            for (int it = first; it < n_items && ok; it += stride) {
+            for (int n = 0; ok; ++n) {
+                const int it = claimed(n);
+                if (it < 0 || it >= n_items) { ok = it >= 0; break; }
+                if (rank == 0) mbar_arrive(bar_go);  // lets the scheduler claim the item after this one
                 const int4 item = p.items[it];       // {kind | expert << 8, band 0, band 1 or -1, tile}
                 const int kind = item.x & 0xff, e = item.x >> 8, tile = item.w;
                 const int band = (rank == 0 || item.z < 0) ? item.y : item.z;
@@ -329,10 +365,12 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            for (int it = first; it < n_items && ok; it += stride) {
+            for (int n = 0; ok; ++n) {
+                const int it = claimed(n);
+                if (it < 0 || it >= n_items) break;
                 const int kind = p.items[it].x & 0xff;
                 const int ksteps = (kind == KIND_G1 ? p.d : p.F) / TB_K;
-                ok = mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, p, SITE_MMA_TEMPTY, it);
+                ok = mbar_wait<true>(bar_tempty + 8 * acc, acc_phase ^ 1u, p, SITE_MMA_TEMPTY, it);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * TB_N;
@@ -359,6 +397,23 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             const unsigned long long t0 = globaltimer_ns();
             while (!mbar_try_wait(bar_drain, 0) && globaltimer_ns() - t0 < p.timeout_ns) {}
         }
+    } else if (warp == 6) {
+        // ---------------- scheduler (leader CTA): claim items in schedule order, one ahead of the TMA warp
+        if (lane == 0 && rank == 0) {
+            const uint32_t peer_ring = map_to_cta(ring, 1), peer_bar = map_to_cta(bar_ring, 1);
+            for (int n = 0;; ++n) {
+                // claim n is taken when the TMA thread starts item n-1: exactly one item ahead, so the claim's
+                // latency is hidden and no role can fall a whole ring behind
+                if (n >= 1 && !mbar_wait(bar_go, (uint32_t)(n - 1) & 1u, p, SITE_SCHED_GO, n)) break;
+                const int it = atomicAdd(p.next_item, 1);
+                const int slot = n % PROD_RING;
+                ring_gen[slot] = it;
+                asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_ring + 4 * slot), "r"(it) : "memory");
+                mbar_arrive(bar_ring + 8 * slot);
+                mbar_arrive_cluster(peer_bar + 8 * slot);        // release at cluster scope: orders the store above
+                if (it >= n_items) break;
+            }
+        }
     } else {
         // ---------------- epilogue: warps 2..5 own tensor-memory lanes 32*(warp % 4) .. +31
         const int q = warp & 3;
@@ -367,7 +422,10 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int it = first; it < n_items && ok; it += stride) {
+        for (int n = 0; ok; ++n) {
+            const int it = claimed(n);
+            if (!epilogue_all(it >= 0)) break;            // leave together if any thread gave up
+            if (it >= n_items) break;
             const int4 item = p.items[it];
             const int kind = item.x & 0xff, tile = item.w;
             const bool present = (rank == 0) || item.z >= 0;        // the pair's second band may be absent
