@@ -65,8 +65,9 @@ struct Params {
     int4 *items;          // [max_items] {kind | expert << 8, band 0, band 1 or -1, tile}
     int4 *segs;           // [max_bands] {first band, bands, dest, rows}
     int *seg_slot0;       // [max_bands]
-    int *tok_slot;        // [R*T*kmax]
+    int *tok_slot;        // [R*T*kmax] slot + 1 of each of the token's rows, ascending expert; 0 = none
     float *tok_gate;      // [R*T*kmax]
+    int *plan_ticket;     // blocks of the plan kernel that have finished marking
     int *next_item;       // schedule items claimed so far (GEMM CTA pairs take them in order)
     unsigned *hcount;     // [max_bands] first-GEMM tiles finished per band
     unsigned *flags;      // [max_bands*n2] epoch of the call that finished the tile

@@ -29,8 +29,7 @@ inline size_t align_up(size_t v, size_t a = ALIGN) { return (v + a - 1) / a * a;
 struct Layout {
     // offsets into the workspace, in bytes
     size_t Xa, H, Y;
-    size_t zero_begin, bitmap, hcount, status, next_item, zero_end;   // cleared to 0 at the start of every call
-    size_t tok_slot, tok_slot_bytes;                       // filled with -1 at the start of every call
+    size_t zero_begin, bitmap, hcount, status, next_item, tok_slot, zero_end;   // cleared at the start of every call
     size_t wordpfx, group_rows, group_start, group_slot, pos, slot;
     size_t band_expert, band_dest, band_valid, band_slot0, sched_band, items, segs, seg_slot0;
     size_t tok_gate, flags, meta;
@@ -51,6 +50,7 @@ int check_config(const moe_ovl_config *c)
         c->producer_sm_limit < 0 || c->d_model < 1 || c->d_ffn < 1)
         return MOE_OVL_ERR_INVALID_ARG;
     if (c->d_model % TB_N != 0 || c->d_ffn % H_TILE != 0) return MOE_OVL_ERR_UNSUPPORTED;
+    if ((long long)c->num_src_ranks * c->tokens_per_rank * (c->d_model / 8) >= (1ll << 31)) return MOE_OVL_ERR_UNSUPPORTED;
     if (c->num_local_experts > PLAN_MAX_EXPERTS ||
         (long long)c->num_local_experts * c->num_src_ranks > PLAN_MAX_GROUPS)
         return MOE_OVL_ERR_UNSUPPORTED;
@@ -82,10 +82,9 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->bitmap = take((size_t)G * L->words * 4);
     L->hcount = take((size_t)L->max_bands * 4);
     L->status = take(ST_COUNT * 4);
-    L->next_item = take(4);
+    L->next_item = take(8);
+    L->tok_slot = take(ntok * L->kmax * 4);
     L->zero_end = off;
-    L->tok_slot_bytes = ntok * L->kmax * 4;
-    L->tok_slot = take(L->tok_slot_bytes);
     L->tok_gate = take(ntok * L->kmax * 4);
     L->wordpfx = take((size_t)G * L->words * 4);
     L->group_rows = take((size_t)G * 4);
@@ -125,6 +124,7 @@ struct moe_ovl_ctx {
     Layout L;
     uint8_t *ws;
     int num_sms;
+    int combine_blocks_per_sm, scatter_blocks_per_sm;
     unsigned epoch;
     cudaStream_t s_prod, s_cons;
     cudaEvent_t ev_fork, ev_prod_done, ev_cons_done;
@@ -191,6 +191,7 @@ Params make_params(moe_ovl_ctx *ctx)
     p.seg_slot0 = at<int>(ctx, L.seg_slot0); p.tok_slot = at<int>(ctx, L.tok_slot);
     p.tok_gate = at<float>(ctx, L.tok_gate); p.hcount = at<unsigned>(ctx, L.hcount);
     p.next_item = at<int>(ctx, L.next_item);
+    p.plan_ticket = at<int>(ctx, L.next_item) + 1;
     p.flags = at<unsigned>(ctx, L.flags); p.meta = at<int>(ctx, L.meta); p.status = at<int>(ctx, L.status);
     return p;
 }
@@ -277,6 +278,12 @@ int moe_ovl_create(moe_ovl_ctx **out, const moe_ovl_config *cfg, void *workspace
     CREATE_CHECK(cudaFuncSetAttribute(producer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PROD_SMEM_BYTES));
     CREATE_CHECK(cudaFuncSetAttribute(consumer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       CONSUMER_SMEM_BYTES));
+    // grid-stride kernels get exactly one resident wave: a partial second wave would run at a fraction of the
+    // occupancy and stretch the kernel
+    CREATE_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctx->combine_blocks_per_sm, combine_kernel, 256, 0));
+    CREATE_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctx->scatter_blocks_per_sm, scatter_kernel, 256, 0));
+    ctx->combine_blocks_per_sm = std::max(1, ctx->combine_blocks_per_sm);
+    ctx->scatter_blocks_per_sm = std::max(1, ctx->scatter_blocks_per_sm);
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     CREATE_CHECK(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
@@ -361,17 +368,14 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     CU_CHECK(ctx, cudaEventRecord(ctx->t_begin, st));
     // ---- plan + gather (8a-1 .. 8a-3): integer kernels on the caller's stream
     CU_CHECK(ctx, cudaMemsetAsync(ctx->ws + L.zero_begin, 0, L.zero_end - L.zero_begin, st));
-    CU_CHECK(ctx, cudaMemsetAsync(ctx->ws + L.tok_slot, 0xff, L.tok_slot_bytes, st));
-    if (p.M > 0) {
-        plan_mark_kernel<<<(p.M + 255) / 256, 256, 0, st>>>(p);
-        ++launches;
-    }
-    plan_build_kernel<<<1, PLAN_THREADS, 0, st>>>(p, sc);
+    plan_mark_build_kernel<<<std::max(1, (p.M + PLAN_THREADS - 1) / PLAN_THREADS), PLAN_THREADS, 0, st>>>(p, sc);
     ++launches;
     if (p.M > 0) {
-        plan_rows_kernel<<<(p.M + 7) / 8, 256, 0, st>>>(p);
-        plan_zero_pad_kernel<<<std::min(L.max_bands, 4 * ctx->num_sms), 256, 0, st>>>(p);
-        launches += 2;
+        // one resident wave of row blocks (3 per SM) minus the blocks that zero the padding rows
+        const int pad_blocks = std::min(L.max_bands, ctx->num_sms / 2);
+        const int row_blocks = std::max(1, std::min((p.M + 7) / 8, 3 * ctx->num_sms - pad_blocks));
+        plan_rows_kernel<<<row_blocks + pad_blocks, 256, 0, st>>>(p, row_blocks);
+        ++launches;
     }
     CU_CHECK(ctx, cudaGetLastError());
     CU_CHECK(ctx, cudaEventRecord(ctx->t_prep, st));
@@ -397,11 +401,11 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
         producer_kernel<<<prod_ctas, PROD_THREADS, PROD_SMEM_BYTES, st>>>(maps, p, 0);
         CU_CHECK(ctx, cudaEventRecord(ctx->t_p1, st));
         CU_CHECK(ctx, cudaEventRecord(ctx->t_m0, st));
-        scatter_kernel<<<8 * ctx->num_sms, 256, 0, st>>>(p);
+        scatter_kernel<<<ctx->scatter_blocks_per_sm * ctx->num_sms, 256, 0, st>>>(p);
         CU_CHECK(ctx, cudaEventRecord(ctx->t_m1, st));
     }
-    launches += 2;
-    combine_kernel<<<8 * ctx->num_sms, 256, 0, st>>>(p);
+    launches += 2;                               // GEMM + consumer or scatter
+    combine_kernel<<<ctx->combine_blocks_per_sm * ctx->num_sms, 256, 0, st>>>(p);
     ++launches;
     CU_CHECK(ctx, cudaGetLastError());
     CU_CHECK(ctx, cudaEventRecord(ctx->t_end, st));
@@ -525,6 +529,8 @@ int moe_ovl_get_plan(moe_ovl_ctx *ctx, const moe_ovl_plan_view *v)
     };
     for (auto &e : cp)
         if (e.dst && e.bytes) CU_CHECK(ctx, cudaMemcpy(e.dst, ctx->ws + e.off, e.bytes, cudaMemcpyDeviceToHost));
+    if (v->tok_slot)                           // stored as slot + 1 with 0 = none; reported as slot with -1 = none
+        for (size_t i = 0; i < ntokk; ++i) v->tok_slot[i] -= 1;
     return MOE_OVL_OK;
 }
 

@@ -80,38 +80,66 @@ __global__ void __launch_bounds__(256) scatter_kernel(const Params p)
     }
 }
 
-// One CTA per token at a time; thread v handles 8 consecutive features.
+// One CTA works on one token at a time (grid-stride over tokens); thread v handles 8 consecutive features.
+// The next token's list is fetched while the current token's rows are in flight.
 __global__ void __launch_bounds__(256) combine_kernel(const Params p)
 {
     const int ntok = p.R * p.T;
     const int nv = p.d / 8;
+    constexpr int KFAST = 2;                      // list entries kept in registers
+    int slot[KFAST];
+    float gate[KFAST];
+    auto fetch = [&](int tok) {
+#pragma unroll
+        for (int j = 0; j < KFAST; ++j) {
+            const bool use = tok < ntok && j < p.kmax;
+            slot[j] = use ? __ldg(p.tok_slot + (size_t)tok * p.kmax + j) : 0;
+            gate[j] = use ? __ldg(p.tok_gate + (size_t)tok * p.kmax + j) : 0.f;
+        }
+    };
+    fetch(blockIdx.x);
     for (int tok = blockIdx.x; tok < ntok; tok += gridDim.x) {
-        const int r = tok / p.T;
-        const int *ts = p.tok_slot + (size_t)tok * p.kmax;
-        const float *tg = p.tok_gate + (size_t)tok * p.kmax;
-        const uint16_t *base = p.ret + (size_t)r * p.ret_rows_per_rank * p.d;
+        const uint16_t *region = p.ret + (size_t)(tok / p.T) * p.ret_rows_per_rank * p.d;
         uint4 *o = reinterpret_cast<uint4 *>(p.out + (size_t)tok * p.d);
+        int cs[KFAST];
+        float cg[KFAST];
+#pragma unroll
+        for (int j = 0; j < KFAST; ++j) { cs[j] = slot[j]; cg[j] = gate[j]; }
+        fetch(tok + gridDim.x);
         for (int v = threadIdx.x; v < nv; v += blockDim.x) {
+            uint4 row[KFAST];
+#pragma unroll
+            for (int j = 0; j < KFAST; ++j)
+                row[j] = cs[j] > 0 ? __ldcs(reinterpret_cast<const uint4 *>(region + (size_t)(cs[j] - 1) * p.d) + v)
+                                   : make_uint4(0, 0, 0, 0);
             float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            for (int j = 0; j < p.kmax; ++j) {           // ascending local expert
-                const int slot = ts[j];
-                if (slot < 0) break;
-                const float g = tg[j];
-                const uint4 q = __ldcs(reinterpret_cast<const uint4 *>(base + (size_t)slot * p.d) + v);
+            auto add = [&](const uint4 &q, float g) {
                 const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     acc[2 * i] += g * __uint_as_float(w[i] << 16);
                     acc[2 * i + 1] += g * __uint_as_float(w[i] & 0xffff0000u);
                 }
+            };
+            // ascending local expert; the list is dense, so the first empty entry (0) ends it
+            bool open = true;
+#pragma unroll
+            for (int j = 0; j < KFAST; ++j) {
+                open = open && cs[j] > 0;
+                if (open) add(row[j], cg[j]);
+            }
+            if (open) {
+                for (int j = KFAST; j < p.kmax; ++j) {        // tokens with more than two local rows
+                    const int s = p.tok_slot[(size_t)tok * p.kmax + j];
+                    if (s <= 0) break;
+                    add(__ldcs(reinterpret_cast<const uint4 *>(region + (size_t)(s - 1) * p.d) + v),
+                        p.tok_gate[(size_t)tok * p.kmax + j]);
+                }
             }
             uint32_t w[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint32_t r2;
-                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r2) : "f"(acc[2 * i + 1]), "f"(acc[2 * i]));
-                w[i] = r2;
-            }
+            for (int i = 0; i < 4; ++i)
+                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(acc[2 * i + 1]), "f"(acc[2 * i]));
             o[v] = make_uint4(w[0], w[1], w[2], w[3]);
         }
     }

@@ -15,6 +15,7 @@ namespace moe_ovl {
 constexpr int PLAN_MAX_GROUPS = 1024;   // El * R
 constexpr int PLAN_MAX_EXPERTS = 256;   // El
 constexpr int PLAN_THREADS = 1024;
+constexpr int PLAN_SB_STAGE = 512;      // super-bands whose sizes are staged in shared memory for the serial pass
 
 // Scratch arrays of the plan kernel, one entry per super-band.
 struct PlanScratch {
@@ -51,10 +52,8 @@ __device__ __forceinline__ void load_expert_prefix(const Params &p, int *pre)
 }
 
 // ---- step 1: mark (expert, rank, token) of every row ---------------------------------------
-__global__ void __launch_bounds__(256) plan_mark_kernel(Params p)
+__device__ __forceinline__ void plan_mark(const Params &p, const int *pre)
 {
-    __shared__ int pre[PLAN_MAX_EXPERTS + 1];
-    load_expert_prefix(p, pre);
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= p.M) return;
     if (i >= pre[p.El]) {
@@ -78,8 +77,21 @@ __device__ __forceinline__ int num_segments(int nb, int mgb)
 }
 
 // ---- step 2: everything that is per group / band / segment / schedule item -------------------
-__global__ void __launch_bounds__(PLAN_THREADS, 1) plan_build_kernel(Params p, PlanScratch sc)
+// One launch does both steps: every block marks its rows, and the block that finishes last (ticket counter)
+// builds the plan, which needs all marks.
+__global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params p, PlanScratch sc)
 {
+    __shared__ int pre[PLAN_MAX_EXPERTS + 1];
+    __shared__ int s_last;
+    load_expert_prefix(p, pre);
+    plan_mark(p, pre);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(p.plan_ticket, 1) == (int)gridDim.x - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+
     __shared__ int n[PLAN_MAX_GROUPS], nb[PLAN_MAX_GROUPS], gstart[PLAN_MAX_GROUPS], gslot[PLAN_MAX_GROUPS];
     __shared__ int gsched[PLAN_MAX_GROUPS], gsegoff[PLAN_MAX_GROUPS];
     __shared__ int key[PLAN_MAX_EXPERTS], eorder[PLAN_MAX_EXPERTS];
@@ -87,6 +99,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_build_kernel(Params p, P
     __shared__ int run_exp[2 * PLAN_MAX_EXPERTS];
     __shared__ int segs_per_rank[PLAN_MAX_GROUPS];
     __shared__ int s_nsb;
+    __shared__ int s_sb_nb[PLAN_SB_STAGE], s_sb_end[PLAN_SB_STAGE];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
     const int G = p.El * p.R;
@@ -99,7 +112,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_build_kernel(Params p, P
         int run = 0;
         for (int w0 = 0; w0 < p.words; w0 += 32) {
             const int w = w0 + lane;
-            const int c = w < p.words ? __popc(bm[w]) : 0;
+            const int c = w < p.words ? __popc(__ldcg(bm + w)) : 0;    // written by other blocks' atomics
             int inc = c;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -232,29 +245,39 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_build_kernel(Params p, P
     //    index is the outer loop and the band pair the inner one, so that the CTA pairs working side by side
     //    share a weight tile.  The second-GEMM block of a super-band is issued lag_items items after its
     //    first-GEMM block, so that its input is normally complete when a CTA pair reaches it.
-    if (tid == 0) {
+    //    (The loop is serial; band counts and block ends are staged in shared memory when they fit, so that
+    //    each step costs shared-memory latency, not a round trip to L2.)
+    {
         const int nsb = s_nsb;
-        int ng1 = 0, off = 0;
-        for (int ng2 = 0; ng2 < nsb; ++ng2) {
-            while (ng1 < nsb && (ng1 <= ng2 || off - sc.sb_g1end[ng2] < p.lag_items)) {
-                sc.sb_g1off[ng1] = off;
-                off += ((sc.sb_nb[ng1] + 1) / 2) * p.n1;
-                sc.sb_g1end[ng1] = off;
-                ++ng1;
+        const bool staged = nsb <= PLAN_SB_STAGE;
+        if (staged)
+            for (int i = tid; i < nsb; i += blockDim.x) s_sb_nb[i] = sc.sb_nb[i];
+        __syncthreads();
+        if (tid == 0) {
+            int *nbv = staged ? s_sb_nb : sc.sb_nb;
+            int *endv = staged ? s_sb_end : sc.sb_g1end;
+            int ng1 = 0, off = 0;
+            for (int ng2 = 0; ng2 < nsb; ++ng2) {
+                while (ng1 < nsb && (ng1 <= ng2 || off - endv[ng2] < p.lag_items)) {
+                    sc.sb_g1off[ng1] = off;
+                    off += ((nbv[ng1] + 1) / 2) * p.n1;
+                    endv[ng1] = off;
+                    ++ng1;
+                }
+                sc.sb_g2off[ng2] = off;
+                off += ((nbv[ng2] + 1) / 2) * p.n2;
             }
-            sc.sb_g2off[ng2] = off;
-            off += ((sc.sb_nb[ng2] + 1) / 2) * p.n2;
+            p.meta[META_ITEMS] = off;
         }
-        p.meta[META_ITEMS] = off;
     }
     __syncthreads();
 
-    // G: the item list
-    for (int sb = 0; sb < s_nsb; ++sb) {
+    // G: the item list, one warp per super-band
+    for (int sb = warp; sb < s_nsb; sb += nwarps) {
         const int start = sc.sb_start[sb], cnt = sc.sb_nb[sb], e = sc.sb_expert[sb];
         const int np = (cnt + 1) / 2;
         const int o1 = sc.sb_g1off[sb], o2 = sc.sb_g2off[sb];
-        for (int idx = tid; idx < np * (p.n1 + p.n2); idx += blockDim.x) {
+        for (int idx = lane; idx < np * (p.n1 + p.n2); idx += 32) {
             const bool g1 = idx < np * p.n1;
             const int k = g1 ? idx : idx - np * p.n1;
             const int pair = k % np, tile = k / np;
@@ -265,54 +288,89 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_build_kernel(Params p, P
     }
 }
 
-// ---- step 3: per row: aligned position, return slot, per-token list entry, copy into the layout ---
-__global__ void __launch_bounds__(256) plan_rows_kernel(Params p)
+// ---- step 3: per row: aligned position, return slot, per-token list entry, copy into the layout;
+//      the blocks after the row blocks zero the padding rows of every band (Section 3.2.1: zero-filled rows)
+struct RowMeta {
+    int pos, slot, j, tok;    // pos < 0: row skipped (bad metadata)
+};
+
+__device__ __forceinline__ RowMeta resolve_row(const Params &p, const int *pre, int i, int lane)
 {
-    __shared__ int pre[PLAN_MAX_EXPERTS + 1];
-    load_expert_prefix(p, pre);
-    const int lane = threadIdx.x & 31;
-    const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (i >= p.M || i >= pre[p.El]) return;
+    RowMeta m{-1, -1, 0, 0};
+    if (i >= p.M || i >= pre[p.El]) return m;
     const int e = expert_of_row(pre, p.El, i);
     const int r = p.src_rank[i], t = p.src_token[i];
-    if (r < 0 || r >= p.R || t < 0 || t >= p.T) return;
+    if (r < 0 || r >= p.R || t < 0 || t >= p.T) return m;
     const int g = e * p.R + r;
     const size_t w = (size_t)g * p.words + (t >> 5);
     const int q = p.wordpfx[w] + __popc(p.bitmap[w] & ((1u << (t & 31)) - 1u));
-    const int pos = p.group_start[g] + q;
-    const int slot = p.group_slot[g] + q;
+    m.pos = p.group_start[g] + q;
+    m.slot = p.group_slot[g] + q;
+    m.tok = r * p.T + t;
     // entry of this row in its token's list: number of lower-indexed local experts the token also selected
     int j = 0;
     for (int o = lane; o < e; o += 32)
         j += (p.bitmap[(size_t)(o * p.R + r) * p.words + (t >> 5)] >> (t & 31)) & 1u;
-    j = __reduce_add_sync(0xffffffffu, j);
-    if (lane == 0) {
-        p.pos[i] = pos;
-        p.slot[i] = slot;
-        if (p.slot_out) p.slot_out[i] = slot;
-        if (j < p.kmax) {
-            const size_t at = ((size_t)r * p.T + t) * p.kmax + j;
-            p.tok_slot[at] = slot;
-            p.tok_gate[at] = p.gate[i];
-        } else {
-            report_error(p.status, ERR_BAD_ROUTING, SITE_TOK_OVERFLOW, i);
-        }
-    }
-    const uint4 *src = reinterpret_cast<const uint4 *>(p.x + (size_t)i * p.d);
-    uint4 *dst = reinterpret_cast<uint4 *>(p.Xa + (size_t)pos * p.d);
-    const int nv = p.d / 8;
-    for (int v = lane; v < nv; v += 32) dst[v] = __ldg(src + v);
+    m.j = __reduce_add_sync(0xffffffffu, j);
+    return m;
 }
 
-// ---- step 4: zero the padding rows of every band (Section 3.2.1: zero-filled rows) -----------
-__global__ void __launch_bounds__(256) plan_zero_pad_kernel(Params p)
+constexpr int ROWS_CHUNK = 8;       // 16-byte vectors per lane in flight before the row's position is needed
+__global__ void __launch_bounds__(256, 3) plan_rows_kernel(Params p, int row_blocks)
 {
-    const int nbands = p.meta[META_BANDS];
-    for (int band = blockIdx.x; band < nbands; band += gridDim.x) {
-        const int valid = p.band_valid[band];
-        uint4 *dst = reinterpret_cast<uint4 *>(p.Xa + ((size_t)band * TB_M + valid) * p.d);
-        const size_t nv = (size_t)(TB_M - valid) * p.d / 8;
-        for (size_t v = threadIdx.x; v < nv; v += blockDim.x) dst[v] = make_uint4(0, 0, 0, 0);
+    __shared__ int pre[PLAN_MAX_EXPERTS + 1];
+    const int lane = threadIdx.x & 31;
+    const int nv = p.d / 8;
+    if ((int)blockIdx.x >= row_blocks) {
+        const int nbands = p.meta[META_BANDS];
+        for (int band = blockIdx.x - row_blocks; band < nbands; band += gridDim.x - row_blocks) {
+            const int valid = p.band_valid[band];
+            uint4 *dst = reinterpret_cast<uint4 *>(p.Xa + ((size_t)band * TB_M + valid) * p.d);
+            const size_t n = (size_t)(TB_M - valid) * nv;
+            for (size_t v = threadIdx.x; v < n; v += blockDim.x) dst[v] = make_uint4(0, 0, 0, 0);
+        }
+        return;
+    }
+    load_expert_prefix(p, pre);
+    // warps walk the rows with a grid stride; the position of the NEXT row is resolved while the loads of the
+    // current row are in flight, so the chain of dependent metadata loads is off the critical path
+    const int nwarps = row_blocks * (blockDim.x >> 5);
+    int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    RowMeta cur = resolve_row(p, pre, i, lane);
+    for (; i < p.M; i += nwarps) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(p.x + (size_t)i * p.d);
+        uint4 buf[ROWS_CHUNK];
+#pragma unroll
+        for (int k = 0; k < ROWS_CHUNK; ++k)
+            if (lane + 32 * k < nv) buf[k] = __ldcs(src + lane + 32 * k);
+        const RowMeta nxt = resolve_row(p, pre, i + nwarps, lane);
+        if (cur.pos >= 0) {
+            uint4 *dst = reinterpret_cast<uint4 *>(p.Xa + (size_t)cur.pos * p.d);
+#pragma unroll
+            for (int k = 0; k < ROWS_CHUNK; ++k)
+                if (lane + 32 * k < nv) dst[lane + 32 * k] = buf[k];
+            for (int v0 = 32 * ROWS_CHUNK; v0 < nv; v0 += 32 * ROWS_CHUNK) {
+#pragma unroll
+                for (int k = 0; k < ROWS_CHUNK; ++k)
+                    if (v0 + lane + 32 * k < nv) buf[k] = __ldcs(src + v0 + lane + 32 * k);
+#pragma unroll
+                for (int k = 0; k < ROWS_CHUNK; ++k)
+                    if (v0 + lane + 32 * k < nv) dst[v0 + lane + 32 * k] = buf[k];
+            }
+            if (lane == 0) {
+                p.pos[i] = cur.pos;
+                p.slot[i] = cur.slot;
+                if (p.slot_out) p.slot_out[i] = cur.slot;
+                if (cur.j < p.kmax) {
+                    const size_t at = (size_t)cur.tok * p.kmax + cur.j;
+                    p.tok_slot[at] = cur.slot + 1;            // 0 (the cleared state) means "no row"
+                    p.tok_gate[at] = p.gate[i];
+                } else {
+                    report_error(p.status, ERR_BAD_ROUTING, SITE_TOK_OVERFLOW, i);
+                }
+            }
+        }
+        cur = nxt;
     }
 }
 
