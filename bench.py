@@ -28,9 +28,9 @@ import numpy as np  # noqa: E402
 METRIC = "moe_expert_return_tflops"
 UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of one producer launch, from the ncu capture summarised in
-# profiles/ (captured on a smaller case and scaled by the number of tiles); None until captured.
-NCU_PRODUCER_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum of one producer launch, from the one-pass ncu launch lists of the
+# full-size workloads summarised in profiles/.
+NCU_PRODUCER_TRAFFIC_BYTES = {"mixtral": 3953099008 + 309059200, "fine": 497301248 + 342024576}
 
 
 def load_peaks():
@@ -49,59 +49,66 @@ def flops_of(shape, rows: int) -> float:
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """Samples SM clock, power and throttle reasons (read-only NVML queries) every few milliseconds while the
+    timed region runs; falls back to nothing if NVML is not importable."""
 
     def __init__(self, index: int):
         self.index = index
-        self.lines = []
-        self.proc = None
+        self.samples = []
+        self.stop_flag = False
         self.thread = None
+        self.nv = None
+        self.handle = None
+        self.max_mhz = None
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE,
-                                         stderr=subprocess.DEVNULL, text=True)
+            import pynvml as nv
+            nv.nvmlInit()
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = self.index
+            if vis:
+                ids = [v.strip() for v in vis.split(",") if v.strip()]
+                if self.index < len(ids) and ids[self.index].isdigit():
+                    phys = int(ids[self.index])
+            self.handle = nv.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = float(nv.nvmlDeviceGetMaxClockInfo(self.handle, nv.NVML_CLOCK_SM))
+            self.nv = nv
         except Exception:
-            self.proc = None
+            self.nv = None
             return
         self.thread = threading.Thread(target=self._pump, daemon=True)
         self.thread.start()
 
     def _pump(self):
-        for line in self.proc.stdout:
-            self.lines.append((time.time(), line.strip()))
+        nv = self.nv
+        while not self.stop_flag:
+            try:
+                mhz = float(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
+                mw = float(nv.nvmlDeviceGetPowerUsage(self.handle))
+                get = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                    nv.nvmlDeviceGetCurrentClocksThrottleReasons
+                reasons = int(get(self.handle))
+            except Exception:
+                break
+            self.samples.append((time.time(), mhz, mw / 1e3, reasons))
+            time.sleep(0.004)
 
     def stop(self, t0: float, t1: float):
-        if self.proc is None:
+        self.stop_flag = True
+        if self.nv is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, mx, pw, reasons = [], [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ts, line in self.lines:
-            if ts < t0 or ts > t1 + 0.2:
-                continue
-            f = [x.strip() for x in line.split(",")]
-            if len(f) < 7:
-                continue
-            try:
-                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
-            except ValueError:
-                continue
-            for n, v in zip(names, f[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w": statistics.median(pw) if pw else None, "reasons": sorted(reasons), "samples": len(sm)}
+        self.thread.join(timeout=2)
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        reasons = sorted(n for n, bit in names.items() if any(s[3] & bit for s in inside))
+        return {"sm_mhz": statistics.median(s[1] for s in inside) if inside else None, "sm_max_mhz": self.max_mhz,
+                "power_w": statistics.median(s[2] for s in inside) if inside else None, "reasons": reasons,
+                "samples": len(inside), "window": "timed region of the headline steps"}
 
 
 def sample_for_cpu(shape, dsp, n_tokens: int, seed: int = 0):
@@ -246,9 +253,9 @@ def main():
 
     # ---- headline: K steps in the chosen mode (overlap unless asked otherwise)
     head_mode = B.MODE_OVERLAP if args.mode == "overlap" else B.MODE_NON_OVERLAP
-    sampler = ClockSampler(local_rank if os.environ.get("CUDA_VISIBLE_DEVICES") is None else 0)
+    sampler = ClockSampler(local_rank)
     sampler.start()
-    time.sleep(0.3)
+    time.sleep(0.05)
     total_ms, per, rep, (t0, t1) = timed(head_mode, args.consumer_sms, args.steps, args.warmup)
     clocks = sampler.stop(t0, t1)
     secs = D.max_over_ranks(total_ms / 1e3, dev)
@@ -271,31 +278,39 @@ def main():
                 "launch_ms": prod, "flops_per_launch": step_flops,
                 "traffic": NCU_PRODUCER_TRAFFIC_BYTES.get(shape.name)}
 
-    # ---- comparison: the in-build non-overlap baseline, same steps
-    non_overlap = None
+    # ---- comparison against the in-build non-overlap baseline.  The GPU is power-limited under this load, so a
+    #      block of steps measured later runs slower than one measured earlier: the variants are therefore
+    #      interleaved call by call (order reversed every round) and compared by their medians.
+    non_overlap, sweep = None, []
     if args.mode == "overlap":
-        nov_ms, nov_per, nov_rep, _ = timed(B.MODE_NON_OVERLAP, 0, args.steps, 3)
-        nov_secs = D.max_over_ranks(nov_ms / 1e3, dev)
-        nov_er = []
-        for _ in range(min(args.steps, 10)):
-            Hn.run(ctx, prob, mode=B.MODE_NON_OVERLAP)
-            nov_er.append(ctx.moe_ovl_get_report())
-        non_overlap = {"ms_per_step": nov_secs / args.steps * 1e3,
-                       "tflops": step_flops * args.steps * world / nov_secs / 1e12,
-                       "expert_return_us": statistics.mean(r.ms_expert_return for r in nov_er) * 1e3,
-                       "gemm_us": statistics.mean(r.ms_producer for r in nov_er) * 1e3,
-                       "scatter_us": statistics.mean(r.ms_mover for r in nov_er) * 1e3}
-
-    sweep = []
-    if not args.no_sweep and world == 1 and args.mode == "overlap":
-        for csm in (2, 4, 8, 16, 32):
-            ms, _, _, _ = timed(B.MODE_OVERLAP, csm, max(3, args.steps // 4), 2)
-            ers = []
-            for _ in range(3):
-                Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=csm)
-                ers.append(ctx.moe_ovl_get_report().ms_expert_return)
-            sweep.append({"consumer_sms": csm, "ms_per_step": ms / max(3, args.steps // 4),
-                          "expert_return_us": statistics.mean(ers) * 1e3})
+        csms = [args.consumer_sms] if (args.no_sweep or world > 1) else sorted({2, 4, 8, 16, 32, args.consumer_sms})
+        variants = [("non_overlap", B.MODE_NON_OVERLAP, 0)] + [(f"overlap{c}", B.MODE_OVERLAP, c) for c in csms]
+        rounds = max(6, args.steps)
+        evs = {n: [] for n, _, _ in variants}
+        for r in range(rounds + 2):
+            for name, mode, csm in (variants if r % 2 == 0 else variants[::-1]):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                Hn.run(ctx, prob, mode=mode, consumer_sm_count=max(csm, 2))
+                b.record()
+                if r >= 2:
+                    evs[name].append((a, b))
+        torch.cuda.synchronize()
+        med = {n: statistics.median(a.elapsed_time(b) for a, b in v) for n, v in evs.items()}
+        phases = {}
+        for name, mode, csm in variants[:1] + [v for v in variants if v[2] == args.consumer_sms]:
+            reps = []
+            for _ in range(5):
+                Hn.run(ctx, prob, mode=mode, consumer_sm_count=max(csm, 2))
+                reps.append(ctx.moe_ovl_get_report())
+            phases[name] = {k: statistics.median(getattr(r, "ms_" + k) for r in reps) * 1e3
+                            for k in ("prep", "expert_return", "producer", "mover", "combine")}
+        non_overlap = {"interleaved_rounds": rounds, "us_per_layer": med["non_overlap"] * 1e3,
+                       "tflops": step_flops / med["non_overlap"] / 1e9,
+                       "overlap_us_per_layer_same_rounds": med[f"overlap{args.consumer_sms}"] * 1e3,
+                       "phases_us": phases}
+        sweep = [{"consumer_sms": c, "us_per_layer": med[f"overlap{c}"] * 1e3,
+                  "vs_non_overlap": med[f"overlap{c}"] / med["non_overlap"]} for c in csms]
 
     # ---- end to end through the host-buffer entry point: H2D of the step's inputs and D2H of out inside the timing
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()

@@ -68,6 +68,7 @@ struct Params {
     int *tok_slot;        // [R*T*kmax] slot + 1 of each of the token's rows, ascending expert; 0 = none
     float *tok_gate;      // [R*T*kmax]
     int *plan_ticket;     // blocks of the plan kernel that have finished marking
+    int *next_seg;        // segments claimed so far (consumer CTAs, and GEMM CTAs once they are out of tiles)
     int *next_item;       // schedule items claimed so far (GEMM CTA pairs take them in order)
     unsigned *hcount;     // [max_bands] first-GEMM tiles finished per band
     unsigned *flags;      // [max_bands*n2] epoch of the call that finished the tile

@@ -82,7 +82,7 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->bitmap = take((size_t)G * L->words * 4);
     L->hcount = take((size_t)L->max_bands * 4);
     L->status = take(ST_COUNT * 4);
-    L->next_item = take(8);
+    L->next_item = take(12);
     L->tok_slot = take(ntok * L->kmax * 4);
     L->zero_end = off;
     L->tok_gate = take(ntok * L->kmax * 4);
@@ -192,6 +192,7 @@ Params make_params(moe_ovl_ctx *ctx)
     p.tok_gate = at<float>(ctx, L.tok_gate); p.hcount = at<unsigned>(ctx, L.hcount);
     p.next_item = at<int>(ctx, L.next_item);
     p.plan_ticket = at<int>(ctx, L.next_item) + 1;
+    p.next_seg = at<int>(ctx, L.next_item) + 2;
     p.flags = at<unsigned>(ctx, L.flags); p.meta = at<int>(ctx, L.meta); p.status = at<int>(ctx, L.status);
     return p;
 }

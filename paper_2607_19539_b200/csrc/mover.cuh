@@ -1,7 +1,8 @@
 // Return path and weighted reduction.
-//   consumer_kernel  persistent, one CTA per dedicated SM: polls the ready flags of its
-//                    next segment and moves the segment's valid rows into the owner
-//                    rank's receive buffer with one contiguous copy (Section 3.3.2-3.3.3)
+//   consumer_kernel  persistent, one CTA per dedicated SM: claims the next segment in schedule
+//                    order, polls its ready flags and moves its valid rows into the owner
+//                    rank's receive buffer with one contiguous copy (Section 3.3.2-3.3.3);
+//                    GEMM CTAs that run out of tiles join in, which removes the tail
 //   scatter_kernel   the non-overlap comparison: all bands, whole GPU, after the GEMM
 //   combine_kernel   out[r,t] = sum_j gate_j * ret[r][slot_j]  (Section 2.1 step 5)
 // All three are HBM/L2-bandwidth work: 16-byte coalesced loads and stores.
@@ -20,16 +21,51 @@ __device__ __forceinline__ void copy_rows_16B(const uint16_t *src, uint16_t *dst
 {
     const uint4 *s = reinterpret_cast<const uint4 *>(src);
     uint4 *d = reinterpret_cast<uint4 *>(dst);
+    constexpr int U = 8;                           // 16-byte loads in flight per thread
     size_t v = tid;
-    for (; v + 3 * (size_t)nthr < nvec; v += 4 * (size_t)nthr) {
-        const uint4 a = __ldcg(s + v), b = __ldcg(s + v + nthr), c = __ldcg(s + v + 2 * (size_t)nthr),
-                    e = __ldcg(s + v + 3 * (size_t)nthr);
-        __stcs(d + v, a);
-        __stcs(d + v + nthr, b);
-        __stcs(d + v + 2 * (size_t)nthr, c);
-        __stcs(d + v + 3 * (size_t)nthr, e);
+    for (; v + (U - 1) * (size_t)nthr < nvec; v += U * (size_t)nthr) {
+        uint4 r[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k) r[k] = __ldcg(s + v + k * (size_t)nthr);
+#pragma unroll
+        for (int k = 0; k < U; ++k) __stcs(d + v + k * (size_t)nthr, r[k]);
     }
     for (; v < nvec; v += nthr) __stcs(d + v, __ldcg(s + v));
+}
+
+// Segment mover shared by the consumer CTAs and by GEMM CTAs that have run out of tiles: claim the next
+// segment in schedule order, wait (bounded, acquire) until every tile of every one of its bands is flagged,
+// then move its valid rows into the owner rank's receive buffer with one contiguous copy.
+// s_seg: two ints of shared memory.  All threads of the CTA must call this together.
+__device__ __forceinline__ void move_segments(const Params &p, volatile int *s_seg)
+{
+    const int nseg = p.meta[META_SEGS];
+    const int lane = threadIdx.x & 31;
+    for (;;) {
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            int s = 0;
+            if (lane == 0) s = atomicAdd(p.next_seg, 1);
+            s = __shfl_sync(0xffffffffu, s, 0);
+            bool ok = true;
+            if (s < nseg) {
+                const int4 seg = p.segs[s];          // {first band, bands, dest, rows}
+                const int nflags = seg.y * p.n2;
+                const unsigned *f = p.flags + (size_t)seg.x * p.n2;
+                for (int i = lane; i < nflags && ok; i += 32)
+                    ok = wait_global(f + i, p.epoch, false, p, SITE_CONS_FLAG, (long long)seg.x * p.n2 + i, 2048);
+                ok = __all_sync(0xffffffffu, ok);
+            }
+            if (lane == 0) { s_seg[0] = s; s_seg[1] = ok ? 1 : 0; }
+        }
+        __syncthreads();
+        const int s = s_seg[0];
+        if (s >= nseg || !s_seg[1]) return;
+        const int4 seg = p.segs[s];
+        const uint16_t *src = p.Y + (size_t)seg.x * TB_M * p.d;
+        uint16_t *dst = p.ret + ((size_t)seg.z * p.ret_rows_per_rank + p.seg_slot0[s]) * p.d;
+        copy_rows_16B(src, dst, (size_t)seg.w * p.d / 8, threadIdx.x, blockDim.x);
+    }
 }
 
 // Launched as clusters of two so that the consumer takes whole SM pairs and leaves whole pairs to the GEMM,
@@ -37,29 +73,8 @@ __device__ __forceinline__ void copy_rows_16B(const uint16_t *src, uint16_t *dst
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MOVER_THREADS, 1) consumer_kernel(const Params p)
 {
     extern __shared__ uint8_t unused_smem[];
-    __shared__ int s_ok;
-    const int nseg = p.meta[META_SEGS];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // segments are listed in schedule order; CTA c takes segments c, c + cSM, ...
-    for (int s = blockIdx.x; s < nseg; s += gridDim.x) {
-        const int4 seg = p.segs[s];                  // {first band, bands, dest, rows}
-        if (warp == 0) {
-            // a segment is ready when every tile of every one of its bands is flagged (acquire)
-            const int nflags = seg.y * p.n2;
-            const unsigned *f = p.flags + (size_t)seg.x * p.n2;
-            bool ok = true;
-            for (int i = lane; i < nflags && ok; i += 32)
-                ok = wait_global(f + i, p.epoch, false, p, SITE_CONS_FLAG, (long long)seg.x * p.n2 + i, 2048);
-            ok = __all_sync(0xffffffffu, ok);
-            if (lane == 0) s_ok = ok ? 1 : 0;
-        }
-        __syncthreads();
-        if (!s_ok) return;
-        const uint16_t *src = p.Y + (size_t)seg.x * TB_M * p.d;
-        uint16_t *dst = p.ret + ((size_t)seg.z * p.ret_rows_per_rank + p.seg_slot0[s]) * p.d;
-        copy_rows_16B(src, dst, (size_t)seg.w * p.d / 8, threadIdx.x, blockDim.x);
-        __syncthreads();
-    }
+    __shared__ int s_seg[2];
+    move_segments(p, s_seg);
 }
 
 // One CTA per (band, chunk of rows): grid-stride over bands x chunks.

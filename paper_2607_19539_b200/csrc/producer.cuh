@@ -30,6 +30,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "mover.cuh"
 
 namespace moe_ovl {
 
@@ -499,6 +500,9 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
         tc_fence_after();
         tmem_dealloc(tmem_base, PROD_TMEM_COLS);
     }
+    // Out of tiles: help the consumer drain what is left, so that the last segments do not wait for the few
+    // consumer SMs (the tail Section 3.3.3 warns about when the consumer budget is small).
+    if (raise_flags) move_segments(p, reinterpret_cast<volatile int *>(smem_gen));
 }
 
 }  // namespace moe_ovl
