@@ -78,6 +78,8 @@ typedef struct {
 } moe_ovl_config;
 
 #define MOE_OVL_FLAG_HOST_STAGING 1u /* reserve workspace for moe_ovl_expert_return_host */
+#define MOE_OVL_FLAG_TEST_NO_FLAGS 2u /* test hook: in OVERLAP mode the GEMM raises no ready flags, so the consumer's
+                                         bounded wait runs out and the call ends with MOE_OVL_ERR_TIMEOUT */
 
 typedef struct {
     uint32_t struct_size;
@@ -174,10 +176,19 @@ int moe_ovl_create(moe_ovl_ctx **ctx, const moe_ovl_config *cfg, void *workspace
  * here; device-side errors are reported by moe_ovl_query_status. */
 int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *args);
 
-/* Same pass with per-call tensors in HOST memory: copies inputs to staging buffers
- * in the workspace, runs the pass, copies `out` back.  Needs MOE_OVL_FLAG_HOST_STAGING.
- * Asynchronous with respect to the host if the buffers are pinned. */
+/* Same pass with per-call tensors in HOST memory (pinned, for asynchronous copies): copies
+ * the inputs to staging buffers in the workspace, runs the pass on args->stream, copies
+ * `out` back.  Needs MOE_OVL_FLAG_HOST_STAGING.  The copies run on two internal streams and
+ * two staging slots, so that consecutive calls pipeline: the inputs of call i+1 travel while
+ * call i computes, and the result of call i travels while call i+1 computes.  Consequences:
+ * the host input buffers are read from the moment of the call (not ordered after earlier work
+ * on args->stream) and must stay unchanged until the call's pass has started; `out` of a call
+ * is complete once moe_ovl_host_join has been enqueued and its stream synchronised (or after
+ * moe_ovl_query_status), NOT merely when args->stream has drained. */
 int moe_ovl_expert_return_host(moe_ovl_ctx *ctx, const moe_ovl_host_args *args);
+
+/* Makes `stream` (cudaStream_t) wait for the result copies of every host-buffer call issued so far. */
+int moe_ovl_host_join(moe_ovl_ctx *ctx, void *stream);
 
 /* Waits for the last call and returns its device status: *code is MOE_OVL_OK,
  * MOE_OVL_ERR_TIMEOUT or MOE_OVL_ERR_BAD_ROUTING; *detail identifies the wait or

@@ -19,12 +19,13 @@ OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_WORKSPACE, ERR_TIMEOUT, ERR_BAD_ROUTING = -1, -2, -3, -4, -5, -6
 MODE_OVERLAP, MODE_NON_OVERLAP = 0, 1
 FLAG_HOST_STAGING = 1
+FLAG_TEST_NO_FLAGS = 2
 BUF_XA, BUF_H, BUF_Y = 0, 1, 2
 TB_M, TB_N, H_TILE = 128, 256, 128
 
 EXPORTS = [
     "moe_ovl_workspace_bytes", "moe_ovl_limits", "moe_ovl_create", "moe_ovl_expert_return",
-    "moe_ovl_expert_return_host", "moe_ovl_query_status", "moe_ovl_get_report", "moe_ovl_get_plan",
+    "moe_ovl_expert_return_host", "moe_ovl_host_join", "moe_ovl_query_status", "moe_ovl_get_report", "moe_ovl_get_plan",
     "moe_ovl_read_buffer", "moe_ovl_destroy", "moe_ovl_strerror", "moe_ovl_last_cuda_error",
     "moe_ovl_return_slots_static",
 ]
@@ -101,6 +102,7 @@ def load(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moe_ovl_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(Config), C.c_void_p, C.c_size_t]
     lib.moe_ovl_expert_return.argtypes = [C.c_void_p, C.POINTER(Args)]
     lib.moe_ovl_expert_return_host.argtypes = [C.c_void_p, C.POINTER(HostArgs)]
+    lib.moe_ovl_host_join.argtypes = [C.c_void_p, C.c_void_p]
     lib.moe_ovl_query_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
     lib.moe_ovl_get_report.argtypes = [C.c_void_p, C.POINTER(Report)]
     lib.moe_ovl_get_plan.argtypes = [C.c_void_p, C.POINTER(PlanView)]
@@ -224,6 +226,10 @@ class MoeOvl:
                      _ptr(gate), _ptr(w1), _ptr(w2), int(consumer_sm_count), int(mode), _ptr(out), st.cuda_stream)
         self.last_rows = M
         self._check(self.lib.moe_ovl_expert_return_host(self.ctx, C.byref(h)), "moe_ovl_expert_return_host")
+
+    def moe_ovl_host_join(self, stream=None) -> None:
+        st = self._torch.cuda.current_stream(self.cfg.device) if stream is None else stream
+        self._check(self.lib.moe_ovl_host_join(self.ctx, st.cuda_stream), "moe_ovl_host_join")
 
     def moe_ovl_query_status(self):
         code, detail = C.c_int32(0), C.c_int64(0)

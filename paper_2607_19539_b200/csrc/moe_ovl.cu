@@ -35,7 +35,7 @@ struct Layout {
     size_t tok_gate, flags, meta;
     size_t sb[6];
     // host staging (MOE_OVL_FLAG_HOST_STAGING)
-    size_t st_x, st_counts, st_rank, st_token, st_gate, st_ret, st_out;
+    size_t st_x[2], st_counts[2], st_rank[2], st_token[2], st_gate[2], st_out[2], st_ret;   // two staging slots
     size_t total;
     int max_bands, max_items, words, kmax, n1, n2;
     long long st_ret_rows;
@@ -105,13 +105,15 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     for (int i = 0; i < 6; ++i) L->sb[i] = take((size_t)L->max_bands * 4);
     L->st_ret_rows = (long long)c->tokens_per_rank * L->kmax;
     if (c->flags & MOE_OVL_FLAG_HOST_STAGING) {
-        L->st_x = take((size_t)std::max(c->max_rows, 1) * d * 2);
-        L->st_counts = take((size_t)c->num_local_experts * 4);
-        L->st_rank = take((size_t)std::max(c->max_rows, 1) * 4);
-        L->st_token = take((size_t)std::max(c->max_rows, 1) * 4);
-        L->st_gate = take((size_t)std::max(c->max_rows, 1) * 4);
+        for (int s = 0; s < 2; ++s) {
+            L->st_x[s] = take((size_t)std::max(c->max_rows, 1) * d * 2);
+            L->st_counts[s] = take((size_t)c->num_local_experts * 4);
+            L->st_rank[s] = take((size_t)std::max(c->max_rows, 1) * 4);
+            L->st_token[s] = take((size_t)std::max(c->max_rows, 1) * 4);
+            L->st_gate[s] = take((size_t)std::max(c->max_rows, 1) * 4);
+            L->st_out[s] = take(ntok * d * 2);
+        }
         L->st_ret = take((size_t)c->num_src_ranks * L->st_ret_rows * d * 2);
-        L->st_out = take(ntok * d * 2);
     }
     L->total = off;
     return MOE_OVL_OK;
@@ -127,6 +129,9 @@ struct moe_ovl_ctx {
     int combine_blocks_per_sm, scatter_blocks_per_sm;
     unsigned epoch;
     cudaStream_t s_prod, s_cons;
+    cudaStream_t s_h2d, s_d2h;                        // host-buffer entry point: copies overlap the previous/next pass
+    cudaEvent_t ev_h2d[2], ev_comp[2], ev_d2h[2];
+    unsigned long long host_calls;
     cudaEvent_t ev_fork, ev_prod_done, ev_cons_done;
     // timing: call start, after prep, GEMM start/end, mover start/end, call end
     cudaEvent_t t_begin, t_prep, t_p0, t_p1, t_m0, t_m1, t_end;
@@ -200,6 +205,7 @@ Params make_params(moe_ovl_ctx *ctx)
 int sync_last(moe_ovl_ctx *ctx)
 {
     if (ctx->ran) CU_CHECK(ctx, cudaStreamSynchronize(ctx->last_stream));
+    if (ctx->s_d2h) CU_CHECK(ctx, cudaStreamSynchronize(ctx->s_d2h));
     return MOE_OVL_OK;
 }
 
@@ -272,6 +278,15 @@ int moe_ovl_create(moe_ovl_ctx **out, const moe_ovl_config *cfg, void *workspace
     // the consumer stream gets the higher priority (Section 3.3.3)
     CREATE_CHECK(cudaStreamCreateWithPriority(&ctx->s_cons, cudaStreamNonBlocking, hi));
     CREATE_CHECK(cudaStreamCreateWithPriority(&ctx->s_prod, cudaStreamNonBlocking, lo));
+    if (cfg->flags & MOE_OVL_FLAG_HOST_STAGING) {
+        CREATE_CHECK(cudaStreamCreateWithFlags(&ctx->s_h2d, cudaStreamNonBlocking));
+        CREATE_CHECK(cudaStreamCreateWithFlags(&ctx->s_d2h, cudaStreamNonBlocking));
+        for (int s = 0; s < 2; ++s) {
+            CREATE_CHECK(cudaEventCreateWithFlags(&ctx->ev_h2d[s], cudaEventDisableTiming));
+            CREATE_CHECK(cudaEventCreateWithFlags(&ctx->ev_comp[s], cudaEventDisableTiming));
+            CREATE_CHECK(cudaEventCreateWithFlags(&ctx->ev_d2h[s], cudaEventDisableTiming));
+        }
+    }
     cudaEvent_t *plain[] = {&ctx->ev_fork, &ctx->ev_prod_done, &ctx->ev_cons_done};
     for (auto e : plain) CREATE_CHECK(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
     cudaEvent_t *timed[] = {&ctx->t_begin, &ctx->t_prep, &ctx->t_p0, &ctx->t_p1, &ctx->t_m0, &ctx->t_m1, &ctx->t_end};
@@ -309,6 +324,11 @@ int moe_ovl_destroy(moe_ovl_ctx *ctx)
     if (ctx->ran) cudaStreamSynchronize(ctx->last_stream);
     if (ctx->s_prod) { cudaStreamSynchronize(ctx->s_prod); cudaStreamDestroy(ctx->s_prod); }
     if (ctx->s_cons) { cudaStreamSynchronize(ctx->s_cons); cudaStreamDestroy(ctx->s_cons); }
+    if (ctx->s_h2d) { cudaStreamSynchronize(ctx->s_h2d); cudaStreamDestroy(ctx->s_h2d); }
+    if (ctx->s_d2h) { cudaStreamSynchronize(ctx->s_d2h); cudaStreamDestroy(ctx->s_d2h); }
+    for (int s = 0; s < 2; ++s)
+        for (cudaEvent_t e : {ctx->ev_h2d[s], ctx->ev_comp[s], ctx->ev_d2h[s]})
+            if (e) cudaEventDestroy(e);
     cudaEvent_t evs[] = {ctx->ev_fork, ctx->ev_prod_done, ctx->ev_cons_done, ctx->t_begin, ctx->t_prep, ctx->t_p0,
                          ctx->t_p1, ctx->t_m0, ctx->t_m1, ctx->t_end};
     for (auto e : evs)
@@ -391,7 +411,8 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
         CU_CHECK(ctx, cudaEventRecord(ctx->t_m1, ctx->s_cons));
         CU_CHECK(ctx, cudaEventRecord(ctx->ev_cons_done, ctx->s_cons));
         CU_CHECK(ctx, cudaEventRecord(ctx->t_p0, ctx->s_prod));
-        producer_kernel<<<prod_ctas, PROD_THREADS, PROD_SMEM_BYTES, ctx->s_prod>>>(maps, p, 1);
+        producer_kernel<<<prod_ctas, PROD_THREADS, PROD_SMEM_BYTES, ctx->s_prod>>>(
+            maps, p, (c.flags & MOE_OVL_FLAG_TEST_NO_FLAGS) ? 0 : 1);
         CU_CHECK(ctx, cudaEventRecord(ctx->t_p1, ctx->s_prod));
         CU_CHECK(ctx, cudaEventRecord(ctx->ev_prod_done, ctx->s_prod));
         CU_CHECK(ctx, cudaStreamWaitEvent(st, ctx->ev_cons_done, 0));
@@ -431,35 +452,58 @@ int moe_ovl_expert_return_host(moe_ovl_ctx *ctx, const moe_ovl_host_args *h)
     if (h->num_rows > 0 && (!h->x || !h->src_rank || !h->src_token || !h->gate)) return MOE_OVL_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(h->stream);
     const size_t M = (size_t)h->num_rows, d = c.d_model;
+    const int slot = (int)(ctx->host_calls & 1);
+    const bool reused = ctx->host_calls >= 2;          // this slot has been through a full pass before
     CU_CHECK(ctx, cudaSetDevice(c.device));
-    CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_counts, h->expert_counts, (size_t)c.num_local_experts * 4,
-                                  cudaMemcpyHostToDevice, st));
+    // inputs: on the copy-in stream, once the pass that last read this slot's staging buffers is done
+    if (reused) CU_CHECK(ctx, cudaStreamWaitEvent(ctx->s_h2d, ctx->ev_comp[slot], 0));
+    CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_counts[slot], h->expert_counts, (size_t)c.num_local_experts * 4,
+                                  cudaMemcpyHostToDevice, ctx->s_h2d));
     if (M > 0) {
-        CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_x, h->x, M * d * 2, cudaMemcpyHostToDevice, st));
-        CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_rank, h->src_rank, M * 4, cudaMemcpyHostToDevice, st));
-        CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_token, h->src_token, M * 4, cudaMemcpyHostToDevice, st));
-        CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_gate, h->gate, M * 4, cudaMemcpyHostToDevice, st));
+        CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_x[slot], h->x, M * d * 2, cudaMemcpyHostToDevice, ctx->s_h2d));
+        CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_rank[slot], h->src_rank, M * 4, cudaMemcpyHostToDevice, ctx->s_h2d));
+        CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_token[slot], h->src_token, M * 4, cudaMemcpyHostToDevice, ctx->s_h2d));
+        CU_CHECK(ctx, cudaMemcpyAsync(ctx->ws + L.st_gate[slot], h->gate, M * 4, cudaMemcpyHostToDevice, ctx->s_h2d));
     }
+    CU_CHECK(ctx, cudaEventRecord(ctx->ev_h2d[slot], ctx->s_h2d));
+    // the pass itself, on the caller's stream: needs this slot's inputs, and its staged output buffer free again
+    CU_CHECK(ctx, cudaStreamWaitEvent(st, ctx->ev_h2d[slot], 0));
+    if (reused) CU_CHECK(ctx, cudaStreamWaitEvent(st, ctx->ev_d2h[slot], 0));
     moe_ovl_args a;
     std::memset(&a, 0, sizeof(a));
     a.struct_size = sizeof(a);
     a.num_rows = h->num_rows;
-    a.x = ctx->ws + L.st_x;
-    a.expert_counts = at<int32_t>(ctx, L.st_counts);
-    a.src_rank = at<int32_t>(ctx, L.st_rank);
-    a.src_token = at<int32_t>(ctx, L.st_token);
-    a.gate = at<float>(ctx, L.st_gate);
+    a.x = ctx->ws + L.st_x[slot];
+    a.expert_counts = at<int32_t>(ctx, L.st_counts[slot]);
+    a.src_rank = at<int32_t>(ctx, L.st_rank[slot]);
+    a.src_token = at<int32_t>(ctx, L.st_token[slot]);
+    a.gate = at<float>(ctx, L.st_gate[slot]);
     a.w1 = h->w1; a.w2 = h->w2;
     a.consumer_sm_count = h->consumer_sm_count;
     a.mode = h->mode;
     a.ret = ctx->ws + L.st_ret;
     a.ret_rows_per_rank = L.st_ret_rows;
-    a.out = ctx->ws + L.st_out;
+    a.out = ctx->ws + L.st_out[slot];
     a.stream = h->stream;
     const int rc = moe_ovl_expert_return(ctx, &a);
     if (rc != MOE_OVL_OK) return rc;
-    CU_CHECK(ctx, cudaMemcpyAsync(h->out, ctx->ws + L.st_out, (size_t)c.num_src_ranks * c.tokens_per_rank * d * 2,
-                                  cudaMemcpyDeviceToHost, st));
+    CU_CHECK(ctx, cudaEventRecord(ctx->ev_comp[slot], st));
+    // result: on the copy-out stream, so that it overlaps the next call's pass
+    CU_CHECK(ctx, cudaStreamWaitEvent(ctx->s_d2h, ctx->ev_comp[slot], 0));
+    CU_CHECK(ctx, cudaMemcpyAsync(h->out, ctx->ws + L.st_out[slot], (size_t)c.num_src_ranks * c.tokens_per_rank * d * 2,
+                                  cudaMemcpyDeviceToHost, ctx->s_d2h));
+    CU_CHECK(ctx, cudaEventRecord(ctx->ev_d2h[slot], ctx->s_d2h));
+    ++ctx->host_calls;
+    return MOE_OVL_OK;
+}
+
+int moe_ovl_host_join(moe_ovl_ctx *ctx, void *stream)
+{
+    if (!ctx) return MOE_OVL_ERR_INVALID_ARG;
+    if (!(ctx->cfg.flags & MOE_OVL_FLAG_HOST_STAGING)) return MOE_OVL_ERR_WORKSPACE;
+    const unsigned long long n = ctx->host_calls < 2 ? ctx->host_calls : 2;
+    for (unsigned long long k = 0; k < n; ++k)
+        CU_CHECK(ctx, cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), ctx->ev_d2h[(ctx->host_calls - 1 - k) & 1], 0));
     return MOE_OVL_OK;
 }
 

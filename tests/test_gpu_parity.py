@@ -70,24 +70,61 @@ def test_segment_and_group_knobs(name, mgb, gb):
 
 @pytest.mark.parametrize("name", ["tiny", "small_zipf_rot"])
 def test_overlap_equals_non_overlap_bitwise(name):
-    """Both modes run the same GEMM code on the same tiles: any difference is a protocol bug, not rounding."""
+    """Both modes run the same GEMM code on the same tiles: any difference is a protocol bug, not rounding.
+    Two different problems alternate on one context, so that before every overlapped run the internal buffers
+    hold the OTHER problem's rows: a segment moved before its tiles were flagged would carry foreign values."""
     torch, B, Hn = _gpu()
     shape = I.SHAPES[name]
-    inp = I.make_inputs(shape)
-    dsp = I.dispatch(inp)
-    ctx = Hn.make_context(shape, max_rows=dsp.M)
-    base = Hn.upload(inp, dsp)
-    Hn.run(ctx, base, mode=B.MODE_NON_OVERLAP)
-    torch.cuda.synchronize()
-    ref_out, ref_ret = base.out.clone(), base.ret.clone()
-    for it in range(20):
+    probs = []
+    ctx = None
+    for seed in (shape.seed, shape.seed + 101):
+        inp = I.make_inputs(I.with_seed(shape, seed))
+        dsp = I.dispatch(inp)
+        probs.append((inp, dsp))
+    ctx = Hn.make_context(shape, max_rows=max(d.M for _, d in probs))
+    refs = []
+    for inp, dsp in probs:
+        base = Hn.upload(inp, dsp)
+        Hn.run(ctx, base, mode=B.MODE_NON_OVERLAP)
+        torch.cuda.synchronize()
+        refs.append((base, base.out.clone(), base.ret.clone()))
+    assert not torch.equal(refs[0][1].view(torch.int16), refs[1][1].view(torch.int16))
+    for it in range(24):
         csm = (2, 4, 8, 16, 32)[it % 5]
+        inp, dsp = probs[it % 2]
+        base, ref_out, ref_ret = refs[it % 2]
         prob = Hn.upload(inp, dsp, w1=base.w1, w2=base.w2)
         Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=csm)
         torch.cuda.synchronize()
         assert ctx.moe_ovl_query_status()[0] == 0
         assert torch.equal(prob.out.view(torch.int16), ref_out.view(torch.int16))
         assert torch.equal(prob.ret.view(torch.int16), ref_ret.view(torch.int16))
+
+
+def test_bounded_wait_gives_up_cleanly():
+    """A flag that nothing sets: the consumer's wait runs out after the configured bound, the call ends with a
+    timeout status (no hang, no fault), and the device stays usable."""
+    torch, B, Hn = _gpu()
+    shape = I.SHAPES["tiny"]
+    inp = I.make_inputs(shape)
+    dsp = I.dispatch(inp)
+    ctx = Hn.make_context(shape, max_rows=dsp.M, wait_timeout_us=20_000, flags=B.FLAG_TEST_NO_FLAGS)
+    prob = Hn.upload(inp, dsp)
+    Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=4)
+    torch.cuda.synchronize()
+    code, detail = ctx.moe_ovl_query_status()
+    assert code == B.ERR_TIMEOUT
+    assert detail >> 48 == 6                      # the wait that gave up: a consumer polling a tile flag
+    # the same context in non-overlap mode (no flags involved), and a fresh context, still work
+    Hn.run(ctx, prob, mode=B.MODE_NON_OVERLAP)
+    torch.cuda.synchronize()
+    assert ctx.moe_ovl_query_status()[0] == 0
+    ok = Hn.make_context(shape, max_rows=dsp.M)
+    prob2 = Hn.upload(inp, dsp, w1=prob.w1, w2=prob.w2)
+    Hn.run(ok, prob2, mode=B.MODE_OVERLAP, consumer_sm_count=4)
+    torch.cuda.synchronize()
+    assert ok.moe_ovl_query_status()[0] == 0
+    assert torch.equal(prob2.out.view(torch.int16), prob.out.view(torch.int16))
 
 
 def test_identity_experts_reproduce_x_bit_exactly():
@@ -206,8 +243,23 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     hx = pin(dsp.x_rows.view(np.int16))
     hc, hr, ht, hg = pin(dsp.expert_counts), pin(dsp.src_rank), pin(dsp.src_token), pin(dsp.gate)
     hout = torch.zeros((shape.R * shape.T, shape.d), dtype=torch.int16).pin_memory()
-    ctx.moe_ovl_expert_return_host(x=hx, expert_counts=hc, src_rank=hr, src_token=ht, gate=hg, w1=prob.w1,
-                                   w2=prob.w2, out=hout, consumer_sm_count=8, mode=B.MODE_OVERLAP)
+    # several calls in a row exercise both staging slots and the copy pipeline; a second problem in between
+    # makes a result that came from the wrong slot visible
+    inp2 = I.make_inputs(I.with_seed(shape, 5))
+    dsp2 = I.dispatch(inp2)
+    ctx2 = Hn.make_context(shape, max_rows=dsp2.M)
+    prob_b = Hn.upload(inp2, dsp2, w1=prob.w1, w2=prob.w2)
+    Hn.run(ctx2, prob_b, mode=B.MODE_OVERLAP, consumer_sm_count=8)
+    hx2 = pin(dsp2.x_rows.view(np.int16))
+    hc2, hr2, ht2, hg2 = pin(dsp2.expert_counts), pin(dsp2.src_rank), pin(dsp2.src_token), pin(dsp2.gate)
+    houts = [torch.zeros_like(hout).pin_memory() for _ in range(5)]
+    for i, ho in enumerate(houts):
+        a = (hx, hc, hr, ht, hg) if i % 2 == 0 else (hx2, hc2, hr2, ht2, hg2)
+        ctx.moe_ovl_expert_return_host(x=a[0], expert_counts=a[1], src_rank=a[2], src_token=a[3], gate=a[4],
+                                       w1=prob.w1, w2=prob.w2, out=ho, consumer_sm_count=8, mode=B.MODE_OVERLAP)
+    ctx.moe_ovl_host_join()
     torch.cuda.synchronize()
     assert ctx.moe_ovl_query_status()[0] == 0
-    assert torch.equal(hout, prob.out.view(torch.int16).cpu())
+    want = [prob.out.view(torch.int16).cpu(), prob_b.out.view(torch.int16).cpu()]
+    for i, ho in enumerate(houts):
+        assert torch.equal(ho, want[i % 2]), i
