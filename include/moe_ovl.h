@@ -71,7 +71,7 @@ typedef struct {
     int32_t d_ffn;              /* F, multiple of 128 */
     int32_t max_rows;           /* capacity for M */
     int32_t mid_seg_bands;      /* bands per middle segment (x of Figure 3b), >= 1 */
-    int32_t group_bands;        /* bands whose tiles are interleaved so that they share weight tiles in L2; 0 = default */
+    int32_t group_bands;        /* bands whose tiles are interleaved so that they share weight tiles in L2; 0 = default (16) */
     int32_t wait_timeout_us;    /* bound on every device-side wait; 0 = default (2 s) */
     int32_t producer_sm_limit;  /* NON_OVERLAP only: cap on GEMM CTAs (diagnostic baseline); 0 = all SMs */
     uint32_t flags;             /* MOE_OVL_FLAG_* */
@@ -91,7 +91,8 @@ typedef struct {
     const float *gate;            /* DEVICE [M] fp32 gate weight of (token, expert) */
     const void *w1;               /* DEVICE [El, 2F, d] bf16: rows 0..F-1 gate projection, F..2F-1 up projection */
     const void *w2;               /* DEVICE [El, d, F] bf16 */
-    int32_t consumer_sm_count;    /* SMs dedicated to the consumer (OVERLAP); 1..SMs/2, rounded up to a whole SM pair */
+    int32_t consumer_sm_count;    /* SMs dedicated to the consumer (OVERLAP); 1..SMs/2, rounded up to a whole SM pair;
+                                     0 = chosen by the library from the shape (see moe_ovl_report.consumer_ctas) */
     int32_t mode;                 /* MOE_OVL_MODE_* */
     void *ret;                    /* DEVICE [R][ret_rows_per_rank, d] bf16: simulated peer receive buffers.
                                      Row s of region r is written iff s < rows_per_rank[r]; the rest is untouched. */

@@ -183,7 +183,7 @@ Params make_params(moe_ovl_ctx *ctx)
     p.R = c.num_src_ranks; p.r_self = c.self_rank; p.T = c.tokens_per_rank; p.El = c.num_local_experts;
     p.kmax = L.kmax; p.d = c.d_model; p.F = c.d_ffn;
     p.mgb = std::max(1, c.mid_seg_bands);
-    p.group_bands = c.group_bands > 0 ? c.group_bands : 8;
+    p.group_bands = c.group_bands > 0 ? c.group_bands : 16;
     p.words = L.words; p.n1 = L.n1; p.n2 = L.n2; p.max_bands = L.max_bands; p.max_items = L.max_items;
     p.timeout_ns = (unsigned long long)(c.wait_timeout_us > 0 ? c.wait_timeout_us : 2000000) * 1000ull;
     p.Xa = at<uint16_t>(ctx, L.Xa); p.H = at<uint16_t>(ctx, L.H); p.Y = at<uint16_t>(ctx, L.Y);
@@ -354,8 +354,18 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     const bool overlap = a->mode == MOE_OVL_MODE_OVERLAP;
     int prod_ctas, cons_ctas = 0;
     if (overlap) {
-        if (a->consumer_sm_count < 1 || a->consumer_sm_count > ctx->num_sms / 2) return MOE_OVL_ERR_INVALID_ARG;
-        cons_ctas = (a->consumer_sm_count + 1) & ~1;        // whole SM pairs: the GEMM's CTAs work in pairs
+        if (a->consumer_sm_count < 0 || a->consumer_sm_count > ctx->num_sms / 2) return MOE_OVL_ERR_INVALID_ARG;
+        int want = a->consumer_sm_count;
+        if (want == 0) {
+            // Automatic budget (Section 3.3.3: too few consumer SMs and the transfer falls behind, too many and
+            // the GEMM loses capacity).  Every SM given up costs 1/SMs of the GEMM time; the return it hides is
+            // worth t_return.  Take about half of the break-even count SMs * t_return / t_gemm, with
+            // t_return = 4*d bytes per row at ~5 TB/s and t_gemm = 6*d*F flop per row at ~1.2 PFLOP/s.
+            const double t_ret = 4.0 * c.d_model / 5.0e12, t_gemm = 6.0 * c.d_model * (double)c.d_ffn / 1.2e15;
+            const double breakeven = ctx->num_sms * t_ret / t_gemm;
+            want = std::min(16, std::max(2, 2 * (int)(breakeven / 4.0 + 0.5)));
+        }
+        cons_ctas = (want + 1) & ~1;                        // whole SM pairs: the GEMM's CTAs work in pairs
         prod_ctas = (ctx->num_sms - cons_ctas) & ~1;        // disjoint SM sets: grids sum to the SM count
     } else {
         prod_ctas = (c.producer_sm_limit > 0 ? std::min(c.producer_sm_limit, ctx->num_sms) : ctx->num_sms) & ~1;

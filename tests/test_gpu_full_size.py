@@ -27,11 +27,15 @@ def sample_tokens(shape, dsp, per_rank, seed=0):
     return np.unique(np.concatenate(picks)).astype(np.int32)
 
 
-@pytest.mark.parametrize("name,csm,per_rank", [("mixtral", 8, 16), ("fine", 8, 24), ("mixtral_zipf", 8, 8)])
+@pytest.mark.parametrize("name,csm,per_rank", [
+    ("mixtral", 8, 16), ("fine", 8, 24), ("mixtral_zipf", 8, 8),
+    # points of the sweep grid: 4 local experts of 16, d=4096; (tokens per local expert, ffn, router)
+    ((1024, 1024, "uniform"), 2, 16), ((128, 2816, "zipf"), 16, 8), ((4096, 1024, "zipf"), 32, 8),
+])
 def test_full_size_parity(name, csm, per_rank):
     import torch
     from paper_2607_19539_b200 import binding as B, harness as Hn
-    shape = I.SHAPES[name]
+    shape = I.SHAPES[name] if isinstance(name, str) else I.sweep_shape(*name)
     inp = I.make_inputs(shape)
     dsp = I.dispatch(inp)
     ctx = Hn.make_context(shape, max_rows=dsp.M)

@@ -101,6 +101,39 @@ def test_overlap_equals_non_overlap_bitwise(name):
         assert torch.equal(prob.ret.view(torch.int16), ref_ret.view(torch.int16))
 
 
+def test_automatic_consumer_budget():
+    """consumer_sm_count = 0 lets the library size the consumer partition from the shape: small for wide FFNs
+    (the return is cheap next to the GEMM), larger for narrow ones; results do not depend on it."""
+    torch, B, Hn = _gpu()
+    got = {}
+    for name in ("tiny", "small"):
+        shape = I.SHAPES[name]
+        inp = I.make_inputs(shape)
+        dsp = I.dispatch(inp)
+        ctx = Hn.make_context(shape, max_rows=dsp.M)
+        ref = Hn.upload(inp, dsp)
+        Hn.run(ctx, ref, mode=B.MODE_NON_OVERLAP)
+        prob = Hn.upload(inp, dsp, w1=ref.w1, w2=ref.w2)
+        Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=0)
+        torch.cuda.synchronize()
+        assert ctx.moe_ovl_query_status()[0] == 0
+        assert torch.equal(prob.out.view(torch.int16), ref.out.view(torch.int16))
+        got[name] = ctx.moe_ovl_get_report().consumer_ctas
+        assert got[name] % 2 == 0 and 2 <= got[name] <= 16
+    wide = Hn.make_context(I.SHAPES["mixtral"], max_rows=128)     # only the shape matters for the choice
+    narrow = Hn.make_context(I.SHAPES["fine"], max_rows=128)
+    for c, sh in ((wide, I.SHAPES["mixtral"]), (narrow, I.SHAPES["fine"])):
+        z = I.Dispatched(np.zeros((0, sh.d), np.uint16), np.zeros(sh.El, np.int32), np.zeros(0, np.int32),
+                         np.zeros(0, np.int32), np.zeros(0, np.float32), np.zeros(0, np.int32))
+        inp0 = I.MoEInputs(sh, np.zeros((sh.R, sh.T, sh.d), np.uint16), np.zeros((sh.El, 2 * sh.F, sh.d), np.uint16),
+                           np.zeros((sh.El, sh.d, sh.F), np.uint16), np.zeros((sh.R, sh.T, sh.k), np.int32),
+                           np.zeros((sh.R, sh.T, sh.k), np.float32))
+        p0 = Hn.upload(inp0, z)
+        Hn.run(c, p0, mode=B.MODE_OVERLAP, consumer_sm_count=0)
+        torch.cuda.synchronize()
+    assert wide.moe_ovl_get_report().consumer_ctas == 2 and narrow.moe_ovl_get_report().consumer_ctas == 8
+
+
 def test_bounded_wait_gives_up_cleanly():
     """A flag that nothing sets: the consumer's wait runs out after the configured bound, the call ends with a
     timeout status (no hang, no fault), and the device stays usable."""
@@ -224,7 +257,10 @@ def test_bad_routing_is_reported_not_fatal():
     assert ctx.moe_ovl_query_status()[0] == 0
     # synchronous argument errors
     with pytest.raises(B.MoeOvlError) as e:
-        Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=0)
+        Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=-1)
+    assert e.value.code == B.ERR_INVALID_ARG
+    with pytest.raises(B.MoeOvlError) as e:
+        Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=100)
     assert e.value.code == B.ERR_INVALID_ARG
     with pytest.raises(B.MoeOvlError):
         Hn.run(ctx, prob, mode=7)
