@@ -44,7 +44,10 @@ def load_peaks():
 
 
 def flops_of(shape, rows: int) -> float:
-    """6*d*F per valid row: gate, up and down projections at 2 flop per multiply-add."""
+    """6*d*F per valid row: gate, up and down projections at 2 flop per multiply-add
+    (2*d*N for shapes whose experts are one projection each)."""
+    if shape.N_out:
+        return 2.0 * shape.d * shape.N_out * rows
     return 6.0 * shape.d * shape.F * rows
 
 
@@ -118,6 +121,14 @@ def sample_for_cpu(shape, dsp, n_tokens: int, seed: int = 0):
     return np.sort(pick).astype(np.int32)
 
 
+def oracle_forward(inp, sel):
+    from oracle import value_oracle as VO
+    sh = inp.shape
+    if sh.N_out:
+        return VO.forward_tokens_single(inp.x, inp.expert, inp.gate, inp.w1, sh.El, sh.first_local, sel)
+    return VO.forward_tokens(inp.x, inp.expert, inp.gate, inp.w1, inp.w2, sh.El, sh.first_local, sel)
+
+
 def time_oracle(inp, dsp, target_s: float):
     """Times the CPU oracle, as it stands, on a bounded sample of tokens that own local rows.
     Returns (TFLOP/s, seconds, tokens, rows, threads)."""
@@ -130,7 +141,7 @@ def time_oracle(inp, dsp, target_s: float):
     def run(n):
         sel = sample_for_cpu(shape, dsp, n)
         t0 = time.perf_counter()
-        VO.forward_tokens(inp.x, inp.expert, inp.gate, inp.w1, inp.w2, shape.El, shape.first_local, sel)
+        oracle_forward(inp, sel)
         dt = time.perf_counter() - t0
         return dt, len(sel), int(rows_of[sel].sum())
 
@@ -156,9 +167,8 @@ def run_reference(args, shape):
     times = []
     for i in range(args.warmup + args.steps):
         sel = sample_for_cpu(shape, dsp, n, seed=i)
-        from oracle import value_oracle as VO
         t0 = time.perf_counter()
-        VO.forward_tokens(inp.x, inp.expert, inp.gate, inp.w1, inp.w2, shape.El, shape.first_local, sel)
+        oracle_forward(inp, sel)
         if i >= args.warmup:
             times.append(time.perf_counter() - t0)
     rows_of = np.zeros(shape.R * shape.T, np.int64)
@@ -179,8 +189,9 @@ def run_reference(args, shape):
 
 
 def workload_config(shape, args):
+    kind = f"one projection N={shape.N_out}" if shape.N_out else f"ffn={shape.F}"
     return {"workload": f"{shape.name}: {shape.R} simulated ranks x {shape.T} tokens, {shape.Eg} experts "
-                        f"top-{shape.k}, {shape.El} local, d={shape.d}, ffn={shape.F}, {shape.router} router",
+                        f"top-{shape.k}, {shape.El} local, d={shape.d}, {kind}, {shape.router} router",
             "consumer_sms": args.consumer_sms, "mode": getattr(args, "mode", "overlap"), "seed": shape.seed,
             "l2": "inputs larger than L2 (weights + activations >> 126 MB), no flush",
             "parallelism": f"replicas x{args.gpus}" if args.gpus > 1 else "single GPU"}

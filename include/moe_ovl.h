@@ -74,6 +74,10 @@ typedef struct {
     int32_t group_bands;        /* bands whose tiles are interleaved so that they share weight tiles in L2; 0 = default (16) */
     int32_t wait_timeout_us;    /* bound on every device-side wait; 0 = default (2 s) */
     int32_t producer_sm_limit;  /* NON_OVERLAP only: cap on GEMM CTAs (diagnostic baseline); 0 = all SMs */
+    int32_t single_gemm_out;    /* 0: SwiGLU FFN experts.  N > 0: the operator the paper evaluates (Table 2) -- each
+                                   expert is ONE projection y = x . W^T with W[N, d_model]; N multiple of 256,
+                                   d_model multiple of 64; w1 holds W as [El, N, d_model], w2 and d_ffn are
+                                   ignored, and ret / out rows are N wide */
     uint32_t flags;             /* MOE_OVL_FLAG_* */
 } moe_ovl_config;
 
@@ -89,15 +93,17 @@ typedef struct {
     const int32_t *src_rank;      /* DEVICE [M] in 0..R-1: owner rank of the row's token */
     const int32_t *src_token;     /* DEVICE [M] in 0..T-1: token index on the owner rank */
     const float *gate;            /* DEVICE [M] fp32 gate weight of (token, expert) */
-    const void *w1;               /* DEVICE [El, 2F, d] bf16: rows 0..F-1 gate projection, F..2F-1 up projection */
-    const void *w2;               /* DEVICE [El, d, F] bf16 */
+    const void *w1;               /* DEVICE [El, 2F, d] bf16: rows 0..F-1 gate projection, F..2F-1 up projection
+                                     (single-projection mode: [El, N, d]) */
+    const void *w2;               /* DEVICE [El, d, F] bf16 (single-projection mode: ignored, may be NULL) */
     int32_t consumer_sm_count;    /* SMs dedicated to the consumer (OVERLAP); 1..SMs/2, rounded up to a whole SM pair;
                                      0 = chosen by the library from the shape (see moe_ovl_report.consumer_ctas) */
     int32_t mode;                 /* MOE_OVL_MODE_* */
     void *ret;                    /* DEVICE [R][ret_rows_per_rank, d] bf16: simulated peer receive buffers.
                                      Row s of region r is written iff s < rows_per_rank[r]; the rest is untouched. */
     int64_t ret_rows_per_rank;    /* >= T * min(k, El) */
-    void *out;                    /* DEVICE [R*T, d] bf16, fully overwritten (tokens with no local row get +0) */
+    void *out;                    /* DEVICE [R*T, d] bf16, fully overwritten (tokens with no local row get +0);
+                                     ret and out rows are N wide in single-projection mode */
     int32_t *slot_out;            /* DEVICE [M] or NULL: receive-buffer slot of every input row */
     int32_t *rows_per_rank_out;   /* DEVICE [R] or NULL */
     int32_t *segs_per_rank_out;   /* DEVICE [R] or NULL: segments sent to each rank */

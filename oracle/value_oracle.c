@@ -22,6 +22,9 @@
  * returned row y, and the final output.  Gates are used as given; y is returned
  * unscaled because the scaling happens at the owner rank.
  *
+ * moe_oracle_tokens_single is the same for experts that are one projection each
+ * (the operator of the paper's Table 2).
+ *
  * Pins (tests/test_oracle_values.py): float64 NumPy evaluation of the
  * definition on tiny inputs, a one-expert case against library matmul/silu,
  * zero gate projection => exact zeros, identity experts with unit gates
@@ -140,6 +143,70 @@ int moe_oracle_tokens(int T, int k, int d, int F, int El, int first_local,
         }
         free(xf);
         free(hf);
+        free(acc);
+    }
+    return bad ? -1 : 0;
+}
+
+/* The operator the paper evaluates (Table 2: one M x K x N GEMM per expert, "the expert output projection"):
+ * each expert is a single projection, y_j = bf16( sum_c x[c] * W[e][j][c] ), j = 0..N-1, followed by the same
+ * gate-weighted sum at the owner.  Same arguments as moe_oracle_tokens with w [El, N, d]; out [n_sel, N],
+ * y [n_sel, kmax, N]. */
+int moe_oracle_tokens_single(int T, int k, int d, int N, int El, int first_local,
+                             const uint16_t *x, const int32_t *expert, const float *gate, const uint16_t *w,
+                             int n_sel, const int32_t *sel, int kmax,
+                             uint16_t *out, uint16_t *y, int32_t *y_exp, int nthreads)
+{
+    int bad = 0;
+    (void)T;
+#ifdef _OPENMP
+    if (nthreads > 0)
+        omp_set_num_threads(nthreads);
+#endif
+#pragma omp parallel
+    {
+        float *xf = (float *)malloc(sizeof(float) * (size_t)d);
+        float *acc = (float *)malloc(sizeof(float) * (size_t)N);
+#pragma omp for schedule(dynamic, 1)
+        for (int s = 0; s < n_sel; ++s) {
+            const int tok = sel[s];
+            for (int c = 0; c < d; ++c)
+                xf[c] = bf16_to_f32(x[(size_t)tok * d + c]);
+            for (int j = 0; j < N; ++j)
+                acc[j] = 0.0f;
+            int nloc = 0;
+            for (int j = 0; j < kmax; ++j) {
+                y_exp[(size_t)s * kmax + j] = -1;
+                memset(y + ((size_t)s * kmax + j) * N, 0, sizeof(uint16_t) * (size_t)N);
+            }
+            for (int e = 0; e < El; ++e) {
+                int hit = -1;
+                for (int q = 0; q < k; ++q)
+                    if (expert[(size_t)tok * k + q] == first_local + e)
+                        hit = q;
+                if (hit < 0)
+                    continue;
+                if (nloc >= kmax) {
+                    bad = 1;
+                    break;
+                }
+                uint16_t *yr = y + ((size_t)s * kmax + nloc) * N;
+                const float g = gate[(size_t)tok * k + hit];
+                for (int j = 0; j < N; ++j) {
+                    const uint16_t *wr = w + ((size_t)e * N + j) * d;
+                    float v = 0.0f;
+                    for (int c = 0; c < d; ++c)
+                        v += xf[c] * bf16_to_f32(wr[c]);
+                    yr[j] = f32_to_bf16(v);
+                    acc[j] += g * bf16_to_f32(yr[j]);
+                }
+                y_exp[(size_t)s * kmax + nloc] = e;
+                ++nloc;
+            }
+            for (int j = 0; j < N; ++j)
+                out[(size_t)s * N + j] = f32_to_bf16(acc[j]);
+        }
+        free(xf);
         free(acc);
     }
     return bad ? -1 : 0;

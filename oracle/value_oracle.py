@@ -29,6 +29,7 @@ def _load() -> ctypes.CDLL:
     if _lib is None:
         _lib = ctypes.CDLL(build())
         _lib.moe_oracle_tokens.restype = ctypes.c_int
+        _lib.moe_oracle_tokens_single.restype = ctypes.c_int
         _lib.moe_oracle_threads.restype = ctypes.c_int
     return _lib
 
@@ -65,6 +66,33 @@ def forward_tokens(x: np.ndarray, expert: np.ndarray, gate: np.ndarray, w1: np.n
     rc = _load().moe_oracle_tokens(
         ctypes.c_int(T), ctypes.c_int(k), ctypes.c_int(d), ctypes.c_int(F), ctypes.c_int(El),
         ctypes.c_int(first_local), _p(x), _p(expert), _p(gate), _p(w1), _p(w2),
+        ctypes.c_int(n), _p(sel), ctypes.c_int(kmax), _p(out), _p(y), _p(y_exp), ctypes.c_int(nthreads))
+    if rc != 0:
+        raise ValueError("a token selects more local experts than min(k, El)")
+    return out, y, y_exp
+
+
+def forward_tokens_single(x: np.ndarray, expert: np.ndarray, gate: np.ndarray, w: np.ndarray, El: int,
+                          first_local: int, sel: np.ndarray, nthreads: int = 0
+                          ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Single-projection experts: x [R,T,d]; w [El,N,d].  Returns (out [n,N], y [n,kmax,N], y_expert [n,kmax])."""
+    R, T, d = x.shape
+    k = expert.shape[-1]
+    N = w.shape[1]
+    assert w.shape == (El, N, d)
+    kmax = min(k, El)
+    x = np.ascontiguousarray(x, np.uint16)
+    expert = np.ascontiguousarray(expert, np.int32)
+    gate = np.ascontiguousarray(gate, np.float32)
+    w = np.ascontiguousarray(w, np.uint16)
+    sel = np.ascontiguousarray(sel, np.int32)
+    n = int(sel.shape[0])
+    out = np.zeros((n, N), np.uint16)
+    y = np.zeros((n, kmax, N), np.uint16)
+    y_exp = np.full((n, kmax), -1, np.int32)
+    rc = _load().moe_oracle_tokens_single(
+        ctypes.c_int(T), ctypes.c_int(k), ctypes.c_int(d), ctypes.c_int(N), ctypes.c_int(El),
+        ctypes.c_int(first_local), _p(x), _p(expert), _p(gate), _p(w),
         ctypes.c_int(n), _p(sel), ctypes.c_int(kmax), _p(out), _p(y), _p(y_exp), ctypes.c_int(nthreads))
     if rc != 0:
         raise ValueError("a token selects more local experts than min(k, El)")

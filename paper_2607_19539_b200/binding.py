@@ -36,7 +36,7 @@ class Config(C.Structure):
                 ("self_rank", C.c_int32), ("tokens_per_rank", C.c_int32), ("num_local_experts", C.c_int32),
                 ("top_k", C.c_int32), ("d_model", C.c_int32), ("d_ffn", C.c_int32), ("max_rows", C.c_int32),
                 ("mid_seg_bands", C.c_int32), ("group_bands", C.c_int32), ("wait_timeout_us", C.c_int32),
-                ("producer_sm_limit", C.c_int32), ("flags", C.c_uint32)]
+                ("producer_sm_limit", C.c_int32), ("single_gemm_out", C.c_int32), ("flags", C.c_uint32)]
 
 
 class Args(C.Structure):
@@ -120,9 +120,11 @@ def strerror(code: int) -> str:
 
 def make_config(*, device: int, num_src_ranks: int, self_rank: int, tokens_per_rank: int, num_local_experts: int,
                 top_k: int, d_model: int, d_ffn: int, max_rows: int, mid_seg_bands: int = 1, group_bands: int = 0,
-                wait_timeout_us: int = 0, producer_sm_limit: int = 0, flags: int = 0) -> Config:
+                wait_timeout_us: int = 0, producer_sm_limit: int = 0, single_gemm_out: int = 0,
+                flags: int = 0) -> Config:
     return Config(C.sizeof(Config), device, num_src_ranks, self_rank, tokens_per_rank, num_local_experts, top_k,
-                  d_model, d_ffn, max_rows, mid_seg_bands, group_bands, wait_timeout_us, producer_sm_limit, flags)
+                  d_model, d_ffn, max_rows, mid_seg_bands, group_bands, wait_timeout_us, producer_sm_limit,
+                  single_gemm_out, flags)
 
 
 def moe_ovl_workspace_bytes(cfg: Config) -> int:
@@ -264,7 +266,11 @@ class MoeOvl:
 
     def moe_ovl_read_buffer(self, which: int, row0: int, rows: int) -> np.ndarray:
         """Rows [row0, row0+rows) of the aligned input (BUF_XA), hidden (BUF_H) or output (BUF_Y) buffer, bf16 bits."""
-        cols = self.cfg.d_ffn if which == BUF_H else self.cfg.d_model
+        cols = self.cfg.d_model
+        if which == BUF_H:
+            cols = self.cfg.d_ffn
+        elif which == BUF_Y and self.cfg.single_gemm_out:
+            cols = self.cfg.single_gemm_out
         out = np.zeros((rows, cols), np.uint16)
         self._check(self.lib.moe_ovl_read_buffer(self.ctx, which, row0 * cols * 2, rows * cols * 2, out.ctypes.data),
                     "moe_ovl_read_buffer")

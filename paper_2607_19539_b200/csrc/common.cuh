@@ -34,12 +34,15 @@ enum : long long {
 struct Params {
     // problem
     int R, r_self, T, El, kmax, d, F;
+    int dout;           // width of Y / ret / out rows: d for FFN experts, N for single-projection experts
+    int k2;             // K extent of the GEMM that writes Y: F for FFN experts, d for single-projection experts
+    int single;         // single-projection experts: no first GEMM, the output GEMM reads Xa
     int M;
     int mgb;            // bands per middle segment
     int group_bands;    // bands interleaved in one super-band
     int lag_items;      // schedule items between a band's last first-GEMM tile and its first second-GEMM tile
     int words;          // 32-bit words of one (expert, rank) token bitmap = ceil(T / 32)
-    int n1, n2;         // tiles per band: F / 128 and d / 256
+    int n1, n2;         // tiles per band: F / 128 (0 for single-projection experts) and dout / 256
     int max_bands, max_items;
     unsigned epoch;
     unsigned long long timeout_ns;

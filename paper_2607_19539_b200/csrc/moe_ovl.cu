@@ -38,6 +38,7 @@ struct Layout {
     size_t st_x[2], st_counts[2], st_rank[2], st_token[2], st_gate[2], st_out[2], st_ret;   // two staging slots
     size_t total;
     int max_bands, max_items, words, kmax, n1, n2;
+    int dout, k2, f_eff, single;
     long long st_ret_rows;
 };
 
@@ -47,10 +48,16 @@ int check_config(const moe_ovl_config *c)
     if (c->num_src_ranks < 1 || c->self_rank < 0 || c->self_rank >= c->num_src_ranks) return MOE_OVL_ERR_INVALID_ARG;
     if (c->tokens_per_rank < 1 || c->num_local_experts < 1 || c->top_k < 1) return MOE_OVL_ERR_INVALID_ARG;
     if (c->max_rows < 0 || c->mid_seg_bands < 0 || c->group_bands < 0 || c->wait_timeout_us < 0 ||
-        c->producer_sm_limit < 0 || c->d_model < 1 || c->d_ffn < 1)
+        c->producer_sm_limit < 0 || c->d_model < 1 || c->single_gemm_out < 0 ||
+        (c->single_gemm_out == 0 && c->d_ffn < 1))
         return MOE_OVL_ERR_INVALID_ARG;
-    if (c->d_model % TB_N != 0 || c->d_ffn % H_TILE != 0) return MOE_OVL_ERR_UNSUPPORTED;
-    if ((long long)c->num_src_ranks * c->tokens_per_rank * (c->d_model / 8) >= (1ll << 31)) return MOE_OVL_ERR_UNSUPPORTED;
+    if (c->single_gemm_out > 0) {
+        if (c->d_model % TB_K != 0 || c->single_gemm_out % TB_N != 0) return MOE_OVL_ERR_UNSUPPORTED;
+    } else if (c->d_model % TB_N != 0 || c->d_ffn % H_TILE != 0) {
+        return MOE_OVL_ERR_UNSUPPORTED;
+    }
+    const int dout = c->single_gemm_out > 0 ? c->single_gemm_out : c->d_model;
+    if ((long long)c->num_src_ranks * c->tokens_per_rank * (dout / 8) >= (1ll << 31)) return MOE_OVL_ERR_UNSUPPORTED;
     if (c->num_local_experts > PLAN_MAX_EXPERTS ||
         (long long)c->num_local_experts * c->num_src_ranks > PLAN_MAX_GROUPS)
         return MOE_OVL_ERR_UNSUPPORTED;
@@ -63,21 +70,25 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     if (rc != MOE_OVL_OK) return rc;
     const long long G = (long long)c->num_local_experts * c->num_src_ranks;
     const long long max_bands_ll = ((long long)c->max_rows + TB_M - 1) / TB_M + G;
-    L->n1 = c->d_ffn / H_TILE;
-    L->n2 = c->d_model / TB_N;
+    L->single = c->single_gemm_out > 0;
+    L->dout = L->single ? c->single_gemm_out : c->d_model;
+    L->k2 = L->single ? c->d_model : c->d_ffn;
+    L->f_eff = L->single ? H_TILE : c->d_ffn;       // the hidden buffer is unused by single-projection experts
+    L->n1 = L->single ? 0 : c->d_ffn / H_TILE;
+    L->n2 = L->dout / TB_N;
     const long long max_items_ll = max_bands_ll * (L->n1 + L->n2);
     if (max_bands_ll > (1 << 24) || max_items_ll > (1ll << 30)) return MOE_OVL_ERR_UNSUPPORTED;
     L->max_bands = (int)max_bands_ll;
     L->max_items = (int)max_items_ll;
     L->words = (c->tokens_per_rank + 31) / 32;
     L->kmax = std::min(c->top_k, c->num_local_experts);
-    const size_t P = (size_t)L->max_bands * TB_M, d = c->d_model, F = c->d_ffn;
+    const size_t P = (size_t)L->max_bands * TB_M, d = c->d_model, F = L->f_eff, dout = L->dout;
     const size_t ntok = (size_t)c->num_src_ranks * c->tokens_per_rank;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
     L->Xa = take(P * d * 2);
     L->H = take(P * F * 2);
-    L->Y = take(P * d * 2);
+    L->Y = take(P * dout * 2);
     L->zero_begin = off;
     L->bitmap = take((size_t)G * L->words * 4);
     L->hcount = take((size_t)L->max_bands * 4);
@@ -111,9 +122,9 @@ int make_layout(const moe_ovl_config *c, Layout *L)
             L->st_rank[s] = take((size_t)std::max(c->max_rows, 1) * 4);
             L->st_token[s] = take((size_t)std::max(c->max_rows, 1) * 4);
             L->st_gate[s] = take((size_t)std::max(c->max_rows, 1) * 4);
-            L->st_out[s] = take(ntok * d * 2);
+            L->st_out[s] = take(ntok * dout * 2);
         }
-        L->st_ret = take((size_t)c->num_src_ranks * L->st_ret_rows * d * 2);
+        L->st_ret = take((size_t)c->num_src_ranks * L->st_ret_rows * dout * 2);
     }
     L->total = off;
     return MOE_OVL_OK;
@@ -181,7 +192,8 @@ Params make_params(moe_ovl_ctx *ctx)
     Params p;
     std::memset(&p, 0, sizeof(p));
     p.R = c.num_src_ranks; p.r_self = c.self_rank; p.T = c.tokens_per_rank; p.El = c.num_local_experts;
-    p.kmax = L.kmax; p.d = c.d_model; p.F = c.d_ffn;
+    p.kmax = L.kmax; p.d = c.d_model; p.F = L.f_eff;
+    p.dout = L.dout; p.k2 = L.k2; p.single = L.single;
     p.mgb = std::max(1, c.mid_seg_bands);
     p.group_bands = c.group_bands > 0 ? c.group_bands : 16;
     p.words = L.words; p.n1 = L.n1; p.n2 = L.n2; p.max_bands = L.max_bands; p.max_items = L.max_items;
@@ -307,7 +319,7 @@ int moe_ovl_create(moe_ovl_ctx **out, const moe_ovl_config *cfg, void *workspace
     ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
     const size_t P = (size_t)L.max_bands * TB_M;
     rc = encode_map(ctx, &ctx->map_xa, ctx->ws + L.Xa, P, cfg->d_model);
-    if (rc == MOE_OVL_OK) rc = encode_map(ctx, &ctx->map_h, ctx->ws + L.H, P, cfg->d_ffn);
+    if (rc == MOE_OVL_OK) rc = encode_map(ctx, &ctx->map_h, ctx->ws + L.H, P, L.f_eff);
     if (rc != MOE_OVL_OK) return fail(rc);
     // flags hold the epoch of the call that finished the tile: clear them once, never again
     CREATE_CHECK(cudaMemset(ctx->ws + L.flags, 0, (size_t)L.max_bands * L.n2 * 4));
@@ -343,7 +355,7 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     const moe_ovl_config &c = ctx->cfg;
     const Layout &L = ctx->L;
     if (a->num_rows < 0 || a->num_rows > c.max_rows) return MOE_OVL_ERR_INVALID_ARG;
-    if (!a->expert_counts || !a->w1 || !a->w2 || !a->ret || !a->out) return MOE_OVL_ERR_INVALID_ARG;
+    if (!a->expert_counts || !a->w1 || (!a->w2 && !L.single) || !a->ret || !a->out) return MOE_OVL_ERR_INVALID_ARG;
     if (a->num_rows > 0 && (!a->x || !a->src_rank || !a->src_token || !a->gate)) return MOE_OVL_ERR_INVALID_ARG;
     if (a->ret_rows_per_rank < (int64_t)c.tokens_per_rank * L.kmax) return MOE_OVL_ERR_INVALID_ARG;
     if (a->mode != MOE_OVL_MODE_OVERLAP && a->mode != MOE_OVL_MODE_NON_OVERLAP) return MOE_OVL_ERR_INVALID_ARG;
@@ -361,7 +373,8 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
             // the GEMM loses capacity).  Every SM given up costs 1/SMs of the GEMM time; the return it hides is
             // worth t_return.  Take about half of the break-even count SMs * t_return / t_gemm, with
             // t_return = 4*d bytes per row at ~5 TB/s and t_gemm = 6*d*F flop per row at ~1.2 PFLOP/s.
-            const double t_ret = 4.0 * c.d_model / 5.0e12, t_gemm = 6.0 * c.d_model * (double)c.d_ffn / 1.2e15;
+            const double t_ret = 4.0 * L.dout / 5.0e12;
+            const double t_gemm = (L.single ? 2.0 * c.d_model * (double)L.dout : 6.0 * c.d_model * (double)c.d_ffn) / 1.2e15;
             const double breakeven = ctx->num_sms * t_ret / t_gemm;
             want = std::min(16, std::max(2, 2 * (int)(breakeven / 4.0 + 0.5)));
         }
@@ -387,8 +400,15 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     ProducerMaps maps;
     maps.xa = ctx->map_xa;
     maps.h = ctx->map_h;
-    int rc = encode_map(ctx, &maps.w1, a->w1, (size_t)c.num_local_experts * 2 * c.d_ffn, c.d_model);
-    if (rc == MOE_OVL_OK) rc = encode_map(ctx, &maps.w2, a->w2, (size_t)c.num_local_experts * c.d_model, c.d_ffn);
+    int rc;
+    if (L.single) {
+        // one projection per expert: W[El, N, d] is the B operand of the GEMM that writes Y
+        rc = encode_map(ctx, &maps.w2, a->w1, (size_t)c.num_local_experts * L.dout, c.d_model);
+        maps.w1 = maps.w2;
+    } else {
+        rc = encode_map(ctx, &maps.w1, a->w1, (size_t)c.num_local_experts * 2 * c.d_ffn, c.d_model);
+        if (rc == MOE_OVL_OK) rc = encode_map(ctx, &maps.w2, a->w2, (size_t)c.num_local_experts * c.d_model, c.d_ffn);
+    }
     if (rc != MOE_OVL_OK) return rc;
 
     PlanScratch sc;
@@ -500,7 +520,7 @@ int moe_ovl_expert_return_host(moe_ovl_ctx *ctx, const moe_ovl_host_args *h)
     CU_CHECK(ctx, cudaEventRecord(ctx->ev_comp[slot], st));
     // result: on the copy-out stream, so that it overlaps the next call's pass
     CU_CHECK(ctx, cudaStreamWaitEvent(ctx->s_d2h, ctx->ev_comp[slot], 0));
-    CU_CHECK(ctx, cudaMemcpyAsync(h->out, ctx->ws + L.st_out[slot], (size_t)c.num_src_ranks * c.tokens_per_rank * d * 2,
+    CU_CHECK(ctx, cudaMemcpyAsync(h->out, ctx->ws + L.st_out[slot], (size_t)c.num_src_ranks * c.tokens_per_rank * L.dout * 2,
                                   cudaMemcpyDeviceToHost, ctx->s_d2h));
     CU_CHECK(ctx, cudaEventRecord(ctx->ev_d2h[slot], ctx->s_d2h));
     ++ctx->host_calls;
@@ -597,8 +617,8 @@ int moe_ovl_read_buffer(moe_ovl_ctx *ctx, int32_t which, size_t offset, size_t b
     size_t base, cap;
     switch (which) {
     case MOE_OVL_BUF_XA: base = L.Xa; cap = P * ctx->cfg.d_model * 2; break;
-    case MOE_OVL_BUF_H: base = L.H; cap = P * ctx->cfg.d_ffn * 2; break;
-    case MOE_OVL_BUF_Y: base = L.Y; cap = P * ctx->cfg.d_model * 2; break;
+    case MOE_OVL_BUF_H: base = L.H; cap = P * (size_t)L.f_eff * 2; break;
+    case MOE_OVL_BUF_Y: base = L.Y; cap = P * (size_t)L.dout * 2; break;
     default: return MOE_OVL_ERR_INVALID_ARG;
     }
     if (offset > cap || bytes > cap - offset) return MOE_OVL_ERR_INVALID_ARG;

@@ -62,9 +62,9 @@ __device__ __forceinline__ void move_segments(const Params &p, volatile int *s_s
         const int s = s_seg[0];
         if (s >= nseg || !s_seg[1]) return;
         const int4 seg = p.segs[s];
-        const uint16_t *src = p.Y + (size_t)seg.x * TB_M * p.d;
-        uint16_t *dst = p.ret + ((size_t)seg.z * p.ret_rows_per_rank + p.seg_slot0[s]) * p.d;
-        copy_rows_16B(src, dst, (size_t)seg.w * p.d / 8, threadIdx.x, blockDim.x);
+        const uint16_t *src = p.Y + (size_t)seg.x * TB_M * p.dout;
+        uint16_t *dst = p.ret + ((size_t)seg.z * p.ret_rows_per_rank + p.seg_slot0[s]) * p.dout;
+        copy_rows_16B(src, dst, (size_t)seg.w * p.dout / 8, threadIdx.x, blockDim.x);
     }
 }
 
@@ -89,9 +89,9 @@ __global__ void __launch_bounds__(256) scatter_kernel(const Params p)
         const int r0 = chunk * rows_per_chunk;
         if (r0 >= valid) continue;
         const int rows = min(rows_per_chunk, valid - r0);
-        const uint16_t *src = p.Y + ((size_t)band * TB_M + r0) * p.d;
-        uint16_t *dst = p.ret + ((size_t)p.band_dest[band] * p.ret_rows_per_rank + p.band_slot0[band] + r0) * p.d;
-        copy_rows_16B(src, dst, (size_t)rows * p.d / 8, threadIdx.x, blockDim.x);
+        const uint16_t *src = p.Y + ((size_t)band * TB_M + r0) * p.dout;
+        uint16_t *dst = p.ret + ((size_t)p.band_dest[band] * p.ret_rows_per_rank + p.band_slot0[band] + r0) * p.dout;
+        copy_rows_16B(src, dst, (size_t)rows * p.dout / 8, threadIdx.x, blockDim.x);
     }
 }
 
@@ -100,7 +100,7 @@ __global__ void __launch_bounds__(256) scatter_kernel(const Params p)
 __global__ void __launch_bounds__(256) combine_kernel(const Params p)
 {
     const int ntok = p.R * p.T;
-    const int nv = p.d / 8;
+    const int nv = p.dout / 8;
     constexpr int KFAST = 2;                      // list entries kept in registers
     int slot[KFAST];
     float gate[KFAST];
@@ -114,8 +114,8 @@ __global__ void __launch_bounds__(256) combine_kernel(const Params p)
     };
     fetch(blockIdx.x);
     for (int tok = blockIdx.x; tok < ntok; tok += gridDim.x) {
-        const uint16_t *region = p.ret + (size_t)(tok / p.T) * p.ret_rows_per_rank * p.d;
-        uint4 *o = reinterpret_cast<uint4 *>(p.out + (size_t)tok * p.d);
+        const uint16_t *region = p.ret + (size_t)(tok / p.T) * p.ret_rows_per_rank * p.dout;
+        uint4 *o = reinterpret_cast<uint4 *>(p.out + (size_t)tok * p.dout);
         int cs[KFAST];
         float cg[KFAST];
 #pragma unroll
@@ -125,7 +125,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const Params p)
             uint4 row[KFAST];
 #pragma unroll
             for (int j = 0; j < KFAST; ++j)
-                row[j] = cs[j] > 0 ? __ldcs(reinterpret_cast<const uint4 *>(region + (size_t)(cs[j] - 1) * p.d) + v)
+                row[j] = cs[j] > 0 ? __ldcs(reinterpret_cast<const uint4 *>(region + (size_t)(cs[j] - 1) * p.dout) + v)
                                    : make_uint4(0, 0, 0, 0);
             float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
             auto add = [&](const uint4 &q, float g) {
@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const Params p)
                 for (int j = KFAST; j < p.kmax; ++j) {        // tokens with more than two local rows
                     const int s = p.tok_slot[(size_t)tok * p.kmax + j];
                     if (s <= 0) break;
-                    add(__ldcs(reinterpret_cast<const uint4 *>(region + (size_t)(s - 1) * p.d) + v),
+                    add(__ldcs(reinterpret_cast<const uint4 *>(region + (size_t)(s - 1) * p.dout) + v),
                         p.tok_gate[(size_t)tok * p.kmax + j]);
                 }
             }

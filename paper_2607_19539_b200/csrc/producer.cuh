@@ -323,13 +323,16 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     b_row = e * 2 * p.F + tile * H_TILE + (int)rank * p.F;
                     ksteps = p.d / TB_K;
                 } else {
-                    amap = &maps.h; bmap = &maps.w2;
-                    b_row = e * p.d + tile * TB_N + (int)rank * (TB_N / 2);
-                    ksteps = p.F / TB_K;
-                    // every first-GEMM tile of this band must have landed in H
-                    ok = wait_global(&p.hcount[band], (unsigned)p.n1, true, p, SITE_TMA_HCOUNT, band);
-                    if (!ok) break;
-                    asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
+                    // single-projection experts: the output GEMM reads the aligned input itself
+                    amap = p.single ? &maps.xa : &maps.h; bmap = &maps.w2;
+                    b_row = e * p.dout + tile * TB_N + (int)rank * (TB_N / 2);
+                    ksteps = p.k2 / TB_K;
+                    if (p.n1 > 0) {
+                        // every first-GEMM tile of this band must have landed in H
+                        ok = wait_global(&p.hcount[band], (unsigned)p.n1, true, p, SITE_TMA_HCOUNT, band);
+                        if (!ok) break;
+                        asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
+                    }
                 }
                 const int a_row = band * TB_M;
                 for (int ks = 0; ks < ksteps; ++ks) {
@@ -370,7 +373,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 const int it = claimed(n);
                 if (it < 0 || it >= n_items) break;
                 const int kind = p.items[it].x & 0xff;
-                const int ksteps = (kind == KIND_G1 ? p.d : p.F) / TB_K;
+                const int ksteps = (kind == KIND_G1 ? p.d : p.k2) / TB_K;
                 ok = mbar_wait<true>(bar_tempty + 8 * acc, acc_phase ^ 1u, p, SITE_MMA_TEMPTY, it);
                 if (!ok) break;
                 tc_fence_after();
@@ -457,7 +460,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     for (int j = 0; j < 4; ++j) d4[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
                 }
             } else {
-                uint16_t *dst = p.Y + grow * p.d + (size_t)tile * TB_N;
+                uint16_t *dst = p.Y + grow * p.dout + (size_t)tile * TB_N;
 #pragma unroll 1
                 for (int c = 0; c < TB_N; c += 32) {
                     uint32_t v[32];

@@ -53,9 +53,9 @@ def upload(inp: MoEInputs, dsp: Dispatched, device="cuda:0", w1: Optional[torch.
         expert_counts=i32(dsp.expert_counts), src_rank=i32(dsp.src_rank), src_token=i32(dsp.src_token),
         gate=torch.from_numpy(np.ascontiguousarray(dsp.gate, np.float32)).to(dev),
         w1=bits_to_device(inp.w1, dev) if w1 is None else w1,
-        w2=bits_to_device(inp.w2, dev) if w2 is None else w2,
-        ret=torch.full((sh.R, sh.T * sh.kmax, sh.d), float("nan"), dtype=torch.bfloat16, device=dev),
-        out=torch.full((sh.R * sh.T, sh.d), float("nan"), dtype=torch.bfloat16, device=dev),
+        w2=(bits_to_device(inp.w2, dev) if inp.w2.size else None) if w2 is None else w2,
+        ret=torch.full((sh.R, sh.T * sh.kmax, sh.dout), float("nan"), dtype=torch.bfloat16, device=dev),
+        out=torch.full((sh.R * sh.T, sh.dout), float("nan"), dtype=torch.bfloat16, device=dev),
         slot_out=torch.full((max(M, 1),), -7, dtype=torch.int32, device=dev),
         rows_per_rank_out=torch.full((sh.R,), -7, dtype=torch.int32, device=dev),
         segs_per_rank_out=torch.full((sh.R,), -7, dtype=torch.int32, device=dev),
@@ -65,7 +65,7 @@ def upload(inp: MoEInputs, dsp: Dispatched, device="cuda:0", w1: Optional[torch.
 def make_context(shape: MoEShape, max_rows: int, device: int = 0, **kw) -> B.MoeOvl:
     cfg = B.make_config(device=device, num_src_ranks=shape.R, self_rank=shape.self_rank, tokens_per_rank=shape.T,
                         num_local_experts=shape.El, top_k=shape.k, d_model=shape.d, d_ffn=shape.F,
-                        max_rows=max_rows, **kw)
+                        single_gemm_out=shape.N_out, max_rows=max_rows, **kw)
     return B.MoeOvl(cfg)
 
 

@@ -13,7 +13,8 @@ for a dataset.  Recipe:
 
 * tokens ``x[R, T, d] ~ N(0, 1)`` rounded to bf16;
 * expert weights ``W1[El, 2F, d]`` (rows ``0..F-1`` gate projection, rows
-  ``F..2F-1`` up projection) and ``W2[El, d, F]``, both ``~ N(0, 1/d)``, bf16;
+  ``F..2F-1`` up projection) and ``W2[El, d, F]``, both ``~ N(0, 1/d)``, bf16
+  (single-projection shapes: one ``W[El, N, d] ~ N(0, 1/d)`` per expert);
 * router logits ``l[R, T, Eg] ~ N(0, 1)``;
 * ``uniform`` router: experts = top-k of the logits, gate = softmax of the k
   selected logits (fp32);
@@ -47,6 +48,11 @@ class MoEShape:
     self_rank: int = 0
     first_local: int = 0      # global id of local expert 0
     zipf_s: float = 1.2
+    N_out: int = 0            # > 0: each expert is one projection y = x W^T, W[N_out, d] (the paper's operator); F unused
+
+    @property
+    def dout(self) -> int:
+        return self.N_out if self.N_out > 0 else self.d
 
     @property
     def kmax(self) -> int:
@@ -62,6 +68,13 @@ SHAPES: Dict[str, MoEShape] = {
     "fine": MoEShape("fine", R=8, T=8192, Eg=64, k=6, El=8, d=2048, F=1408),
     # a quarter of the Mixtral-shaped layer's tokens, same weights: small enough for a full profiler capture
     "mixtral_quarter": MoEShape("mixtral_quarter", R=4, T=1024, Eg=8, k=2, El=2, d=4096, F=14336),
+    # the operator the paper evaluates (Table 2): one projection per expert, M = 2 x tokens-per-rank rows,
+    # K = 2048, N = 8192, E experts per rank, 4 ranks, top-2
+    "paper_op_e4": MoEShape("paper_op_e4", R=4, T=8192, Eg=16, k=2, El=4, d=2048, F=0, N_out=8192),
+    "paper_op_e16": MoEShape("paper_op_e16", R=4, T=8192, Eg=64, k=2, El=16, d=2048, F=0, N_out=8192),
+    "paper_op_e16_zipf": MoEShape("paper_op_e16_zipf", R=4, T=8192, Eg=64, k=2, El=16, d=2048, F=0, N_out=8192,
+                                  router="zipf"),
+    "single_small": MoEShape("single_small", R=3, T=600, Eg=6, k=2, El=2, d=192, F=0, N_out=512, self_rank=2, seed=2),
     # mid-size shapes for parity tests (several bands per group, ragged tails)
     "small": MoEShape("small", R=3, T=700, Eg=6, k=2, El=3, d=512, F=384, self_rank=1),
     "small_zipf_rot": MoEShape("small_zipf_rot", R=4, T=900, Eg=8, k=3, El=2, d=256, F=640,
@@ -143,7 +156,10 @@ def make_inputs(shape: MoEShape, weights: bool = True) -> MoEInputs:
     rng = np.random.Generator(np.random.PCG64(shape.seed))
     x = _normal_bf16(rng, (shape.R, shape.T, shape.d), 1.0)
     expert, gate = make_router(shape, rng)
-    if weights:
+    if weights and shape.N_out > 0:
+        w1 = _normal_bf16(rng, (shape.El, shape.N_out, shape.d), float(shape.d) ** -0.5)
+        w2 = np.zeros((0,), np.uint16)
+    elif weights:
         s = float(shape.d) ** -0.5
         w1 = _normal_bf16(rng, (shape.El, 2 * shape.F, shape.d), s)
         w2 = _normal_bf16(rng, (shape.El, shape.d, shape.F), s)

@@ -18,7 +18,7 @@ def rel_dist(a, b):
 
 def oracle_plan(shape, dsp, mgb=1):
     return build_plan(dsp.expert_counts.tolist(), dsp.src_rank.tolist(), dsp.src_token.tolist(), shape.R,
-                      shape.self_rank, 128, mgb, shape.d // 256, gate=dsp.gate.tolist(), T=shape.T)
+                      shape.self_rank, 128, mgb, shape.dout // 256, gate=dsp.gate.tolist(), T=shape.T)
 
 
 def check_indices(shape, dsp, plan, gpu_plan, slot_out, rows_per_rank, segs_per_rank, report):
@@ -56,7 +56,7 @@ def check_indices(shape, dsp, plan, gpu_plan, slot_out, rows_per_rank, segs_per_
         if b1 >= 0:
             rows.append((x & 0xff, b1, tile, x >> 8))
     items = np.asarray(rows, np.int64).reshape(-1, 4)
-    n1, n2 = shape.F // 128, shape.d // 256
+    n1, n2 = (0 if shape.N_out else shape.F // 128), shape.dout // 256
     g2 = items[items[:, 0] == 1]
     g1 = items[items[:, 0] == 0]
     expect = sorted((b.band, j) for b in plan.bands for j in range(n2))
@@ -73,7 +73,7 @@ def check_indices(shape, dsp, plan, gpu_plan, slot_out, rows_per_rank, segs_per_
     runs = [e for i, e in enumerate(ex) if i == 0 or ex[i - 1] != e]
     assert runs == [e for e in plan.expert_order if any(b.expert == e and not b.local for b in plan.bands)]
     # a second-GEMM tile is issued after every first-GEMM tile of its band
-    last_g1 = {}
+    last_g1 = {b.band: -1 for b in plan.bands}
     for idx, (kind, b, j, e) in enumerate(items.tolist()):
         if kind == 0:
             last_g1[b] = idx
@@ -83,6 +83,9 @@ def check_indices(shape, dsp, plan, gpu_plan, slot_out, rows_per_rank, segs_per_
 
 def oracle_values(inp, tokens):
     sh = inp.shape
+    if sh.N_out:
+        return VO.forward_tokens_single(inp.x, inp.expert, inp.gate, inp.w1, sh.El, sh.first_local,
+                                        np.asarray(tokens, np.int32))
     return VO.forward_tokens(inp.x, inp.expert, inp.gate, inp.w1, inp.w2, sh.El, sh.first_local,
                              np.asarray(tokens, np.int32))
 

@@ -27,7 +27,7 @@ def test_header_symbols_are_exported_and_bound():
 
 def test_struct_sizes_match_header_layout():
     # field-by-field mirror of the header; sizes are what the library checks in struct_size
-    assert ctypes.sizeof(B.Config) == 15 * 4
+    assert ctypes.sizeof(B.Config) == 16 * 4
     assert ctypes.sizeof(B.Args) == 8 + 7 * 8 + 8 + 8 + 8 + 8 + 3 * 8 + 8
     assert ctypes.sizeof(B.Report) == 8 * 4 + 6 * 4
 
@@ -54,6 +54,7 @@ def test_workspace_and_limits_are_host_arithmetic():
     (dict(d_model=300), B.ERR_UNSUPPORTED), (dict(d_ffn=100), B.ERR_UNSUPPORTED),
     (dict(self_rank=4), B.ERR_INVALID_ARG), (dict(num_local_experts=0), B.ERR_INVALID_ARG),
     (dict(num_local_experts=300), B.ERR_UNSUPPORTED), (dict(max_rows=-1), B.ERR_INVALID_ARG),
+    (dict(single_gemm_out=100), B.ERR_UNSUPPORTED), (dict(single_gemm_out=512, d_model=100), B.ERR_UNSUPPORTED),
 ])
 def test_config_errors(kw, code):
     with pytest.raises(B.MoeOvlError) as e:

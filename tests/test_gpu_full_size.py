@@ -28,7 +28,7 @@ def sample_tokens(shape, dsp, per_rank, seed=0):
 
 
 @pytest.mark.parametrize("name,csm,per_rank", [
-    ("mixtral", 8, 16), ("fine", 8, 24), ("mixtral_zipf", 8, 8),
+    ("mixtral", 8, 16), ("fine", 8, 24), ("mixtral_zipf", 8, 8), ("paper_op_e16_zipf", 14, 16),
     # points of the sweep grid: 4 local experts of 16, d=4096; (tokens per local expert, ffn, router)
     ((1024, 1024, "uniform"), 2, 16), ((128, 2816, "zipf"), 16, 8), ((4096, 1024, "zipf"), 32, 8),
 ])
@@ -59,7 +59,7 @@ def test_full_size_parity(name, csm, per_rank):
     pos, slot = np.asarray(plan.pos), np.asarray(plan.slot)
     assert (ret[dsp.src_rank, slot] == Y[pos]).all()
     # (3) every token: out is the gate-weighted sum of its returned rows (recomputed here from the GPU's ret)
-    acc = np.zeros((shape.R * shape.T, shape.d), np.float32)
+    acc = np.zeros((shape.R * shape.T, shape.dout), np.float32)
     tok = dsp.src_rank.astype(np.int64) * shape.T + dsp.src_token
     for e in range(shape.El):                                  # ascending expert = accumulation order
         rows = np.nonzero(dsp.row_expert == e)[0]

@@ -148,3 +148,48 @@ def test_token_subset_and_threads_agree():
     full = VO.forward_tokens(inp.x, inp.expert, inp.gate, inp.w1, inp.w2, shape.El, 0,
                              np.arange(shape.R * shape.T, dtype=np.int32))
     assert (full[0][sel] == a[0]).all()
+
+
+# ---- single-projection experts (the operator of Table 2)
+
+def test_single_projection_against_float64_and_library():
+    shape = I.MoEShape("sp", R=2, T=19, Eg=4, k=2, El=3, d=48, F=0, N_out=80, first_local=1, seed=6)
+    inp = I.make_inputs(shape)
+    toks = np.arange(shape.R * shape.T, dtype=np.int32)
+    out, y, y_exp = VO.forward_tokens_single(inp.x, inp.expert, inp.gate, inp.w1, shape.El, shape.first_local, toks)
+    x = I.bf16_bits_to_f32(inp.x).astype(np.float64).reshape(-1, shape.d)
+    w = I.bf16_bits_to_f32(inp.w1).astype(np.float64)
+    ex = inp.expert.reshape(-1, shape.k)
+    gt = inp.gate.reshape(-1, shape.k).astype(np.float64)
+    ref = np.zeros((len(toks), shape.N_out))
+    for s, tok in enumerate(toks):
+        loc = []
+        for q in range(shape.k):
+            e = ex[tok, q] - shape.first_local
+            if 0 <= e < shape.El:
+                ref[s] += gt[tok, q] * (w[e] @ x[tok])
+                loc.append(int(e))
+        assert [int(v) for v in y_exp[s] if v >= 0] == sorted(loc)
+        for j, e in enumerate(sorted(loc)):
+            assert rel_dist(I.bf16_bits_to_f32(y[s, j])[None], (w[e] @ x[tok])[None])[0] < 1e-2
+    has = np.linalg.norm(ref, axis=1) > 0
+    assert rel_dist(I.bf16_bits_to_f32(out)[has], ref[has]).max() < 1e-2
+    assert (out[~has] == 0).all()
+    # one expert, unit gate: a library matmul
+    sh1 = I.MoEShape("sp1", R=1, T=21, Eg=1, k=1, El=1, d=64, F=0, N_out=32, seed=9)
+    in1 = I.make_inputs(sh1)
+    in1.gate[:] = 1.0
+    o1, y1, _ = VO.forward_tokens_single(in1.x, in1.expert, in1.gate, in1.w1, 1, 0, np.arange(21, dtype=np.int32))
+    lib = torch.from_numpy(I.bf16_bits_to_f32(in1.x[0])) @ torch.from_numpy(I.bf16_bits_to_f32(in1.w1[0])).T
+    assert rel_dist(I.bf16_bits_to_f32(o1), lib.numpy()).max() < 1e-2
+    assert (o1 == y1[:, 0]).all()
+
+
+def test_single_projection_identity_is_exact():
+    shape = I.MoEShape("spi", R=2, T=30, Eg=2, k=1, El=2, d=64, F=0, N_out=64, seed=3)
+    inp = I.make_inputs(shape)
+    inp.w1 = I.f32_to_bf16_bits(np.broadcast_to(np.eye(64, dtype=np.float32), (2, 64, 64)).copy())
+    inp.gate[:] = 1.0
+    toks = np.arange(60, dtype=np.int32)
+    out, y, _ = VO.forward_tokens_single(inp.x, inp.expert, inp.gate, inp.w1, 2, 0, toks)
+    assert (out == inp.x.reshape(-1, 64)).all() and (y[:, 0] == inp.x.reshape(-1, 64)).all()
