@@ -28,9 +28,9 @@ import numpy as np  # noqa: E402
 METRIC = "moe_expert_return_tflops"
 UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of one producer launch, from the one-pass ncu launch lists of the
-# full-size workloads summarised in profiles/.
-NCU_PRODUCER_TRAFFIC_BYTES = {"mixtral": 3953099008 + 309059200, "fine": 497301248 + 342024576}
+# dram__bytes_read.sum + dram__bytes_write.sum of one producer launch at full size, from the ncu capture
+# summarised in profiles/producer_kernel_mixtral.md.
+NCU_PRODUCER_TRAFFIC_BYTES = {"mixtral": 2714303000 + 312693248}
 
 
 def load_peaks():
