@@ -274,12 +274,13 @@ def main():
 
     # the GEMM kernel's own duration, measured per launch by the library with CUDA events on the stream it
     # is launched on; averaged over a few extra steps
-    prod_ms, mover_ms, er_ms, prep_ms, comb_ms = [], [], [], [], []
+    prod_ms, mover_ms, er_ms, prep_ms, comb_ms, ovl_ratio, assist = [], [], [], [], [], [], []
     for _ in range(min(args.steps, 10)):
         Hn.run(ctx, prob, mode=head_mode, consumer_sm_count=args.consumer_sms)
         r = ctx.moe_ovl_get_report()
         prod_ms.append(r.ms_producer); mover_ms.append(r.ms_mover); er_ms.append(r.ms_expert_return)
         prep_ms.append(r.ms_prep); comb_ms.append(r.ms_combine)
+        ovl_ratio.append(r.overlap_ratio); assist.append(r.segments_by_gemm_ctas)
     prod = statistics.mean(prod_ms)
     peak_tf = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
     achieved = step_flops / (prod / 1e3) / 1e12
@@ -372,6 +373,8 @@ def main():
             "combine_us": statistics.mean(comb_ms) * 1e3, "consumer_busy_window_us": statistics.mean(mover_ms) * 1e3,
             "rows": M, "padded_rows": rep.padded_rows, "tiles": rep.num_items, "segments": rep.num_segments,
             "producer_ctas": rep.producer_ctas, "consumer_ctas": rep.consumer_ctas,
+            "overlap_ratio": statistics.mean(ovl_ratio) if args.mode == "overlap" else None,
+            "segments_moved_by_gemm_ctas": statistics.mean(assist) if args.mode == "overlap" else None,
             "roofline": roofline, "non_overlap": non_overlap, "consumer_sm_sweep": sweep,
             "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": rep.kernel_launches * args.steps,
             "clocks": clocks, "paper_context": "paper reports ratios only (up to 2.74x MoE layer, 2.64x end to "

@@ -137,13 +137,20 @@ typedef struct {
     int32_t producer_ctas;
     int32_t consumer_ctas;    /* 0 in NON_OVERLAP */
     int32_t kernel_launches;  /* kernels of this library launched by the call */
-    int32_t reserved;
+    int32_t segments_by_gemm_ctas; /* OVERLAP: segments moved by GEMM CTAs that had run out of tiles */
     float ms_total;           /* whole call on the caller's stream */
     float ms_prep;            /* plan + gather into the aligned layout */
     float ms_expert_return;   /* start of the GEMM to the last row landed in ret */
     float ms_producer;        /* the GEMM kernel alone */
     float ms_mover;           /* consumer (OVERLAP: concurrent with the GEMM) or scatter kernel */
     float ms_combine;
+    /* device timestamps (%globaltimer), microseconds after the first GEMM CTA started; OVERLAP mode */
+    float us_first_flag;      /* first output tile flagged: the consumer's window opens */
+    float us_gemm_done;       /* last output tile flagged */
+    float us_return_done;     /* last segment landed in ret */
+    float overlap_ratio;      /* share of the return window that lies before us_gemm_done:
+                                 1 - max(0, us_return_done - us_gemm_done) / (us_return_done - us_first_flag);
+                                 the share of the second all-to-all hidden behind expert compute (Section 4.2.2) */
 } moe_ovl_report;
 
 /* Integer plan arrays of the last call, copied to HOST buffers (any pointer may be
@@ -206,6 +213,9 @@ int moe_ovl_query_status(moe_ovl_ctx *ctx, int32_t *code, int64_t *detail);
  * `bytes` bytes at `offset` of an internal bf16 buffer (MOE_OVL_BUF_*) to HOST memory. */
 int moe_ovl_get_report(moe_ovl_ctx *ctx, moe_ovl_report *report);
 int moe_ovl_get_plan(moe_ovl_ctx *ctx, const moe_ovl_plan_view *view);
+/* SM (%smid) every GEMM CTA and every consumer CTA of the last call ran on; HOST arrays of
+ * producer_ctas and consumer_ctas entries (moe_ovl_report).  The two kernels must not share an SM. */
+int moe_ovl_get_sm_map(moe_ovl_ctx *ctx, int32_t *producer_smid, int32_t *consumer_smid);
 int moe_ovl_read_buffer(moe_ovl_ctx *ctx, int32_t which, size_t offset, size_t bytes, void *host_dst);
 
 int moe_ovl_destroy(moe_ovl_ctx *ctx);

@@ -26,7 +26,7 @@ TB_M, TB_N, H_TILE = 128, 256, 128
 EXPORTS = [
     "moe_ovl_workspace_bytes", "moe_ovl_limits", "moe_ovl_create", "moe_ovl_expert_return",
     "moe_ovl_expert_return_host", "moe_ovl_host_join", "moe_ovl_query_status", "moe_ovl_get_report", "moe_ovl_get_plan",
-    "moe_ovl_read_buffer", "moe_ovl_destroy", "moe_ovl_strerror", "moe_ovl_last_cuda_error",
+    "moe_ovl_get_sm_map", "moe_ovl_read_buffer", "moe_ovl_destroy", "moe_ovl_strerror", "moe_ovl_last_cuda_error",
     "moe_ovl_return_slots_static",
 ]
 
@@ -58,9 +58,10 @@ class HostArgs(C.Structure):
 class Report(C.Structure):
     _fields_ = [("padded_rows", C.c_int32), ("num_bands", C.c_int32), ("num_items", C.c_int32),
                 ("num_segments", C.c_int32), ("producer_ctas", C.c_int32), ("consumer_ctas", C.c_int32),
-                ("kernel_launches", C.c_int32), ("reserved", C.c_int32), ("ms_total", C.c_float),
+                ("kernel_launches", C.c_int32), ("segments_by_gemm_ctas", C.c_int32), ("ms_total", C.c_float),
                 ("ms_prep", C.c_float), ("ms_expert_return", C.c_float), ("ms_producer", C.c_float),
-                ("ms_mover", C.c_float), ("ms_combine", C.c_float)]
+                ("ms_mover", C.c_float), ("ms_combine", C.c_float), ("us_first_flag", C.c_float),
+                ("us_gemm_done", C.c_float), ("us_return_done", C.c_float), ("overlap_ratio", C.c_float)]
 
 
 class PlanView(C.Structure):
@@ -106,6 +107,7 @@ def load(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moe_ovl_query_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
     lib.moe_ovl_get_report.argtypes = [C.c_void_p, C.POINTER(Report)]
     lib.moe_ovl_get_plan.argtypes = [C.c_void_p, C.POINTER(PlanView)]
+    lib.moe_ovl_get_sm_map.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     lib.moe_ovl_read_buffer.argtypes = [C.c_void_p, C.c_int32, C.c_size_t, C.c_size_t, C.c_void_p]
     lib.moe_ovl_destroy.argtypes = [C.c_void_p]
     lib.moe_ovl_last_cuda_error.argtypes = [C.c_void_p]
@@ -181,6 +183,11 @@ class ReportView:
     ms_producer: float
     ms_mover: float
     ms_combine: float
+    segments_by_gemm_ctas: int = 0
+    us_first_flag: float = 0.0
+    us_gemm_done: float = 0.0
+    us_return_done: float = 0.0
+    overlap_ratio: float = 0.0
 
 
 class MoeOvl:
@@ -243,7 +250,8 @@ class MoeOvl:
         self._check(self.lib.moe_ovl_get_report(self.ctx, C.byref(r)), "moe_ovl_get_report")
         return ReportView(r.padded_rows, r.num_bands, r.num_items, r.num_segments, r.producer_ctas, r.consumer_ctas,
                           r.kernel_launches, r.ms_total, r.ms_prep, r.ms_expert_return, r.ms_producer, r.ms_mover,
-                          r.ms_combine)
+                          r.ms_combine, r.segments_by_gemm_ctas, r.us_first_flag, r.us_gemm_done, r.us_return_done,
+                          r.overlap_ratio)
 
     def moe_ovl_get_plan(self) -> Dict[str, np.ndarray]:
         rep = self.moe_ovl_get_report()
@@ -263,6 +271,13 @@ class MoeOvl:
         arrs["tok_slot"] = arrs["tok_slot"].reshape(-1, self.kmax)
         arrs["tok_gate"] = arrs["tok_gate"].reshape(-1, self.kmax)
         return arrs
+
+    def moe_ovl_get_sm_map(self):
+        rep = self.moe_ovl_get_report()
+        prod = np.full(max(rep.producer_ctas, 1), -1, np.int32)
+        cons = np.full(max(rep.consumer_ctas, 1), -1, np.int32)
+        self._check(self.lib.moe_ovl_get_sm_map(self.ctx, prod.ctypes.data, cons.ctypes.data), "moe_ovl_get_sm_map")
+        return prod[:rep.producer_ctas], cons[:rep.consumer_ctas]
 
     def moe_ovl_read_buffer(self, which: int, row0: int, rows: int) -> np.ndarray:
         """Rows [row0, row0+rows) of the aligned input (BUF_XA), hidden (BUF_H) or output (BUF_Y) buffer, bf16 bits."""

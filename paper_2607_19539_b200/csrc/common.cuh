@@ -18,6 +18,8 @@ constexpr int KIND_G2 = 1;    // H . W2 -> Y, raises the consumer-visible flag
 
 // meta[] slots written by the plan kernel
 enum { META_P = 0, META_BANDS, META_ITEMS, META_SEGS, META_SUPERBANDS, META_COUNT = 8 };
+// stamps[] slots.  "first" stamps hold ~t so that the cleared state (0) is neutral under atomicMax.
+enum { STAMP_START_INV = 0, STAMP_FIRST_FLAG_INV, STAMP_LAST_FLAG, STAMP_LAST_SEG, STAMP_COUNT };
 // status[] slots
 enum { ST_CODE = 0, ST_ABORT = 1, ST_DETAIL_LO = 2, ST_DETAIL_HI = 3, ST_COUNT = 4 };
 
@@ -71,6 +73,9 @@ struct Params {
     int *tok_slot;        // [R*T*kmax] slot + 1 of each of the token's rows, ascending expert; 0 = none
     float *tok_gate;      // [R*T*kmax]
     int *plan_ticket;     // blocks of the plan kernel that have finished marking
+    unsigned long long *stamps;   // [STAMP_COUNT] device timestamps of the call, see the enum
+    int *smid_prod, *smid_cons;   // SM of every GEMM / consumer CTA
+    int *assist_segs;     // segments moved by GEMM CTAs
     int *next_seg;        // segments claimed so far (consumer CTAs, and GEMM CTAs once they are out of tiles)
     int *next_item;       // schedule items claimed so far (GEMM CTA pairs take them in order)
     unsigned *hcount;     // [max_bands] first-GEMM tiles finished per band
@@ -106,6 +111,14 @@ __device__ __forceinline__ unsigned long long globaltimer_ns()
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
+}
+
+__device__ __forceinline__ void stamp_max(unsigned long long *slot, unsigned long long v) { atomicMax(slot, v); }
+__device__ __forceinline__ unsigned smid()
+{
+    unsigned v;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(v));
+    return v;
 }
 
 // First error wins; every later waiter sees ST_ABORT and gives up at once.

@@ -29,7 +29,8 @@ inline size_t align_up(size_t v, size_t a = ALIGN) { return (v + a - 1) / a * a;
 struct Layout {
     // offsets into the workspace, in bytes
     size_t Xa, H, Y;
-    size_t zero_begin, bitmap, hcount, status, next_item, tok_slot, zero_end;   // cleared at the start of every call
+    size_t zero_begin, bitmap, hcount, status, next_item, stamps, tok_slot, zero_end;   // cleared at the start of every call
+    size_t smid;
     size_t wordpfx, group_rows, group_start, group_slot, pos, slot;
     size_t band_expert, band_dest, band_valid, band_slot0, sched_band, items, segs, seg_slot0;
     size_t tok_gate, flags, meta;
@@ -93,7 +94,8 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->bitmap = take((size_t)G * L->words * 4);
     L->hcount = take((size_t)L->max_bands * 4);
     L->status = take(ST_COUNT * 4);
-    L->next_item = take(12);
+    L->next_item = take(16);                 // next_item, plan_ticket, next_seg, assist_segs
+    L->stamps = take(STAMP_COUNT * 8);
     L->tok_slot = take(ntok * L->kmax * 4);
     L->zero_end = off;
     L->tok_gate = take(ntok * L->kmax * 4);
@@ -113,6 +115,7 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->seg_slot0 = take((size_t)L->max_bands * 4);
     L->flags = take((size_t)L->max_bands * L->n2 * 4);
     L->meta = take(META_COUNT * 4);
+    L->smid = take(2 * 1024 * 4);            // SM of every GEMM CTA, then of every consumer CTA
     for (int i = 0; i < 6; ++i) L->sb[i] = take((size_t)L->max_bands * 4);
     L->st_ret_rows = (long long)c->tokens_per_rank * L->kmax;
     if (c->flags & MOE_OVL_FLAG_HOST_STAGING) {
@@ -210,6 +213,10 @@ Params make_params(moe_ovl_ctx *ctx)
     p.next_item = at<int>(ctx, L.next_item);
     p.plan_ticket = at<int>(ctx, L.next_item) + 1;
     p.next_seg = at<int>(ctx, L.next_item) + 2;
+    p.assist_segs = at<int>(ctx, L.next_item) + 3;
+    p.stamps = at<unsigned long long>(ctx, L.stamps);
+    p.smid_prod = at<int>(ctx, L.smid);
+    p.smid_cons = at<int>(ctx, L.smid) + 1024;
     p.flags = at<unsigned>(ctx, L.flags); p.meta = at<int>(ctx, L.meta); p.status = at<int>(ctx, L.status);
     return p;
 }
@@ -574,6 +581,22 @@ int moe_ovl_get_report(moe_ovl_ctx *ctx, moe_ovl_report *r)
     CU_CHECK(ctx, cudaEventElapsedTime(&mover_end, ctx->t_prep, ctx->t_m1));
     r->ms_expert_return = std::max(prod_end, mover_end);
     r->ms_combine = r->ms_total - r->ms_prep - r->ms_expert_return;
+    if (ctx->last_mode == MOE_OVL_MODE_OVERLAP && meta[META_SEGS] > 0) {
+        unsigned long long st[STAMP_COUNT];
+        int misc[4];
+        CU_CHECK(ctx, cudaMemcpy(st, ctx->ws + ctx->L.stamps, sizeof(st), cudaMemcpyDeviceToHost));
+        CU_CHECK(ctx, cudaMemcpy(misc, ctx->ws + ctx->L.next_item, sizeof(misc), cudaMemcpyDeviceToHost));
+        const unsigned long long t0 = ~st[STAMP_START_INV], first = ~st[STAMP_FIRST_FLAG_INV];
+        if (st[STAMP_FIRST_FLAG_INV] != 0 && st[STAMP_LAST_SEG] != 0) {
+            r->us_first_flag = (float)((double)(first - t0) / 1e3);
+            r->us_gemm_done = (float)((double)(st[STAMP_LAST_FLAG] - t0) / 1e3);
+            r->us_return_done = (float)((double)(st[STAMP_LAST_SEG] - t0) / 1e3);
+            const double window = (double)r->us_return_done - r->us_first_flag;
+            const double exposed = std::max(0.0, (double)r->us_return_done - r->us_gemm_done);
+            r->overlap_ratio = window > 0 ? (float)(1.0 - exposed / window) : 1.0f;
+        }
+        r->segments_by_gemm_ctas = misc[3];
+    }
     return MOE_OVL_OK;
 }
 
@@ -606,6 +629,20 @@ int moe_ovl_get_plan(moe_ovl_ctx *ctx, const moe_ovl_plan_view *v)
         if (e.dst && e.bytes) CU_CHECK(ctx, cudaMemcpy(e.dst, ctx->ws + e.off, e.bytes, cudaMemcpyDeviceToHost));
     if (v->tok_slot)                           // stored as slot + 1 with 0 = none; reported as slot with -1 = none
         for (size_t i = 0; i < ntokk; ++i) v->tok_slot[i] -= 1;
+    return MOE_OVL_OK;
+}
+
+int moe_ovl_get_sm_map(moe_ovl_ctx *ctx, int32_t *producer_smid, int32_t *consumer_smid)
+{
+    if (!ctx || !ctx->ran) return MOE_OVL_ERR_INVALID_ARG;
+    int rc = sync_last(ctx);
+    if (rc != MOE_OVL_OK) return rc;
+    if (producer_smid && ctx->last_prod_ctas > 0)
+        CU_CHECK(ctx, cudaMemcpy(producer_smid, ctx->ws + ctx->L.smid, (size_t)ctx->last_prod_ctas * 4,
+                                 cudaMemcpyDeviceToHost));
+    if (consumer_smid && ctx->last_cons_ctas > 0)
+        CU_CHECK(ctx, cudaMemcpy(consumer_smid, ctx->ws + ctx->L.smid + 1024 * 4, (size_t)ctx->last_cons_ctas * 4,
+                                 cudaMemcpyDeviceToHost));
     return MOE_OVL_OK;
 }
 

@@ -37,7 +37,7 @@ __device__ __forceinline__ void copy_rows_16B(const uint16_t *src, uint16_t *dst
 // segment in schedule order, wait (bounded, acquire) until every tile of every one of its bands is flagged,
 // then move its valid rows into the owner rank's receive buffer with one contiguous copy.
 // s_seg: two ints of shared memory.  All threads of the CTA must call this together.
-__device__ __forceinline__ void move_segments(const Params &p, volatile int *s_seg)
+__device__ __forceinline__ void move_segments(const Params &p, volatile int *s_seg, bool gemm_cta)
 {
     const int nseg = p.meta[META_SEGS];
     const int lane = threadIdx.x & 31;
@@ -65,6 +65,11 @@ __device__ __forceinline__ void move_segments(const Params &p, volatile int *s_s
         const uint16_t *src = p.Y + (size_t)seg.x * TB_M * p.dout;
         uint16_t *dst = p.ret + ((size_t)seg.z * p.ret_rows_per_rank + p.seg_slot0[s]) * p.dout;
         copy_rows_16B(src, dst, (size_t)seg.w * p.dout / 8, threadIdx.x, blockDim.x);
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            stamp_max(&p.stamps[STAMP_LAST_SEG], globaltimer_ns());
+            if (gemm_cta) atomicAdd(p.assist_segs, 1);
+        }
     }
 }
 
@@ -74,7 +79,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MOVER_THREADS, 1) co
 {
     extern __shared__ uint8_t unused_smem[];
     __shared__ int s_seg[2];
-    move_segments(p, s_seg);
+    if (threadIdx.x == 0) p.smid_cons[blockIdx.x] = (int)smid();
+    move_segments(p, s_seg, false);
 }
 
 // One CTA per (band, chunk of rows): grid-stride over bands x chunks.

@@ -256,10 +256,8 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
     const uint32_t bar_ring = bar_go + 8;                          // PROD_RING barriers: slot filled
     const uint32_t ring = bar_ring + 8 * PROD_RING;                // PROD_RING claimed item indices
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    const uint32_t bars_off = PROD_STAGES * PROD_STAGE_BYTES;
     volatile uint32_t *tmem_slot_gen = reinterpret_cast<volatile uint32_t *>(smem_gen + (tmem_slot - smem_base));
     volatile int *ring_gen = reinterpret_cast<volatile int *>(smem_gen + (ring - smem_base));
-    (void)bars_off;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();          // 0 = leader: owns the barriers the pair synchronises on
@@ -267,6 +265,8 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
     const uint32_t lead_full = map_to_cta(bar_full, 0), lead_tempty = map_to_cta(bar_tempty, 0);
 
     if (threadIdx.x == 0) {
+        p.smid_prod[blockIdx.x] = (int)smid();
+        stamp_max(&p.stamps[STAMP_START_INV], ~globaltimer_ns());
         for (int s = 0; s < PROD_STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);       // the leader's TMA thread arrives, expecting both CTAs' bytes
             mbar_init(bar_empty + 8 * s, 1);
@@ -488,7 +488,12 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             bar_sync_epilogue();
             if (leader && present) {
                 if (kind == KIND_G1) red_release_add_u32(&p.hcount[band], 1u);
-                else if (raise_flags) st_release_u32(&p.flags[(size_t)band * p.n2 + tile], p.epoch);
+                else if (raise_flags) {
+                    st_release_u32(&p.flags[(size_t)band * p.n2 + tile], p.epoch);
+                    const unsigned long long now = globaltimer_ns();
+                    stamp_max(&p.stamps[STAMP_FIRST_FLAG_INV], ~now);
+                    stamp_max(&p.stamps[STAMP_LAST_FLAG], now);
+                }
             }
             acc ^= 1;
             if (acc == 0) acc_phase ^= 1u;
@@ -505,7 +510,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
     }
     // Out of tiles: help the consumer drain what is left, so that the last segments do not wait for the few
     // consumer SMs (the tail Section 3.3.3 warns about when the consumer budget is small).
-    if (raise_flags) move_segments(p, reinterpret_cast<volatile int *>(smem_gen));
+    if (raise_flags) move_segments(p, reinterpret_cast<volatile int *>(smem_gen), true);
 }
 
 }  // namespace moe_ovl

@@ -101,6 +101,27 @@ def test_overlap_equals_non_overlap_bitwise(name):
         assert torch.equal(prob.ret.view(torch.int16), ref_ret.view(torch.int16))
 
 
+@pytest.mark.parametrize("csm", [2, 8, 16])
+def test_sm_partition_is_disjoint_and_overlap_is_reported(csm):
+    """Section 3.3.3: the two persistent kernels run on disjoint SM sets, one CTA per SM, and together fill the GPU;
+    the report's device timestamps give the share of the return that is hidden behind the GEMM (Section 4.2.2).
+    (The consumer budget stays below the 25 segments of this problem: a consumer CTA that finds no segment left
+    exits at once and frees its SM for a GEMM CTA that has not started yet, which is fine but not what is tested.)"""
+    torch, B, Hn = _gpu()
+    shape = I.SHAPES["small_zipf_rot"]
+    inp, dsp, ctx, prob = _run_case(shape, B.MODE_OVERLAP, csm)
+    rep = ctx.moe_ovl_get_report()
+    prod, cons = ctx.moe_ovl_get_sm_map()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert len(cons) == csm and len(prod) == sms - csm
+    assert len(set(prod.tolist())) == len(prod) and len(set(cons.tolist())) == len(cons)     # one CTA per SM
+    assert not set(prod.tolist()) & set(cons.tolist())                                        # disjoint partitions
+    assert min(prod.min(), cons.min()) >= 0 and max(prod.max(), cons.max()) < sms
+    assert 0.0 <= rep.us_first_flag <= rep.us_gemm_done and rep.us_return_done > rep.us_first_flag
+    assert 0.0 <= rep.overlap_ratio <= 1.0
+    assert 0 <= rep.segments_by_gemm_ctas <= rep.num_segments
+
+
 def test_automatic_consumer_budget():
     """consumer_sm_count = 0 lets the library size the consumer partition from the shape: small for wide FFNs
     (the return is cheap next to the GEMM), larger for narrow ones; results do not depend on it."""
