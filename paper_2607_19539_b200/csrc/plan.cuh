@@ -15,7 +15,7 @@ namespace moe_ovl {
 constexpr int PLAN_MAX_GROUPS = 1024;   // El * R
 constexpr int PLAN_MAX_EXPERTS = 256;   // El
 constexpr int PLAN_THREADS = 1024;
-constexpr int PLAN_SB_STAGE = 512;      // super-bands whose sizes are staged in shared memory for the serial pass
+constexpr int PLAN_SB_STAGE = 256;      // super-bands whose sizes are staged in shared memory for the serial pass
 
 // Scratch arrays of the plan kernel, one entry per super-band.
 struct PlanScratch {
@@ -96,7 +96,9 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     __shared__ int gsched[PLAN_MAX_GROUPS], gsegoff[PLAN_MAX_GROUPS];
     __shared__ int key[PLAN_MAX_EXPERTS], eorder[PLAN_MAX_EXPERTS];
     __shared__ int run_start[2 * PLAN_MAX_EXPERTS], run_nb[2 * PLAN_MAX_EXPERTS], run_sb0[2 * PLAN_MAX_EXPERTS + 1];
-    __shared__ int run_exp[2 * PLAN_MAX_EXPERTS];
+    __shared__ int run_exp[2 * PLAN_MAX_EXPERTS], run_segs[2 * PLAN_MAX_EXPERTS];
+    __shared__ int esize[PLAN_MAX_EXPERTS];
+    __shared__ int s_total;
     __shared__ int segs_per_rank[PLAN_MAX_GROUPS];
     __shared__ int s_nsb;
     __shared__ int s_sb_nb[PLAN_SB_STAGE], s_sb_end[PLAN_SB_STAGE];
@@ -105,58 +107,79 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     const int G = p.El * p.R;
     const int R = p.R, El = p.El, self = p.r_self;
 
-    // A: per group, exclusive popcount prefix over its bitmap words, and n[e][r]
-    for (int g = warp; g < G; g += nwarps) {
-        const unsigned *bm = p.bitmap + (size_t)g * p.words;
-        int *wp = p.wordpfx + (size_t)g * p.words;
-        int run = 0;
+    // A: per group, exclusive popcount prefix over its bitmap words, and n[e][r].  A warp works on four groups
+    //    at a time so that their (independent) loads are in flight together.
+    for (int g0 = warp * 4; g0 < G; g0 += nwarps * 4) {
+        int run[4] = {0, 0, 0, 0};
         for (int w0 = 0; w0 < p.words; w0 += 32) {
             const int w = w0 + lane;
-            const int c = w < p.words ? __popc(__ldcg(bm + w)) : 0;    // written by other blocks' atomics
-            int inc = c;
+            int c[4];
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int v = __shfl_up_sync(0xffffffffu, inc, o);
-                if (lane >= o) inc += v;
+            for (int k = 0; k < 4; ++k)     // written by other blocks' atomics: read through L2
+                c[k] = (g0 + k < G && w < p.words) ? __popc(__ldcg(p.bitmap + (size_t)(g0 + k) * p.words + w)) : 0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                int inc = c[k];
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, inc, o);
+                    if (lane >= o) inc += v;
+                }
+                if (g0 + k < G && w < p.words) p.wordpfx[(size_t)(g0 + k) * p.words + w] = run[k] + inc - c[k];
+                run[k] += __shfl_sync(0xffffffffu, inc, 31);
             }
-            if (w < p.words) wp[w] = run + inc - c;
-            run += __shfl_sync(0xffffffffu, inc, 31);
         }
-        if (lane == 0) n[g] = run;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (lane == 0 && g0 + k < G) n[g0 + k] = run[k];
     }
     for (int r = tid; r < R; r += blockDim.x) segs_per_rank[r] = 0;
     __syncthreads();
 
     // B: row layout (Algorithm 1): per expert, remote owner groups in ascending rank, local group last,
-    //    every group rounded up to a multiple of tb_M; receive-buffer slots expert-major and dense
-    if (tid == 0) {
-        int total = 0, cursor = 0;
-        for (int e = 0; e < El; ++e) {
-            int remote_bands = 0;
-            for (int q = 0; q < R; ++q) {
-                const int r = q < R - 1 ? (q < self ? q : q + 1) : self;   // remote ranks ascending, then self
-                const int g = e * R + r;
-                gstart[g] = cursor;
-                nb[g] = (n[g] + TB_M - 1) / TB_M;
-                cursor += nb[g] * TB_M;
-                total += n[g];
-                if (r != self) remote_bands += nb[g];
-            }
-            key[e] = remote_bands;
+    //    every group rounded up to a multiple of tb_M; receive-buffer slots expert-major and dense.
+    //    One thread per expert lays out its own groups relative to the expert's start; a short prefix over
+    //    the experts then places the experts.
+    if (tid == 0) s_total = 0;
+    __syncthreads();
+    for (int e = tid; e < El; e += blockDim.x) {
+        int cur = 0, remote_bands = 0, rows = 0;
+        for (int q = 0; q < R; ++q) {
+            const int r = q < R - 1 ? (q < self ? q : q + 1) : self;   // remote ranks ascending, then self
+            const int g = e * R + r;
+            const int nbg = (n[g] + TB_M - 1) / TB_M;
+            gstart[g] = cur;
+            nb[g] = nbg;
+            cur += nbg * TB_M;
+            rows += n[g];
+            if (r != self) remote_bands += nbg;
         }
-        for (int r = 0; r < R; ++r) {
-            int acc = 0;
-            for (int e = 0; e < El; ++e) {
-                gslot[e * R + r] = acc;
-                acc += n[e * R + r];
-            }
-            if (p.rows_per_rank_out) p.rows_per_rank_out[r] = acc;
+        key[e] = remote_bands;
+        esize[e] = cur;
+        atomicAdd(&s_total, rows);
+    }
+    for (int r = tid; r < R; r += blockDim.x) {
+        int acc = 0;
+        for (int e = 0; e < El; ++e) {
+            gslot[e * R + r] = acc;
+            acc += n[e * R + r];
+        }
+        if (p.rows_per_rank_out) p.rows_per_rank_out[r] = acc;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int cursor = 0;
+        for (int e = 0; e < El; ++e) {
+            const int sz = esize[e];
+            esize[e] = cursor;                 // now the expert's first aligned position
+            cursor += sz;
         }
         p.meta[META_P] = cursor;
         p.meta[META_BANDS] = cursor / TB_M;
-        if (total != p.M) report_error(p.status, ERR_BAD_ROUTING, SITE_COUNT_SUM, total);
+        if (s_total != p.M) report_error(p.status, ERR_BAD_ROUTING, SITE_COUNT_SUM, s_total);
     }
     __syncthreads();
+    for (int g = tid; g < G; g += blockDim.x) gstart[g] += esize[g / R];
 
     // C: experts by remote band count, descending; ties to the lower index (Algorithm 1, rule (ii))
     for (int e = tid; e < El; e += blockDim.x) {
@@ -167,25 +190,35 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     __syncthreads();
 
     // D: schedule positions of groups.  Runs: the remote bands of each expert in sorted order (rule (i):
-    //    all remote tiles first), then the local bands of each expert in natural order.
+    //    all remote tiles first), then the local bands of each expert in natural order.  One thread per run
+    //    counts its bands, segments and super-bands; a short prefix over the runs places them.
+    for (int run = tid; run < 2 * El; run += blockDim.x) {
+        const bool remote = run < El;
+        const int e = remote ? eorder[run] : run - El;
+        int nbands = 0, nsegs = 0;
+        for (int q = remote ? 0 : R - 1; q < (remote ? R - 1 : R); ++q) {
+            const int r = q < R - 1 ? (q < self ? q : q + 1) : self;
+            const int g = e * R + r;
+            gsched[g] = nbands;                 // relative to the run for now
+            gsegoff[g] = nsegs;
+            const int ns = num_segments(nb[g], p.mgb);
+            nbands += nb[g];
+            nsegs += ns;
+            atomicAdd(&segs_per_rank[r], ns);
+        }
+        run_exp[run] = e;
+        run_nb[run] = nbands;
+        run_segs[run] = nsegs;
+    }
+    __syncthreads();
     if (tid == 0) {
         int spos = 0, segoff = 0, sbcount = 0;
         for (int run = 0; run < 2 * El; ++run) {
-            const bool remote = run < El;
-            const int e = remote ? eorder[run] : run - El;
             run_start[run] = spos;
-            run_exp[run] = e;
-            for (int q = remote ? 0 : R - 1; q < (remote ? R - 1 : R); ++q) {
-                const int r = q < R - 1 ? (q < self ? q : q + 1) : self;
-                const int g = e * R + r;
-                gsched[g] = spos;
-                spos += nb[g];
-                gsegoff[g] = segoff;
-                const int ns = num_segments(nb[g], p.mgb);
-                segoff += ns;
-                segs_per_rank[r] += ns;
-            }
-            run_nb[run] = spos - run_start[run];
+            spos += run_nb[run];
+            const int nsegs = run_segs[run];
+            run_segs[run] = segoff;             // now the run's first segment
+            segoff += nsegs;
             run_sb0[run] = sbcount;
             // super-bands are made of whole band pairs (the GEMM works on two bands at a time)
             const int pairs = (run_nb[run] + 1) / 2, pairs_per_sb = max(1, p.group_bands / 2);
@@ -195,6 +228,17 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
         s_nsb = sbcount;
         p.meta[META_SEGS] = segoff;
         p.meta[META_SUPERBANDS] = sbcount;
+    }
+    __syncthreads();
+    for (int run = tid; run < 2 * El; run += blockDim.x) {
+        const bool remote = run < El;
+        const int e = run_exp[run];
+        for (int q = remote ? 0 : R - 1; q < (remote ? R - 1 : R); ++q) {
+            const int r = q < R - 1 ? (q < self ? q : q + 1) : self;
+            const int g = e * R + r;
+            gsched[g] += run_start[run];
+            gsegoff[g] += run_segs[run];
+        }
     }
     __syncthreads();
 

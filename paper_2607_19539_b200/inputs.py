@@ -74,6 +74,8 @@ SHAPES: Dict[str, MoEShape] = {
     "paper_op_e16": MoEShape("paper_op_e16", R=4, T=8192, Eg=64, k=2, El=16, d=2048, F=0, N_out=8192),
     "paper_op_e16_zipf": MoEShape("paper_op_e16_zipf", R=4, T=8192, Eg=64, k=2, El=16, d=2048, F=0, N_out=8192,
                                   router="zipf"),
+    # many (expert, rank) groups with few rows each: 512 groups, almost every band partial
+    "many_groups": MoEShape("many_groups", R=16, T=300, Eg=64, k=4, El=32, d=256, F=128, self_rank=5, seed=4),
     "single_small": MoEShape("single_small", R=3, T=600, Eg=6, k=2, El=2, d=192, F=0, N_out=512, self_rank=2, seed=2),
     # mid-size shapes for parity tests (several bands per group, ragged tails)
     "small": MoEShape("small", R=3, T=700, Eg=6, k=2, El=3, d=512, F=384, self_rank=1),

@@ -30,7 +30,7 @@ def _run_case(shape, mode, csm, shuffle=None, mgb=1, group_bands=0, inp=None, ds
     return inp, dsp, ctx, prob
 
 
-SMALL = ["tiny", "tiny_zipf", "small", "small_zipf_rot", "single_small"]
+SMALL = ["tiny", "tiny_zipf", "small", "small_zipf_rot", "single_small", "many_groups"]
 
 
 @pytest.mark.parametrize("name", SMALL)

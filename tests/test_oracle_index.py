@@ -78,7 +78,7 @@ def test_paper_sizes():
 
 
 @pytest.mark.parametrize("name,shuffle", [("tiny", None), ("tiny_zipf", 5), ("small", None), ("small", 11),
-                                          ("small_zipf_rot", 2)])
+                                          ("small_zipf_rot", 2), ("many_groups", 1)])
 def test_round_trip_permutation(name, shuffle):
     shape = I.SHAPES[name]
     inp, dsp, plan = _plan_for(shape, shuffle_seed=shuffle)
