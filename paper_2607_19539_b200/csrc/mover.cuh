@@ -101,8 +101,9 @@ __global__ void __launch_bounds__(256) scatter_kernel(const Params p)
     }
 }
 
-// One CTA works on one token at a time (grid-stride over tokens); thread v handles 8 consecutive features.
-// The next token's list is fetched while the current token's rows are in flight.
+// A group of threads (256 for wide rows, down to 32 for narrow ones, so that every thread has two 16-byte
+// vectors of work) handles one token at a time, grid-stride over tokens; thread v handles 8 consecutive
+// features.  The next token's list is fetched while the current token's rows are in flight.
 __global__ void __launch_bounds__(256) combine_kernel(const Params p)
 {
     const int ntok = p.R * p.T;
@@ -118,50 +119,64 @@ __global__ void __launch_bounds__(256) combine_kernel(const Params p)
             gate[j] = use ? __ldg(p.tok_gate + (size_t)tok * p.kmax + j) : 0.f;
         }
     };
-    fetch(blockIdx.x);
-    for (int tok = blockIdx.x; tok < ntok; tok += gridDim.x) {
+    int tpt = 256;                                  // threads per token: power of two, about nv / 2
+    while (tpt > 32 && tpt > nv / 2) tpt >>= 1;
+    const int sub = threadIdx.x / tpt, lt = threadIdx.x % tpt, per_block = blockDim.x / tpt;
+    const int tok_stride = gridDim.x * per_block;
+    fetch(blockIdx.x * per_block + sub);
+    for (int tok = blockIdx.x * per_block + sub; tok < ntok; tok += tok_stride) {
         const uint16_t *region = p.ret + (size_t)(tok / p.T) * p.ret_rows_per_rank * p.dout;
         uint4 *o = reinterpret_cast<uint4 *>(p.out + (size_t)tok * p.dout);
         int cs[KFAST];
         float cg[KFAST];
 #pragma unroll
         for (int j = 0; j < KFAST; ++j) { cs[j] = slot[j]; cg[j] = gate[j]; }
-        fetch(tok + gridDim.x);
-        for (int v = threadIdx.x; v < nv; v += blockDim.x) {
-            uint4 row[KFAST];
-#pragma unroll
-            for (int j = 0; j < KFAST; ++j)
-                row[j] = cs[j] > 0 ? __ldcs(reinterpret_cast<const uint4 *>(region + (size_t)(cs[j] - 1) * p.dout) + v)
-                                   : make_uint4(0, 0, 0, 0);
-            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            auto add = [&](const uint4 &q, float g) {
-                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    acc[2 * i] += g * __uint_as_float(w[i] << 16);
-                    acc[2 * i + 1] += g * __uint_as_float(w[i] & 0xffff0000u);
-                }
-            };
-            // ascending local expert; the list is dense, so the first empty entry (0) ends it
-            bool open = true;
+        fetch(tok + tok_stride);
+        // two 16-byte vectors per thread and iteration: all of their row loads are issued before any arithmetic
+        for (int v0 = lt; v0 < nv; v0 += 2 * tpt) {
+            const int v1 = v0 + tpt;
+            const bool has1 = v1 < nv;
+            uint4 row[2][KFAST];
 #pragma unroll
             for (int j = 0; j < KFAST; ++j) {
-                open = open && cs[j] > 0;
-                if (open) add(row[j], cg[j]);
+                const uint4 *src = reinterpret_cast<const uint4 *>(region + (size_t)(cs[j] > 0 ? cs[j] - 1 : 0) * p.dout);
+                row[0][j] = cs[j] > 0 ? __ldcs(src + v0) : make_uint4(0, 0, 0, 0);
+                row[1][j] = (cs[j] > 0 && has1) ? __ldcs(src + v1) : make_uint4(0, 0, 0, 0);
             }
-            if (open) {
-                for (int j = KFAST; j < p.kmax; ++j) {        // tokens with more than two local rows
-                    const int s = p.tok_slot[(size_t)tok * p.kmax + j];
-                    if (s <= 0) break;
-                    add(__ldcs(reinterpret_cast<const uint4 *>(region + (size_t)(s - 1) * p.dout) + v),
-                        p.tok_gate[(size_t)tok * p.kmax + j]);
-                }
-            }
-            uint32_t w[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(acc[2 * i + 1]), "f"(acc[2 * i]));
-            o[v] = make_uint4(w[0], w[1], w[2], w[3]);
+            for (int u = 0; u < 2; ++u) {
+                const int v = u == 0 ? v0 : v1;
+                if (u == 1 && !has1) break;
+                float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                auto add = [&](const uint4 &q, float g) {
+                    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        acc[2 * i] += g * __uint_as_float(w[i] << 16);
+                        acc[2 * i + 1] += g * __uint_as_float(w[i] & 0xffff0000u);
+                    }
+                };
+                // ascending local expert; the list is dense, so the first empty entry (0) ends it
+                bool open = true;
+#pragma unroll
+                for (int j = 0; j < KFAST; ++j) {
+                    open = open && cs[j] > 0;
+                    if (open) add(row[u][j], cg[j]);
+                }
+                if (open) {
+                    for (int j = KFAST; j < p.kmax; ++j) {        // tokens with more than two local rows
+                        const int s = p.tok_slot[(size_t)tok * p.kmax + j];
+                        if (s <= 0) break;
+                        add(__ldcs(reinterpret_cast<const uint4 *>(region + (size_t)(s - 1) * p.dout) + v),
+                            p.tok_gate[(size_t)tok * p.kmax + j]);
+                    }
+                }
+                uint32_t w[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(acc[2 * i + 1]), "f"(acc[2 * i]));
+                __stcs(o + v, make_uint4(w[0], w[1], w[2], w[3]));
+            }
         }
     }
 }
