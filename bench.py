@@ -272,8 +272,11 @@ def main():
     secs = D.max_over_ranks(total_ms / 1e3, dev)
     value = step_flops * args.steps * world / secs / 1e12
 
-    # the GEMM kernel's own duration, measured per launch by the library with CUDA events on the stream it
-    # is launched on; averaged over a few extra steps
+    # The GEMM kernel's own duration inside the timed region: the library brackets every launch with CUDA events
+    # on the stream it launches the kernel on and keeps the last 64 pairs, so the average over the timed steps
+    # needs no synchronisation between them.
+    prod_in_region_ms, n_hist = ctx.moe_ovl_get_gemm_time(args.steps)     # exactly the timed steps (up to 64)
+    # phase breakdown of single calls (each followed by a synchronisation)
     prod_ms, mover_ms, er_ms, prep_ms, comb_ms, ovl_ratio, assist = [], [], [], [], [], [], []
     for _ in range(min(args.steps, 10)):
         Hn.run(ctx, prob, mode=head_mode, consumer_sm_count=args.consumer_sms)
@@ -281,13 +284,14 @@ def main():
         prod_ms.append(r.ms_producer); mover_ms.append(r.ms_mover); er_ms.append(r.ms_expert_return)
         prep_ms.append(r.ms_prep); comb_ms.append(r.ms_combine)
         ovl_ratio.append(r.overlap_ratio); assist.append(r.segments_by_gemm_ctas)
-    prod = statistics.mean(prod_ms)
+    prod = prod_in_region_ms
     peak_tf = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
     achieved = step_flops / (prod / 1e3) / 1e12
     roofline = {"bound": "tensor", "kernel": "producer_kernel", "achieved": achieved, "peak": peak_tf,
                 "unit": "TFLOP/s", "frac": achieved / peak_tf, "peak_kind": f"bf16 burst, {peaks_kind}",
                 "frac_of_sustained": achieved / float(peaks.get("bf16_tflops_sustained", peak_tf)),
-                "launch_ms": prod, "flops_per_launch": step_flops,
+                "launch_ms": prod, "launches_averaged": n_hist, "launch_ms_single_call": statistics.mean(prod_ms),
+                "flops_per_launch": step_flops,
                 "traffic": NCU_PRODUCER_TRAFFIC_BYTES.get(shape.name)}
 
     # ---- comparison against the in-build non-overlap baseline.  The GPU is power-limited under this load, so a

@@ -128,6 +128,8 @@ typedef struct {
     void *stream;
 } moe_ovl_host_args;
 
+#define MOE_OVL_TIMING_HISTORY 64
+
 /* Sizes of the plan of the last call, and where the time went (milliseconds). */
 typedef struct {
     int32_t padded_rows;      /* P, multiple of 128 */
@@ -213,6 +215,10 @@ int moe_ovl_query_status(moe_ovl_ctx *ctx, int32_t *code, int64_t *detail);
  * `bytes` bytes at `offset` of an internal bf16 buffer (MOE_OVL_BUF_*) to HOST memory. */
 int moe_ovl_get_report(moe_ovl_ctx *ctx, moe_ovl_report *report);
 int moe_ovl_get_plan(moe_ovl_ctx *ctx, const moe_ovl_plan_view *view);
+/* Mean duration (ms) of the GEMM kernel over the last `last_n` calls (at most MOE_OVL_TIMING_HISTORY): every call
+ * brackets the kernel with CUDA events on the stream it is launched on and the context keeps the most recent
+ * pairs, so a run of back-to-back calls can be timed without synchronising between them.  Waits for the last call. */
+int moe_ovl_get_gemm_time(moe_ovl_ctx *ctx, int32_t last_n, float *avg_ms, int32_t *n_used);
 /* SM (%smid) every GEMM CTA and every consumer CTA of the last call ran on; HOST arrays of
  * producer_ctas and consumer_ctas entries (moe_ovl_report).  The two kernels must not share an SM. */
 int moe_ovl_get_sm_map(moe_ovl_ctx *ctx, int32_t *producer_smid, int32_t *consumer_smid);

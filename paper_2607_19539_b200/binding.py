@@ -26,7 +26,7 @@ TB_M, TB_N, H_TILE = 128, 256, 128
 EXPORTS = [
     "moe_ovl_workspace_bytes", "moe_ovl_limits", "moe_ovl_create", "moe_ovl_expert_return",
     "moe_ovl_expert_return_host", "moe_ovl_host_join", "moe_ovl_query_status", "moe_ovl_get_report", "moe_ovl_get_plan",
-    "moe_ovl_get_sm_map", "moe_ovl_read_buffer", "moe_ovl_destroy", "moe_ovl_strerror", "moe_ovl_last_cuda_error",
+    "moe_ovl_get_sm_map", "moe_ovl_get_gemm_time", "moe_ovl_read_buffer", "moe_ovl_destroy", "moe_ovl_strerror", "moe_ovl_last_cuda_error",
     "moe_ovl_return_slots_static",
 ]
 
@@ -107,6 +107,7 @@ def load(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moe_ovl_query_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
     lib.moe_ovl_get_report.argtypes = [C.c_void_p, C.POINTER(Report)]
     lib.moe_ovl_get_plan.argtypes = [C.c_void_p, C.POINTER(PlanView)]
+    lib.moe_ovl_get_gemm_time.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
     lib.moe_ovl_get_sm_map.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     lib.moe_ovl_read_buffer.argtypes = [C.c_void_p, C.c_int32, C.c_size_t, C.c_size_t, C.c_void_p]
     lib.moe_ovl_destroy.argtypes = [C.c_void_p]
@@ -271,6 +272,13 @@ class MoeOvl:
         arrs["tok_slot"] = arrs["tok_slot"].reshape(-1, self.kmax)
         arrs["tok_gate"] = arrs["tok_gate"].reshape(-1, self.kmax)
         return arrs
+
+    def moe_ovl_get_gemm_time(self, last_n: int):
+        """(mean GEMM kernel duration in ms over the last calls, number of calls averaged)."""
+        ms, n = C.c_float(0), C.c_int32(0)
+        self._check(self.lib.moe_ovl_get_gemm_time(self.ctx, int(last_n), C.byref(ms), C.byref(n)),
+                    "moe_ovl_get_gemm_time")
+        return float(ms.value), int(n.value)
 
     def moe_ovl_get_sm_map(self):
         rep = self.moe_ovl_get_report()

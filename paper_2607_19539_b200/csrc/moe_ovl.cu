@@ -149,6 +149,10 @@ struct moe_ovl_ctx {
     cudaEvent_t ev_fork, ev_prod_done, ev_cons_done;
     // timing: call start, after prep, GEMM start/end, mover start/end, call end
     cudaEvent_t t_begin, t_prep, t_p0, t_p1, t_m0, t_m1, t_end;
+    // GEMM start/end of the last HISTORY calls, so that a caller can average the kernel's duration over a run
+    // of back-to-back calls without synchronising between them
+    cudaEvent_t h_p0[MOE_OVL_TIMING_HISTORY], h_p1[MOE_OVL_TIMING_HISTORY];
+    unsigned long long calls;
     cudaStream_t last_stream;
     bool ran;
     int last_mode, last_prod_ctas, last_cons_ctas, last_launches, last_rows;
@@ -310,6 +314,10 @@ int moe_ovl_create(moe_ovl_ctx **out, const moe_ovl_config *cfg, void *workspace
     for (auto e : plain) CREATE_CHECK(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
     cudaEvent_t *timed[] = {&ctx->t_begin, &ctx->t_prep, &ctx->t_p0, &ctx->t_p1, &ctx->t_m0, &ctx->t_m1, &ctx->t_end};
     for (auto e : timed) CREATE_CHECK(cudaEventCreate(e));
+    for (int i = 0; i < MOE_OVL_TIMING_HISTORY; ++i) {
+        CREATE_CHECK(cudaEventCreate(&ctx->h_p0[i]));
+        CREATE_CHECK(cudaEventCreate(&ctx->h_p1[i]));
+    }
     CREATE_CHECK(cudaFuncSetAttribute(producer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PROD_SMEM_BYTES));
     CREATE_CHECK(cudaFuncSetAttribute(consumer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       CONSUMER_SMEM_BYTES));
@@ -352,6 +360,10 @@ int moe_ovl_destroy(moe_ovl_ctx *ctx)
                          ctx->t_p1, ctx->t_m0, ctx->t_m1, ctx->t_end};
     for (auto e : evs)
         if (e) cudaEventDestroy(e);
+    for (int i = 0; i < MOE_OVL_TIMING_HISTORY; ++i) {
+        if (ctx->h_p0[i]) cudaEventDestroy(ctx->h_p0[i]);
+        if (ctx->h_p1[i]) cudaEventDestroy(ctx->h_p1[i]);
+    }
     delete ctx;
     return MOE_OVL_OK;
 }
@@ -423,6 +435,7 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     sc.sb_g1off = at<int>(ctx, L.sb[3]); sc.sb_g2off = at<int>(ctx, L.sb[4]); sc.sb_g1end = at<int>(ctx, L.sb[5]);
 
     int launches = 0;
+    const int hist = (int)(ctx->calls % MOE_OVL_TIMING_HISTORY);
     CU_CHECK(ctx, cudaEventRecord(ctx->t_begin, st));
     // ---- plan + gather (8a-1 .. 8a-3): integer kernels on the caller's stream
     CU_CHECK(ctx, cudaMemsetAsync(ctx->ws + L.zero_begin, 0, L.zero_end - L.zero_begin, st));
@@ -448,17 +461,21 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
         CU_CHECK(ctx, cudaEventRecord(ctx->t_m1, ctx->s_cons));
         CU_CHECK(ctx, cudaEventRecord(ctx->ev_cons_done, ctx->s_cons));
         CU_CHECK(ctx, cudaEventRecord(ctx->t_p0, ctx->s_prod));
+        CU_CHECK(ctx, cudaEventRecord(ctx->h_p0[hist], ctx->s_prod));
         producer_kernel<<<prod_ctas, PROD_THREADS, PROD_SMEM_BYTES, ctx->s_prod>>>(
             maps, p, (c.flags & MOE_OVL_FLAG_TEST_NO_FLAGS) ? 0 : 1);
         CU_CHECK(ctx, cudaEventRecord(ctx->t_p1, ctx->s_prod));
+        CU_CHECK(ctx, cudaEventRecord(ctx->h_p1[hist], ctx->s_prod));
         CU_CHECK(ctx, cudaEventRecord(ctx->ev_prod_done, ctx->s_prod));
         CU_CHECK(ctx, cudaStreamWaitEvent(st, ctx->ev_cons_done, 0));
         CU_CHECK(ctx, cudaStreamWaitEvent(st, ctx->ev_prod_done, 0));
     } else {
         // ---- comparison baseline: the GEMM runs to completion, then a separate scatter kernel
         CU_CHECK(ctx, cudaEventRecord(ctx->t_p0, st));
+        CU_CHECK(ctx, cudaEventRecord(ctx->h_p0[hist], st));
         producer_kernel<<<prod_ctas, PROD_THREADS, PROD_SMEM_BYTES, st>>>(maps, p, 0);
         CU_CHECK(ctx, cudaEventRecord(ctx->t_p1, st));
+        CU_CHECK(ctx, cudaEventRecord(ctx->h_p1[hist], st));
         CU_CHECK(ctx, cudaEventRecord(ctx->t_m0, st));
         scatter_kernel<<<ctx->scatter_blocks_per_sm * ctx->num_sms, 256, 0, st>>>(p);
         CU_CHECK(ctx, cudaEventRecord(ctx->t_m1, st));
@@ -471,6 +488,7 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
 
     ctx->last_stream = st;
     ctx->ran = true;
+    ++ctx->calls;
     ctx->last_mode = a->mode;
     ctx->last_prod_ctas = prod_ctas;
     ctx->last_cons_ctas = cons_ctas;
@@ -629,6 +647,25 @@ int moe_ovl_get_plan(moe_ovl_ctx *ctx, const moe_ovl_plan_view *v)
         if (e.dst && e.bytes) CU_CHECK(ctx, cudaMemcpy(e.dst, ctx->ws + e.off, e.bytes, cudaMemcpyDeviceToHost));
     if (v->tok_slot)                           // stored as slot + 1 with 0 = none; reported as slot with -1 = none
         for (size_t i = 0; i < ntokk; ++i) v->tok_slot[i] -= 1;
+    return MOE_OVL_OK;
+}
+
+int moe_ovl_get_gemm_time(moe_ovl_ctx *ctx, int32_t last_n, float *avg_ms, int32_t *n_used)
+{
+    if (!ctx || !avg_ms || last_n < 1) return MOE_OVL_ERR_INVALID_ARG;
+    int rc = sync_last(ctx);
+    if (rc != MOE_OVL_OK) return rc;
+    const int have = (int)std::min<unsigned long long>(ctx->calls, MOE_OVL_TIMING_HISTORY);
+    const int n = std::min<int>(last_n, have);
+    double sum = 0;
+    for (int k = 1; k <= n; ++k) {
+        const int i = (int)((ctx->calls - k) % MOE_OVL_TIMING_HISTORY);
+        float ms = 0.f;
+        CU_CHECK(ctx, cudaEventElapsedTime(&ms, ctx->h_p0[i], ctx->h_p1[i]));
+        sum += ms;
+    }
+    *avg_ms = n ? (float)(sum / n) : 0.f;
+    if (n_used) *n_used = n;
     return MOE_OVL_OK;
 }
 
