@@ -29,7 +29,7 @@ constexpr int ERR_BAD_ROUTING = -6;
 // wait sites reported in the high bits of the status detail
 enum : long long {
     SITE_TMA_EMPTY = 1, SITE_TMA_HCOUNT, SITE_MMA_FULL, SITE_MMA_TEMPTY, SITE_EPI_TFULL, SITE_CONS_FLAG,
-    SITE_MMA_DRAIN, SITE_TMA_DRAIN, SITE_CLAIM, SITE_SCHED_GO,
+    SITE_MMA_DRAIN, SITE_TMA_DRAIN, SITE_CLAIM, SITE_SCHED_GO, SITE_TMA_XREADY,
     SITE_ROW_RANGE = 16, SITE_ROW_DUP, SITE_COUNT_SUM, SITE_TOK_OVERFLOW
 };
 
@@ -78,6 +78,9 @@ struct Params {
     int *assist_segs;     // segments moved by GEMM CTAs
     int *next_seg;        // segments claimed so far (consumer CTAs, and GEMM CTAs once they are out of tiles)
     int *next_item;       // schedule items claimed so far (GEMM CTA pairs take them in order)
+    int *next_gather;     // gather units claimed so far (GEMM CTAs' gather warps)
+    int *row_at;          // [P] input row held by every aligned position (valid positions only)
+    unsigned *xready;     // [max_bands] rows of the band gathered into Xa (128 = ready)
     unsigned *hcount;     // [max_bands] first-GEMM tiles finished per band
     unsigned *flags;      // [max_bands*n2] epoch of the call that finished the tile
     int *meta;            // [META_COUNT]

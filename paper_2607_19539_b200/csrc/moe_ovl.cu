@@ -31,7 +31,7 @@ struct Layout {
     size_t Xa, H, Y;
     size_t zero_begin, bitmap, hcount, status, next_item, stamps, tok_slot, zero_end;   // cleared at the start of every call
     size_t smid;
-    size_t wordpfx, group_rows, group_start, group_slot, pos, slot;
+    size_t wordpfx, group_rows, group_start, group_slot, pos, slot, row_at, xready;
     size_t band_expert, band_dest, band_valid, band_slot0, sched_band, items, segs, seg_slot0;
     size_t tok_gate, flags, meta;
     size_t sb[6];
@@ -94,7 +94,7 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->bitmap = take((size_t)G * L->words * 4);
     L->hcount = take((size_t)L->max_bands * 4);
     L->status = take(ST_COUNT * 4);
-    L->next_item = take(16);                 // next_item, plan_ticket, next_seg, assist_segs
+    L->next_item = take(32);                 // next_item, plan_ticket, next_seg, assist_segs, next_gather
     L->stamps = take(STAMP_COUNT * 8);
     L->tok_slot = take(ntok * L->kmax * 4);
     L->zero_end = off;
@@ -105,6 +105,8 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->group_slot = take((size_t)G * 4);
     L->pos = take((size_t)std::max(c->max_rows, 1) * 4);
     L->slot = take((size_t)std::max(c->max_rows, 1) * 4);
+    L->row_at = take(P * 4);
+    L->xready = take((size_t)L->max_bands * 4);
     L->band_expert = take((size_t)L->max_bands * 4);
     L->band_dest = take((size_t)L->max_bands * 4);
     L->band_valid = take((size_t)L->max_bands * 4);
@@ -218,6 +220,9 @@ Params make_params(moe_ovl_ctx *ctx)
     p.plan_ticket = at<int>(ctx, L.next_item) + 1;
     p.next_seg = at<int>(ctx, L.next_item) + 2;
     p.assist_segs = at<int>(ctx, L.next_item) + 3;
+    p.next_gather = at<int>(ctx, L.next_item) + 4;
+    p.row_at = at<int>(ctx, L.row_at);
+    p.xready = at<unsigned>(ctx, L.xready);
     p.stamps = at<unsigned long long>(ctx, L.stamps);
     p.smid_prod = at<int>(ctx, L.smid);
     p.smid_cons = at<int>(ctx, L.smid) + 1024;
@@ -442,10 +447,7 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     plan_mark_build_kernel<<<std::max(1, (p.M + PLAN_THREADS - 1) / PLAN_THREADS), PLAN_THREADS, 0, st>>>(p, sc);
     ++launches;
     if (p.M > 0) {
-        // one resident wave of row blocks (3 per SM) minus the blocks that zero the padding rows
-        const int pad_blocks = std::min(L.max_bands, ctx->num_sms / 2);
-        const int row_blocks = std::max(1, std::min((p.M + 7) / 8, 3 * ctx->num_sms - pad_blocks));
-        plan_rows_kernel<<<row_blocks + pad_blocks, 256, 0, st>>>(p, row_blocks);
+        plan_rows_kernel<<<(p.M + 255) / 256, 256, 0, st>>>(p);
         ++launches;
     }
     CU_CHECK(ctx, cudaGetLastError());

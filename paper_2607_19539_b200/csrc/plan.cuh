@@ -253,6 +253,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
             p.band_slot0[band] = gslot[g] + b * TB_M;
             p.sched_band[gsched[g] + b] = band;
             p.hcount[band] = 0;
+            p.xready[band] = 0;
         }
         const int ns = num_segments(nb[g], p.mgb);
         for (int q = lane; q < ns; q += 32) {
@@ -332,89 +333,37 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     }
 }
 
-// ---- step 3: per row: aligned position, return slot, per-token list entry, copy into the layout;
-//      the blocks after the row blocks zero the padding rows of every band (Section 3.2.1: zero-filled rows)
-struct RowMeta {
-    int pos, slot, j, tok;    // pos < 0: row skipped (bad metadata)
-};
-
-__device__ __forceinline__ RowMeta resolve_row(const Params &p, const int *pre, int i, int lane)
+// ---- step 3: per row: aligned position, return slot, entry in its token's list, and the inverse map
+//      (aligned position -> input row) that the GEMM kernel's gather warps follow.  One thread per row; the
+//      rows themselves are moved by the GEMM kernel.
+__global__ void __launch_bounds__(256) plan_rows_kernel(Params p)
 {
-    RowMeta m{-1, -1, 0, 0};
-    if (i >= p.M || i >= pre[p.El]) return m;
+    __shared__ int pre[PLAN_MAX_EXPERTS + 1];
+    load_expert_prefix(p, pre);
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= p.M || i >= pre[p.El]) return;
     const int e = expert_of_row(pre, p.El, i);
     const int r = p.src_rank[i], t = p.src_token[i];
-    if (r < 0 || r >= p.R || t < 0 || t >= p.T) return m;
+    if (r < 0 || r >= p.R || t < 0 || t >= p.T) return;
     const int g = e * p.R + r;
     const size_t w = (size_t)g * p.words + (t >> 5);
     const int q = p.wordpfx[w] + __popc(p.bitmap[w] & ((1u << (t & 31)) - 1u));
-    m.pos = p.group_start[g] + q;
-    m.slot = p.group_slot[g] + q;
-    m.tok = r * p.T + t;
+    const int pos = p.group_start[g] + q;
+    const int slot = p.group_slot[g] + q;
     // entry of this row in its token's list: number of lower-indexed local experts the token also selected
     int j = 0;
-    for (int o = lane; o < e; o += 32)
+    for (int o = 0; o < e; ++o)
         j += (p.bitmap[(size_t)(o * p.R + r) * p.words + (t >> 5)] >> (t & 31)) & 1u;
-    m.j = __reduce_add_sync(0xffffffffu, j);
-    return m;
-}
-
-constexpr int ROWS_CHUNK = 8;       // 16-byte vectors per lane in flight before the row's position is needed
-__global__ void __launch_bounds__(256, 3) plan_rows_kernel(Params p, int row_blocks)
-{
-    __shared__ int pre[PLAN_MAX_EXPERTS + 1];
-    const int lane = threadIdx.x & 31;
-    const int nv = p.d / 8;
-    if ((int)blockIdx.x >= row_blocks) {
-        const int nbands = p.meta[META_BANDS];
-        for (int band = blockIdx.x - row_blocks; band < nbands; band += gridDim.x - row_blocks) {
-            const int valid = p.band_valid[band];
-            uint4 *dst = reinterpret_cast<uint4 *>(p.Xa + ((size_t)band * TB_M + valid) * p.d);
-            const size_t n = (size_t)(TB_M - valid) * nv;
-            for (size_t v = threadIdx.x; v < n; v += blockDim.x) dst[v] = make_uint4(0, 0, 0, 0);
-        }
-        return;
-    }
-    load_expert_prefix(p, pre);
-    // warps walk the rows with a grid stride; the position of the NEXT row is resolved while the loads of the
-    // current row are in flight, so the chain of dependent metadata loads is off the critical path
-    const int nwarps = row_blocks * (blockDim.x >> 5);
-    int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    RowMeta cur = resolve_row(p, pre, i, lane);
-    for (; i < p.M; i += nwarps) {
-        const uint4 *src = reinterpret_cast<const uint4 *>(p.x + (size_t)i * p.d);
-        uint4 buf[ROWS_CHUNK];
-#pragma unroll
-        for (int k = 0; k < ROWS_CHUNK; ++k)
-            if (lane + 32 * k < nv) buf[k] = __ldcs(src + lane + 32 * k);
-        const RowMeta nxt = resolve_row(p, pre, i + nwarps, lane);
-        if (cur.pos >= 0) {
-            uint4 *dst = reinterpret_cast<uint4 *>(p.Xa + (size_t)cur.pos * p.d);
-#pragma unroll
-            for (int k = 0; k < ROWS_CHUNK; ++k)
-                if (lane + 32 * k < nv) dst[lane + 32 * k] = buf[k];
-            for (int v0 = 32 * ROWS_CHUNK; v0 < nv; v0 += 32 * ROWS_CHUNK) {
-#pragma unroll
-                for (int k = 0; k < ROWS_CHUNK; ++k)
-                    if (v0 + lane + 32 * k < nv) buf[k] = __ldcs(src + v0 + lane + 32 * k);
-#pragma unroll
-                for (int k = 0; k < ROWS_CHUNK; ++k)
-                    if (v0 + lane + 32 * k < nv) dst[v0 + lane + 32 * k] = buf[k];
-            }
-            if (lane == 0) {
-                p.pos[i] = cur.pos;
-                p.slot[i] = cur.slot;
-                if (p.slot_out) p.slot_out[i] = cur.slot;
-                if (cur.j < p.kmax) {
-                    const size_t at = (size_t)cur.tok * p.kmax + cur.j;
-                    p.tok_slot[at] = cur.slot + 1;            // 0 (the cleared state) means "no row"
-                    p.tok_gate[at] = p.gate[i];
-                } else {
-                    report_error(p.status, ERR_BAD_ROUTING, SITE_TOK_OVERFLOW, i);
-                }
-            }
-        }
-        cur = nxt;
+    p.pos[i] = pos;
+    p.row_at[pos] = i;
+    p.slot[i] = slot;
+    if (p.slot_out) p.slot_out[i] = slot;
+    if (j < p.kmax) {
+        const size_t at = ((size_t)r * p.T + t) * p.kmax + j;
+        p.tok_slot[at] = slot + 1;            // 0 (the cleared state) means "no row"
+        p.tok_gate[at] = p.gate[i];
+    } else {
+        report_error(p.status, ERR_BAD_ROUTING, SITE_TOK_OVERFLOW, i);
     }
 }
 

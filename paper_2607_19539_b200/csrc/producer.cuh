@@ -12,6 +12,10 @@
 //   warp 1     in the leader CTA one thread issues tcgen05.mma (bf16 x bf16 -> fp32, M=256
 //              N=256 K=16); accumulators in tensor memory, double buffered (2 x 256 columns)
 //   warps 2-5  epilogue: tcgen05.ld -> fp32 math -> bf16 -> global, then publish
+//   warps 7-10 gather: move the dispatched rows into the aligned layout Xa (Section 3.2.1) band by band in
+//              schedule order while the tensor cores work, and count finished rows per band; the TMA warp
+//              waits for a band's count before its first load.  The layout pass therefore costs no time
+//              of its own except for the first few bands.
 //   warp 6     scheduler (leader CTA): claims the next schedule item with an atomic counter, one
 //              item ahead of the TMA warp, and hands it to every role of both CTAs through a
 //              small ring in shared memory.  Items are claimed in schedule order, so the
@@ -38,7 +42,9 @@ constexpr int PROD_STAGES = 6;
 constexpr int PROD_A_BYTES = TB_M * TB_K * 2;          // 16 KiB: this CTA's 128 rows of A
 constexpr int PROD_B_BYTES = (TB_N / 2) * TB_K * 2;    // 16 KiB: this CTA's half of the B tile
 constexpr int PROD_STAGE_BYTES = PROD_A_BYTES + PROD_B_BYTES;
-constexpr int PROD_THREADS = 224;                      // TMA, MMA, 4 epilogue warps, scheduler
+constexpr int PROD_GATHER_WARPS = 4;
+constexpr int PROD_THREADS = 224 + 32 * PROD_GATHER_WARPS;   // TMA, MMA, 4 epilogue warps, scheduler, gather warps
+constexpr int GATHER_ROWS = 8;                         // rows per gather unit
 constexpr int PROD_RING = 16;                          // claimed-item ring; roles are never more than 5 items apart
 constexpr int PROD_TMEM_COLS = 512;
 constexpr int PROD_SMEM_BYTES = PROD_STAGES * PROD_STAGE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers, ring*/;
@@ -322,6 +328,10 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     // rank 0 holds the gate-projection rows of the tile, rank 1 the matching up-projection rows
                     b_row = e * 2 * p.F + tile * H_TILE + (int)rank * p.F;
                     ksteps = p.d / TB_K;
+                    // all 128 rows of the band (padding included) must have been gathered into Xa
+                    ok = wait_global(&p.xready[band], (unsigned)TB_M, true, p, SITE_TMA_XREADY, band);
+                    if (!ok) break;
+                    asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
                 } else {
                     // single-projection experts: the output GEMM reads the aligned input itself
                     amap = p.single ? &maps.xa : &maps.h; bmap = &maps.w2;
@@ -330,9 +340,11 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     if (p.n1 > 0) {
                         // every first-GEMM tile of this band must have landed in H
                         ok = wait_global(&p.hcount[band], (unsigned)p.n1, true, p, SITE_TMA_HCOUNT, band);
-                        if (!ok) break;
-                        asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
+                    } else {
+                        ok = wait_global(&p.xready[band], (unsigned)TB_M, true, p, SITE_TMA_XREADY, band);
                     }
+                    if (!ok) break;
+                    asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
                 }
                 const int a_row = band * TB_M;
                 for (int ks = 0; ks < ksteps; ++ks) {
@@ -417,6 +429,50 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 mbar_arrive_cluster(peer_bar + 8 * slot);        // release at cluster scope: orders the store above
                 if (it >= n_items) break;
             }
+        }
+    } else if (warp >= 7) {
+        // ---------------- gather warps: Xa[band * 128 + r] = x[row_at[...]] for units of GATHER_ROWS rows, claimed in
+        // schedule order; padding rows are zero-filled (Section 3.2.1).  These warps never wait, so the row
+        // counts the TMA warps poll always make progress.
+        const int nbands = p.meta[META_BANDS];
+        const int units_per_band = TB_M / GATHER_ROWS;
+        const int nunits = nbands * units_per_band;
+        const int nv = p.d / 8;
+        int unit = 0;
+        if (lane == 0) unit = atomicAdd(p.next_gather, 1);
+        unit = __shfl_sync(0xffffffffu, unit, 0);
+        while (unit < nunits) {
+            int next = 0;
+            if (lane == 0) next = atomicAdd(p.next_gather, 1);      // claimed while this unit's rows are moving
+            const int band = p.sched_band[unit / units_per_band];
+            const int r0 = (unit % units_per_band) * GATHER_ROWS;
+            const int valid = p.band_valid[band];
+            // source row of each of the unit's rows (lanes 0..GATHER_ROWS-1), -1 for padding
+            int src_row = -1;
+            if (lane < GATHER_ROWS && r0 + lane < valid) src_row = p.row_at[(size_t)band * TB_M + r0 + lane];
+            // 64 lanes-worth of 16-byte vectors (1 KiB of every row) per pass: 16 loads in flight per lane
+            for (int v0 = 0; v0 < nv; v0 += 64) {
+                const int va = v0 + lane, vb = v0 + 32 + lane;
+                uint4 buf[2][GATHER_ROWS];
+#pragma unroll
+                for (int r = 0; r < GATHER_ROWS; ++r) {
+                    const int sr = __shfl_sync(0xffffffffu, src_row, r);
+                    const uint4 *src = reinterpret_cast<const uint4 *>(p.x + (size_t)(sr >= 0 ? sr : 0) * p.d);
+                    buf[0][r] = (sr >= 0 && va < nv) ? __ldcs(src + va) : make_uint4(0, 0, 0, 0);
+                    buf[1][r] = (sr >= 0 && vb < nv) ? __ldcs(src + vb) : make_uint4(0, 0, 0, 0);
+                }
+#pragma unroll
+                for (int r = 0; r < GATHER_ROWS; ++r) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(p.Xa + ((size_t)band * TB_M + r0 + r) * p.d);
+                    if (va < nv) dst[va] = buf[0][r];
+                    if (vb < nv) dst[vb] = buf[1][r];
+                }
+            }
+            __threadfence();
+            asm volatile("fence.proxy.async;" ::: "memory");      // Xa is read through TMA
+            __syncwarp();
+            if (lane == 0) red_release_add_u32(&p.xready[band], (unsigned)GATHER_ROWS);
+            unit = __shfl_sync(0xffffffffu, next, 0);
         }
     } else {
         // ---------------- epilogue: warps 2..5 own tensor-memory lanes 32*(warp % 4) .. +31
