@@ -277,13 +277,13 @@ def main():
     # needs no synchronisation between them.
     prod_in_region_ms, n_hist = ctx.moe_ovl_get_gemm_time(args.steps)     # exactly the timed steps (up to 64)
     # phase breakdown of single calls (each followed by a synchronisation)
-    prod_ms, mover_ms, er_ms, prep_ms, comb_ms, ovl_ratio, assist = [], [], [], [], [], [], []
+    prod_ms, mover_ms, er_ms, prep_ms, comb_ms, ovl_ratio, assist, copy_gbs = [], [], [], [], [], [], [], []
     for _ in range(min(args.steps, 10)):
         Hn.run(ctx, prob, mode=head_mode, consumer_sm_count=args.consumer_sms)
         r = ctx.moe_ovl_get_report()
         prod_ms.append(r.ms_producer); mover_ms.append(r.ms_mover); er_ms.append(r.ms_expert_return)
         prep_ms.append(r.ms_prep); comb_ms.append(r.ms_combine)
-        ovl_ratio.append(r.overlap_ratio); assist.append(r.segments_by_gemm_ctas)
+        ovl_ratio.append(r.overlap_ratio); assist.append(r.segments_by_gemm_ctas); copy_gbs.append(r.copy_gbs_per_cta)
     prod = prod_in_region_ms
     peak_tf = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
     achieved = step_flops / (prod / 1e3) / 1e12
@@ -379,6 +379,7 @@ def main():
             "producer_ctas": rep.producer_ctas, "consumer_ctas": rep.consumer_ctas,
             "overlap_ratio": statistics.mean(ovl_ratio) if args.mode == "overlap" else None,
             "segments_moved_by_gemm_ctas": statistics.mean(assist) if args.mode == "overlap" else None,
+            "return_copy_gbs_per_cta": statistics.mean(copy_gbs) if args.mode == "overlap" else None,
             "roofline": roofline, "non_overlap": non_overlap, "consumer_sm_sweep": sweep,
             "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": rep.kernel_launches * args.steps,
             "clocks": clocks, "paper_context": "paper reports ratios only (up to 2.74x MoE layer, 2.64x end to "

@@ -150,6 +150,8 @@ typedef struct {
     float us_first_flag;      /* first output tile flagged: the consumer's window opens */
     float us_gemm_done;       /* last output tile flagged */
     float us_return_done;     /* last segment landed in ret */
+    float copy_gbs_per_cta;   /* returned bytes / time the moving CTAs spent inside segment copies: the rate one CTA
+                                 sustains while the GEMM runs (GB/s, payload counted once) */
     float overlap_ratio;      /* share of the return window that lies before us_gemm_done:
                                  1 - max(0, us_return_done - us_gemm_done) / (us_return_done - us_first_flag);
                                  the share of the second all-to-all hidden behind expert compute (Section 4.2.2) */

@@ -61,7 +61,8 @@ class Report(C.Structure):
                 ("kernel_launches", C.c_int32), ("segments_by_gemm_ctas", C.c_int32), ("ms_total", C.c_float),
                 ("ms_prep", C.c_float), ("ms_expert_return", C.c_float), ("ms_producer", C.c_float),
                 ("ms_mover", C.c_float), ("ms_combine", C.c_float), ("us_first_flag", C.c_float),
-                ("us_gemm_done", C.c_float), ("us_return_done", C.c_float), ("overlap_ratio", C.c_float)]
+                ("us_gemm_done", C.c_float), ("us_return_done", C.c_float), ("copy_gbs_per_cta", C.c_float),
+                ("overlap_ratio", C.c_float)]
 
 
 class PlanView(C.Structure):
@@ -189,6 +190,7 @@ class ReportView:
     us_gemm_done: float = 0.0
     us_return_done: float = 0.0
     overlap_ratio: float = 0.0
+    copy_gbs_per_cta: float = 0.0
 
 
 class MoeOvl:
@@ -252,7 +254,7 @@ class MoeOvl:
         return ReportView(r.padded_rows, r.num_bands, r.num_items, r.num_segments, r.producer_ctas, r.consumer_ctas,
                           r.kernel_launches, r.ms_total, r.ms_prep, r.ms_expert_return, r.ms_producer, r.ms_mover,
                           r.ms_combine, r.segments_by_gemm_ctas, r.us_first_flag, r.us_gemm_done, r.us_return_done,
-                          r.overlap_ratio)
+                          r.overlap_ratio, r.copy_gbs_per_cta)
 
     def moe_ovl_get_plan(self) -> Dict[str, np.ndarray]:
         rep = self.moe_ovl_get_report()

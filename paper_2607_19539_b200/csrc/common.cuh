@@ -19,7 +19,8 @@ constexpr int KIND_G2 = 1;    // H . W2 -> Y, raises the consumer-visible flag
 // meta[] slots written by the plan kernel
 enum { META_P = 0, META_BANDS, META_ITEMS, META_SEGS, META_SUPERBANDS, META_COUNT = 8 };
 // stamps[] slots.  "first" stamps hold ~t so that the cleared state (0) is neutral under atomicMax.
-enum { STAMP_START_INV = 0, STAMP_FIRST_FLAG_INV, STAMP_LAST_FLAG, STAMP_LAST_SEG, STAMP_COUNT };
+enum { STAMP_START_INV = 0, STAMP_FIRST_FLAG_INV, STAMP_LAST_FLAG, STAMP_LAST_SEG, STAMP_COPY_NS, STAMP_COPY_BYTES,
+       STAMP_COUNT };
 // status[] slots
 enum { ST_CODE = 0, ST_ABORT = 1, ST_DETAIL_LO = 2, ST_DETAIL_HI = 3, ST_COUNT = 4 };
 

@@ -616,6 +616,7 @@ int moe_ovl_get_report(moe_ovl_ctx *ctx, moe_ovl_report *r)
             r->overlap_ratio = window > 0 ? (float)(1.0 - exposed / window) : 1.0f;
         }
         r->segments_by_gemm_ctas = misc[3];
+        if (st[STAMP_COPY_NS] > 0) r->copy_gbs_per_cta = (float)((double)st[STAMP_COPY_BYTES] / (double)st[STAMP_COPY_NS]);
     }
     return MOE_OVL_OK;
 }

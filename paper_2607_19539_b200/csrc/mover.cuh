@@ -62,12 +62,16 @@ __device__ __forceinline__ void move_segments(const Params &p, volatile int *s_s
         const int s = s_seg[0];
         if (s >= nseg || !s_seg[1]) return;
         const int4 seg = p.segs[s];
+        const unsigned long long t_copy = globaltimer_ns();
         const uint16_t *src = p.Y + (size_t)seg.x * TB_M * p.dout;
         uint16_t *dst = p.ret + ((size_t)seg.z * p.ret_rows_per_rank + p.seg_slot0[s]) * p.dout;
         copy_rows_16B(src, dst, (size_t)seg.w * p.dout / 8, threadIdx.x, blockDim.x);
         __syncthreads();
         if (threadIdx.x == 0) {
-            stamp_max(&p.stamps[STAMP_LAST_SEG], globaltimer_ns());
+            const unsigned long long now = globaltimer_ns();
+            stamp_max(&p.stamps[STAMP_LAST_SEG], now);
+            atomicAdd(&p.stamps[STAMP_COPY_NS], now - t_copy);                       // time one CTA spent copying
+            atomicAdd(&p.stamps[STAMP_COPY_BYTES], (unsigned long long)seg.w * p.dout * 2);
             if (gemm_cta) atomicAdd(p.assist_segs, 1);
         }
     }

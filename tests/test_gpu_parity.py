@@ -320,3 +320,42 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     want = [prob.out.view(torch.int16).cpu(), prob_b.out.view(torch.int16).cpu()]
     for i, ho in enumerate(houts):
         assert torch.equal(ho, want[i % 2]), i
+
+
+@pytest.mark.parametrize("seed", list(range(12)))
+def test_random_shapes_full_parity(seed):
+    """Seeded random small problems: rank and expert counts, top-k, widths, local rank, router, arrival order,
+    consumer budget, segment and super-band knobs all vary; every output is checked against the oracle."""
+    torch, B, Hn = _gpu()
+    rng = np.random.Generator(np.random.PCG64(1000 + seed))
+    El = int(rng.integers(1, 6))
+    groups = int(rng.integers(1, 4))
+    Eg = El * groups
+    k = int(rng.integers(1, min(Eg, 4) + 1))
+    R = int(rng.integers(1, 7))
+    single = seed % 4 == 3
+    shape = I.MoEShape(f"rnd{seed}", R=R, T=int(rng.integers(1, 500)), Eg=Eg, k=k, El=El,
+                       d=int(rng.choice([64, 192, 320])) if single else int(rng.choice([256, 512])),
+                       F=0 if single else int(rng.choice([128, 256, 640])),
+                       N_out=int(rng.choice([256, 768])) if single else 0,
+                       router=str(rng.choice(["uniform", "zipf", "zipf_rot"])), seed=seed,
+                       self_rank=int(rng.integers(0, R)), first_local=int(rng.integers(0, groups)) * El)
+    mode = B.MODE_NON_OVERLAP if seed % 5 == 4 else B.MODE_OVERLAP
+    csm = int(rng.choice([0, 1, 2, 6, 24]))
+    mgb = int(rng.integers(1, 4))
+    gb = int(rng.choice([0, 2, 4, 5, 64]))
+    inp = I.make_inputs(shape)
+    dsp = I.dispatch(inp, shuffle_seed=int(rng.integers(0, 99)) if seed % 2 else None)
+    ctx = Hn.make_context(shape, max_rows=max(dsp.M, 1) + int(rng.integers(0, 300)), mid_seg_bands=mgb, group_bands=gb)
+    prob = Hn.upload(inp, dsp)
+    Hn.run(ctx, prob, mode=mode, consumer_sm_count=csm)
+    torch.cuda.synchronize()
+    code, detail = ctx.moe_ovl_query_status()
+    assert code == 0, (code, hex(detail))
+    plan = U.oracle_plan(shape, dsp, mgb=mgb)
+    U.check_indices(shape, dsp, plan, ctx.moe_ovl_get_plan(), prob.slot_out.cpu().numpy(),
+                    prob.rows_per_rank_out.cpu().numpy(), prob.segs_per_rank_out.cpu().numpy(),
+                    ctx.moe_ovl_get_report())
+    toks = np.arange(shape.R * shape.T)
+    o = U.oracle_values(inp, toks)
+    U.check_values(shape, dsp, plan, toks, *o, Hn.device_to_bits(prob.out), Hn.device_to_bits(prob.ret))
