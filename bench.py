@@ -146,10 +146,13 @@ def time_oracle(inp, dsp, target_s: float):
         return dt, len(sel), int(rows_of[sel].sum())
 
     dt, n, rows = run(threads)                       # calibration: one token per thread
-    per_tok = dt / max(n, 1) * threads
-    n_target = int(max(threads, min(8192, target_s / max(per_tok, 1e-9) * threads)))
-    n_target = max(threads, n_target // threads * threads)
-    if n_target > n:
+    for _ in range(3):                               # grow the sample until it takes about target_s
+        if dt >= 0.6 * target_s:
+            break
+        n_target = int(min(shape.R * shape.T, max(n + threads, n * target_s / max(dt, 1e-6))))
+        n_target = max(threads, n_target // threads * threads)
+        if n_target <= n:
+            break
         dt, n, rows = run(n_target)
     return flops_of(shape, rows) / dt / 1e12, dt, n, rows, threads
 
