@@ -31,6 +31,7 @@ def sample_tokens(shape, dsp, per_rank, seed=0):
     ("mixtral", 8, 16), ("fine", 8, 24), ("mixtral_zipf", 8, 8), ("paper_op_e16_zipf", 14, 16),
     # points of the sweep grid: 4 local experts of 16, d=4096; (tokens per local expert, ffn, router)
     ((1024, 1024, "uniform"), 2, 16), ((128, 2816, "zipf"), 16, 8), ((4096, 1024, "zipf"), 32, 8),
+    ((16384, 14336, "uniform"), 4, 4),      # the largest point of the grid: 65893 rows, 6.5 GB of workspace
 ])
 def test_full_size_parity(name, csm, per_rank):
     import torch
