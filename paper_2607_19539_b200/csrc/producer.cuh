@@ -45,6 +45,7 @@ constexpr int PROD_STAGE_BYTES = PROD_A_BYTES + PROD_B_BYTES;
 constexpr int PROD_GATHER_WARPS = 4;
 constexpr int PROD_THREADS = 224 + 32 * PROD_GATHER_WARPS;   // TMA, MMA, 4 epilogue warps, scheduler, gather warps
 constexpr int GATHER_ROWS = 8;                         // rows per gather unit
+constexpr int GATHER_HEAD_ROWS = 2;                    // ... in the first super-band of the schedule
 constexpr int PROD_RING = 16;                          // claimed-item ring; roles are never more than 5 items apart
 constexpr int PROD_TMEM_COLS = 512;
 constexpr int PROD_SMEM_BYTES = PROD_STAGES * PROD_STAGE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers, ring*/;
@@ -244,6 +245,44 @@ __device__ __forceinline__ bool epilogue_all(bool ok)
 
 // ------------------------------------------------------------------ kernel
 
+// One gather unit: ROWS rows of band `band` starting at row r0 are copied from the dispatched input into the
+// aligned layout (padding rows zero-filled), COLS x 32 lanes x 16 bytes of every row per pass, i.e.
+// ROWS * COLS loads in flight per lane; then the band's ready count goes up by ROWS (release).
+template <int ROWS, int COLS>
+__device__ __forceinline__ void gather_unit(const Params &p, int band, int r0, int lane)
+{
+    const int nv = p.d / 8;
+    const int valid = p.band_valid[band];
+    int src_row = -1;                                   // lanes 0..ROWS-1: source row, -1 for padding
+    if (lane < ROWS && r0 + lane < valid) src_row = p.row_at[(size_t)band * TB_M + r0 + lane];
+    for (int v0 = 0; v0 < nv; v0 += 32 * COLS) {
+        uint4 buf[COLS][ROWS];
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r) {
+            const int sr = __shfl_sync(0xffffffffu, src_row, r);
+            const uint4 *src = reinterpret_cast<const uint4 *>(p.x + (size_t)(sr >= 0 ? sr : 0) * p.d);
+#pragma unroll
+            for (int c = 0; c < COLS; ++c) {
+                const int v = v0 + 32 * c + lane;
+                buf[c][r] = (sr >= 0 && v < nv) ? __ldcs(src + v) : make_uint4(0, 0, 0, 0);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r) {
+            uint4 *dst = reinterpret_cast<uint4 *>(p.Xa + ((size_t)band * TB_M + r0 + r) * p.d);
+#pragma unroll
+            for (int c = 0; c < COLS; ++c) {
+                const int v = v0 + 32 * c + lane;
+                if (v < nv) dst[v] = buf[c][r];
+            }
+        }
+    }
+    __threadfence();
+    asm volatile("fence.proxy.async;" ::: "memory");      // Xa is read through TMA
+    __syncwarp();
+    if (lane == 0) red_release_add_u32(&p.xready[band], (unsigned)ROWS);
+}
+
 struct ProducerMaps {
     CUtensorMap xa, h, w1, w2;   // all 2-D bf16 row-major, box 64 x 128, 128-byte swizzle
 };
@@ -434,44 +473,28 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
         // ---------------- gather warps: Xa[band * 128 + r] = x[row_at[...]] for units of GATHER_ROWS rows, claimed in
         // schedule order; padding rows are zero-filled (Section 3.2.1).  These warps never wait, so the row
         // counts the TMA warps poll always make progress.
+        // The first super-band is gathered in small units (2 rows: done after two memory round trips at d = 4096)
+        // so that the first tiles can start a few microseconds after the kernel does; the rest in units of
+        // GATHER_ROWS rows, which cost fewer claims.
         const int nbands = p.meta[META_BANDS];
-        const int units_per_band = TB_M / GATHER_ROWS;
-        const int nunits = nbands * units_per_band;
-        const int nv = p.d / 8;
+        const int head_bands = min(nbands, p.group_bands);
+        const int head_units = head_bands * (TB_M / GATHER_HEAD_ROWS);
+        const int nunits = head_units + (nbands - head_bands) * (TB_M / GATHER_ROWS);
         int unit = 0;
         if (lane == 0) unit = atomicAdd(p.next_gather, 1);
         unit = __shfl_sync(0xffffffffu, unit, 0);
         while (unit < nunits) {
             int next = 0;
             if (lane == 0) next = atomicAdd(p.next_gather, 1);      // claimed while this unit's rows are moving
-            const int band = p.sched_band[unit / units_per_band];
-            const int r0 = (unit % units_per_band) * GATHER_ROWS;
-            const int valid = p.band_valid[band];
-            // source row of each of the unit's rows (lanes 0..GATHER_ROWS-1), -1 for padding
-            int src_row = -1;
-            if (lane < GATHER_ROWS && r0 + lane < valid) src_row = p.row_at[(size_t)band * TB_M + r0 + lane];
-            // 64 lanes-worth of 16-byte vectors (1 KiB of every row) per pass: 16 loads in flight per lane
-            for (int v0 = 0; v0 < nv; v0 += 64) {
-                const int va = v0 + lane, vb = v0 + 32 + lane;
-                uint4 buf[2][GATHER_ROWS];
-#pragma unroll
-                for (int r = 0; r < GATHER_ROWS; ++r) {
-                    const int sr = __shfl_sync(0xffffffffu, src_row, r);
-                    const uint4 *src = reinterpret_cast<const uint4 *>(p.x + (size_t)(sr >= 0 ? sr : 0) * p.d);
-                    buf[0][r] = (sr >= 0 && va < nv) ? __ldcs(src + va) : make_uint4(0, 0, 0, 0);
-                    buf[1][r] = (sr >= 0 && vb < nv) ? __ldcs(src + vb) : make_uint4(0, 0, 0, 0);
-                }
-#pragma unroll
-                for (int r = 0; r < GATHER_ROWS; ++r) {
-                    uint4 *dst = reinterpret_cast<uint4 *>(p.Xa + ((size_t)band * TB_M + r0 + r) * p.d);
-                    if (va < nv) dst[va] = buf[0][r];
-                    if (vb < nv) dst[vb] = buf[1][r];
-                }
+            if (unit < head_units) {
+                const int per = TB_M / GATHER_HEAD_ROWS;
+                gather_unit<GATHER_HEAD_ROWS, 16 / GATHER_HEAD_ROWS>(p, p.sched_band[unit / per],
+                                                                     (unit % per) * GATHER_HEAD_ROWS, lane);
+            } else {
+                const int u = unit - head_units, per = TB_M / GATHER_ROWS;
+                gather_unit<GATHER_ROWS, 16 / GATHER_ROWS>(p, p.sched_band[head_bands + u / per],
+                                                           (u % per) * GATHER_ROWS, lane);
             }
-            __threadfence();
-            asm volatile("fence.proxy.async;" ::: "memory");      // Xa is read through TMA
-            __syncwarp();
-            if (lane == 0) red_release_add_u32(&p.xready[band], (unsigned)GATHER_ROWS);
             unit = __shfl_sync(0xffffffffu, next, 0);
         }
     } else {
