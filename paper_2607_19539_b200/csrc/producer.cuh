@@ -7,7 +7,7 @@
 // as clusters of two that share every MMA (cta_group::2): the pair computes a 256 x 256 tile,
 // each CTA holding its own 128 rows of A and only HALF of the B tile, which cuts the operand
 // traffic from L2 per SM by a third against a single-CTA 128 x 256 tile.
-//   warp 0     TMA loads (cp.async.bulk.tensor, 128-byte swizzle) into a 6-stage ring; both
+//   warp 0     TMA loads (cp.async.bulk.tensor, 128-byte swizzle) into a 7-stage ring; both
 //              CTAs' loads complete on the leader CTA's mbarrier
 //   warp 1     in the leader CTA one thread issues tcgen05.mma (bf16 x bf16 -> fp32, M=256
 //              N=256 K=16); accumulators in tensor memory, double buffered (2 x 256 columns)
@@ -38,7 +38,7 @@
 
 namespace moe_ovl {
 
-constexpr int PROD_STAGES = 6;
+constexpr int PROD_STAGES = 7;
 constexpr int PROD_A_BYTES = TB_M * TB_K * 2;          // 16 KiB: this CTA's 128 rows of A
 constexpr int PROD_B_BYTES = (TB_N / 2) * TB_K * 2;    // 16 KiB: this CTA's half of the B tile
 constexpr int PROD_STAGE_BYTES = PROD_A_BYTES + PROD_B_BYTES;
