@@ -30,7 +30,7 @@ UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one producer launch at full size, from the ncu capture
 # summarised in profiles/producer_kernel_mixtral.md.
-NCU_PRODUCER_TRAFFIC_BYTES = {"mixtral": 2790451000 + 383004672}
+NCU_PRODUCER_TRAFFIC_BYTES = {"mixtral": 2763433000 + 387336448}
 
 
 def load_peaks():
