@@ -191,9 +191,11 @@ int moe_ovl_create(moe_ovl_ctx **ctx, const moe_ovl_config *cfg, void *workspace
 /* Enqueues one pass of the path: plan, gather, expert FFN + return, combine.
  * Asynchronous: ordered after earlier work on args->stream, complete for later work
  * on it.  One call in flight per context.  Synchronous argument errors are returned
- * here; device-side errors are reported by moe_ovl_query_status.  Do not capture the call
- * in a CUDA graph: the epoch that marks this call's ready flags is passed by value, so a
- * replay would find the previous replay's flags already "ready". */
+ * here; device-side errors are reported by moe_ovl_query_status.  The call can be
+ * captured in a CUDA graph on args->stream (its internal streams join the capture) and
+ * replayed with new contents in the same buffers: everything that changes from call to call,
+ * the number marking this call's ready flags included, lives in device memory.  The timing
+ * of moe_ovl_get_report then refers to the last replay. */
 int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *args);
 
 /* Same pass with per-call tensors in HOST memory (pinned, for asynchronous copies): copies

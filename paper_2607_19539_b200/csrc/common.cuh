@@ -47,7 +47,8 @@ struct Params {
     int words;          // 32-bit words of one (expert, rank) token bitmap = ceil(T / 32)
     int n1, n2;         // tiles per band: F / 128 (0 for single-projection experts) and dout / 256
     int max_bands, max_items;
-    unsigned epoch;
+    unsigned *epoch_rw;      // same word, for the plan kernel
+    const unsigned *epoch;   // device word: number of this call; the plan kernel bumps it once per call
     unsigned long long timeout_ns;
     long long ret_rows_per_rank;
     // inputs

@@ -116,7 +116,7 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->segs = take((size_t)L->max_bands * 16);
     L->seg_slot0 = take((size_t)L->max_bands * 4);
     L->flags = take((size_t)L->max_bands * L->n2 * 4);
-    L->meta = take(META_COUNT * 4);
+    L->meta = take(META_COUNT * 4 + 4);      // meta[] and the call counter
     L->smid = take(2 * 1024 * 4);            // SM of every GEMM CTA, then of every consumer CTA
     for (int i = 0; i < 6; ++i) L->sb[i] = take((size_t)L->max_bands * 4);
     L->st_ret_rows = (long long)c->tokens_per_rank * L->kmax;
@@ -143,7 +143,6 @@ struct moe_ovl_ctx {
     uint8_t *ws;
     int num_sms;
     int combine_blocks_per_sm, scatter_blocks_per_sm;
-    unsigned epoch;
     cudaStream_t s_prod, s_cons;
     cudaStream_t s_h2d, s_d2h;                        // host-buffer entry point: copies overlap the previous/next pass
     cudaEvent_t ev_h2d[2], ev_comp[2], ev_d2h[2];
@@ -226,7 +225,9 @@ Params make_params(moe_ovl_ctx *ctx)
     p.stamps = at<unsigned long long>(ctx, L.stamps);
     p.smid_prod = at<int>(ctx, L.smid);
     p.smid_cons = at<int>(ctx, L.smid) + 1024;
-    p.flags = at<unsigned>(ctx, L.flags); p.meta = at<int>(ctx, L.meta); p.status = at<int>(ctx, L.status);
+    p.flags = at<unsigned>(ctx, L.flags);
+    p.epoch_rw = at<unsigned>(ctx, L.meta) + META_COUNT;     // the word after meta[], cleared at creation only
+    p.epoch = p.epoch_rw; p.meta = at<int>(ctx, L.meta); p.status = at<int>(ctx, L.status);
     return p;
 }
 
@@ -343,7 +344,7 @@ int moe_ovl_create(moe_ovl_ctx **out, const moe_ovl_config *cfg, void *workspace
     if (rc != MOE_OVL_OK) return fail(rc);
     // flags hold the epoch of the call that finished the tile: clear them once, never again
     CREATE_CHECK(cudaMemset(ctx->ws + L.flags, 0, (size_t)L.max_bands * L.n2 * 4));
-    CREATE_CHECK(cudaMemset(ctx->ws + L.meta, 0, META_COUNT * 4));
+    CREATE_CHECK(cudaMemset(ctx->ws + L.meta, 0, META_COUNT * 4 + 4));
     CREATE_CHECK(cudaMemset(ctx->ws + L.status, 0, ST_COUNT * 4));
 #undef CREATE_CHECK
     *out = ctx;
@@ -413,7 +414,6 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
 
     Params p = make_params(ctx);
     p.M = a->num_rows;
-    p.epoch = ++ctx->epoch;
     p.lag_items = prod_ctas;                        // two rounds of the prod_ctas / 2 CTA pairs
     p.ret_rows_per_rank = a->ret_rows_per_rank;
     p.x = static_cast<const uint16_t *>(a->x);

@@ -41,6 +41,7 @@ __device__ __forceinline__ void move_segments(const Params &p, volatile int *s_s
 {
     const int nseg = p.meta[META_SEGS];
     const int lane = threadIdx.x & 31;
+    const unsigned epoch = *p.epoch;
     for (;;) {
         __syncthreads();
         if (threadIdx.x < 32) {
@@ -53,7 +54,7 @@ __device__ __forceinline__ void move_segments(const Params &p, volatile int *s_s
                 const int nflags = seg.y * p.n2;
                 const unsigned *f = p.flags + (size_t)seg.x * p.n2;
                 for (int i = lane; i < nflags && ok; i += 32)
-                    ok = wait_global(f + i, p.epoch, false, p, SITE_CONS_FLAG, (long long)seg.x * p.n2 + i, 2048);
+                    ok = wait_global(f + i, epoch, false, p, SITE_CONS_FLAG, (long long)seg.x * p.n2 + i, 2048);
                 ok = __all_sync(0xffffffffu, ok);
             }
             if (lane == 0) { s_seg[0] = s; s_seg[1] = ok ? 1 : 0; }

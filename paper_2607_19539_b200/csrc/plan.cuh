@@ -91,6 +91,9 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     __syncthreads();
     if (!s_last) return;
     __threadfence();
+    // A new call: its ready flags carry a new number.  Kept in device memory (not passed by value) so that a
+    // captured call can be replayed.
+    if (threadIdx.x == 0) *p.epoch_rw += 1u;
 
     __shared__ int n[PLAN_MAX_GROUPS], nb[PLAN_MAX_GROUPS], gstart[PLAN_MAX_GROUPS], gslot[PLAN_MAX_GROUPS];
     __shared__ int gsched[PLAN_MAX_GROUPS], gsegoff[PLAN_MAX_GROUPS];

@@ -338,6 +338,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
     const uint32_t tmem_base = *tmem_slot_gen;
 
     const int n_items = p.meta[META_ITEMS];
+    const unsigned epoch = *p.epoch;
     // n-th item of this cluster: wait until the scheduler has filled ring slot n % PROD_RING, then read it.
     // Returns n_items (or more) when the schedule is exhausted, -1 on a give-up.
     auto claimed = [&](int n) -> int {
@@ -568,7 +569,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             if (leader && present) {
                 if (kind == KIND_G1) red_release_add_u32(&p.hcount[band], 1u);
                 else if (raise_flags) {
-                    st_release_u32(&p.flags[(size_t)band * p.n2 + tile], p.epoch);
+                    st_release_u32(&p.flags[(size_t)band * p.n2 + tile], epoch);
                     const unsigned long long now = globaltimer_ns();
                     stamp_max(&p.stamps[STAMP_FIRST_FLAG_INV], ~now);
                     stamp_max(&p.stamps[STAMP_LAST_FLAG], now);

@@ -359,3 +359,37 @@ def test_random_shapes_full_parity(seed):
     toks = np.arange(shape.R * shape.T)
     o = U.oracle_values(inp, toks)
     U.check_values(shape, dsp, plan, toks, *o, Hn.device_to_bits(prob.out), Hn.device_to_bits(prob.ret))
+
+
+def test_call_can_be_captured_in_a_cuda_graph_and_replayed():
+    """A captured call replays with new contents in the same buffers (the number that marks a call's ready flags
+    lives in device memory, so every replay gets a fresh one); overlap mode, both internal streams in the capture."""
+    torch, B, Hn = _gpu()
+    shape = I.SHAPES["small_zipf_rot"]
+    inp = I.make_inputs(shape)
+    dsp = I.dispatch(inp)
+    ctx = Hn.make_context(shape, max_rows=dsp.M)
+    ref_ctx = Hn.make_context(shape, max_rows=dsp.M)
+    prob = Hn.upload(inp, dsp)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=4)          # warm-up outside the capture
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side, capture_error_mode="thread_local"):
+        Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=4)
+    for scale in (1.0, -0.5, 2.0, 0.25):
+        x_new = (Hn.bits_to_device(dsp.x_rows, "cuda:0").float() * scale).to(torch.bfloat16)
+        prob.x.copy_(x_new)
+        prob.out.fill_(float("nan"))
+        prob.ret.fill_(float("nan"))
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert ctx.moe_ovl_query_status()[0] == 0
+        ref = Hn.upload(inp, dsp, w1=prob.w1, w2=prob.w2)
+        ref.x.copy_(x_new)
+        Hn.run(ref_ctx, ref, mode=B.MODE_NON_OVERLAP)
+        torch.cuda.synchronize()
+        assert torch.equal(prob.out.view(torch.int16), ref.out.view(torch.int16)), scale
+        assert torch.equal(prob.ret.view(torch.int16), ref.ret.view(torch.int16)), scale
