@@ -52,7 +52,16 @@ enum {
     MOE_OVL_ERR_BAD_ROUTING = -6  /* routing metadata inconsistent (asynchronous, see query_status) */
 };
 
-enum { MOE_OVL_MODE_OVERLAP = 0, MOE_OVL_MODE_NON_OVERLAP = 1 };
+enum {
+    MOE_OVL_MODE_OVERLAP = 0,     /* producer + consumer kernel on consumer_sm_count dedicated SMs (Section 3.3.3) */
+    MOE_OVL_MODE_NON_OVERLAP = 1, /* comparison baseline of Section 4.1: GEMM to completion, then scatter */
+    MOE_OVL_MODE_IN_KERNEL = 2,   /* same flag protocol and segments, but the finished segments are moved by spare
+                                     warps inside the GEMM CTAs: no SM is taken from the GEMM, one kernel, nothing
+                                     to co-schedule.  Not in the paper: on one GPU the return is an HBM copy that
+                                     needs a few percent of one SM's load/store slots, not an SM of its own. */
+    MOE_OVL_MODE_AUTO = 3         /* the library picks one of the three (and the consumer budget) from the shape
+                                     and the number of rows; moe_ovl_report.mode_used tells which */
+};
 
 /* tile geometry, fixed by the kernels */
 #define MOE_OVL_TB_M 128  /* rows per band (output tile height, tb_M of Algorithm 1) */
@@ -84,6 +93,11 @@ typedef struct {
 #define MOE_OVL_FLAG_HOST_STAGING 1u /* reserve workspace for moe_ovl_expert_return_host */
 #define MOE_OVL_FLAG_TEST_NO_FLAGS 2u /* test hook: in OVERLAP mode the GEMM raises no ready flags, so the consumer's
                                          bounded wait runs out and the call ends with MOE_OVL_ERR_TIMEOUT */
+#define MOE_OVL_FLAG_TRACE 4u         /* reserve workspace for, and record, the per-item / per-unit device trace
+                                         (moe_ovl_get_trace); off by default, costs nothing when off */
+#define MOE_OVL_FLAG_TEST_SKIP_GATHER 8u /* test hook: the first band of the schedule is never gathered, so the GEMM's
+                                         own bounded wait for it runs out (exercises the give-up path inside the GEMM
+                                         kernel: copies drained, tensor memory freed, MOE_OVL_ERR_TIMEOUT) */
 
 typedef struct {
     uint32_t struct_size;
@@ -139,7 +153,11 @@ typedef struct {
     int32_t producer_ctas;
     int32_t consumer_ctas;    /* 0 in NON_OVERLAP */
     int32_t kernel_launches;  /* kernels of this library launched by the call */
-    int32_t segments_by_gemm_ctas; /* OVERLAP: segments moved by GEMM CTAs that had run out of tiles */
+    int32_t segments_by_gemm_ctas; /* segments (units) moved by GEMM CTAs: in OVERLAP those that had run out of
+                                      tiles, in IN_KERNEL all of them */
+    int32_t mode_used;        /* MOE_OVL_MODE_* the call ran in (differs from args->mode only for MODE_AUTO) */
+    int32_t timing_valid;     /* 0 when the call was captured into a CUDA graph: the ms_* fields are then 0 (events
+                                 recorded during capture carry no time); the us_* device stamps stay valid */
     float ms_total;           /* whole call on the caller's stream */
     float ms_prep;            /* plan + gather into the aligned layout */
     float ms_expert_return;   /* start of the GEMM to the last row landed in ret */
@@ -188,14 +206,23 @@ int moe_ovl_limits(const moe_ovl_config *cfg, int32_t *max_bands, int32_t *max_i
  * allocates no device memory. */
 int moe_ovl_create(moe_ovl_ctx **ctx, const moe_ovl_config *cfg, void *workspace, size_t workspace_bytes);
 
-/* Enqueues one pass of the path: plan, gather, expert FFN + return, combine.
+/* Enqueues one pass of the path.  What it computes, by passage of the paper:
+ *   Section 2.1, steps 3-5      expert FFN on every routed row, return of each output row to the
+ *                               rank that owns the token, gate-weighted sum per token at the owner
+ *   Section 3.2.1, Algorithm 1  remote-owner-aligned row layout (remote groups padded to tb_M, local last)
+ *   Section 3.2.2, Algorithm 1  remote-first tile schedule (experts by remote band count)
+ *   Section 3.2.3               combine plan: destination, receive-buffer offset, valid rows per tile
+ *   Section 3.3.1               rank-wide persistent GEMM, ready flag per finished output tile
+ *   Section 3.3.2, Figure 3b    segment-granular transfer (first / middle / last segments)
+ *   Section 3.3.3               co-scheduling of producer and consumer on disjoint SM sets
  * Asynchronous: ordered after earlier work on args->stream, complete for later work
  * on it.  One call in flight per context.  Synchronous argument errors are returned
  * here; device-side errors are reported by moe_ovl_query_status.  The call can be
  * captured in a CUDA graph on args->stream (its internal streams join the capture) and
  * replayed with new contents in the same buffers: everything that changes from call to call,
- * the number marking this call's ready flags included, lives in device memory.  The timing
- * of moe_ovl_get_report then refers to the last replay. */
+ * the number marking this call's ready flags included, lives in device memory.  A captured
+ * call records no timing events: moe_ovl_get_report then returns timing_valid = 0 with the
+ * ms_* fields zero, and moe_ovl_get_gemm_time skips it. */
 int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *args);
 
 /* Same pass with per-call tensors in HOST memory (pinned, for asynchronous copies): copies
@@ -230,6 +257,30 @@ int moe_ovl_get_gemm_time(moe_ovl_ctx *ctx, int32_t last_n, float *avg_ms, int32
 int moe_ovl_get_sm_map(moe_ovl_ctx *ctx, int32_t *producer_smid, int32_t *consumer_smid);
 int moe_ovl_read_buffer(moe_ovl_ctx *ctx, int32_t which, size_t offset, size_t bytes, void *host_dst);
 
+/* Device trace of the last call (needs MOE_OVL_FLAG_TRACE).  One record per schedule item of the GEMM
+ * kernel and one per moved unit of the return (a unit is a whole segment, or one of moe_ovl_report's
+ * equal row slices of it when spare warps of the GEMM CTAs move the return); times are nanoseconds of the
+ * GPU's global timer after the first GEMM CTA started.  It is what the overlap ratio of Section 4.2.2, the
+ * tail after the last tile and the idle time of the consumer (Section 3.3.3) are read from. */
+enum { MOE_OVL_TRACE_ITEM = 0, MOE_OVL_TRACE_UNIT = 1 };
+typedef struct {
+    int32_t kind;      /* MOE_OVL_TRACE_ITEM / MOE_OVL_TRACE_UNIT */
+    int32_t index;     /* item: position in issue order (moe_ovl_plan_view.item); unit: segment * chunks + chunk */
+    int32_t cta;       /* item: leader CTA of the pair that ran it; unit: CTA that moved it */
+    int32_t who;       /* unit: 0 consumer CTA, 1 GEMM CTA that had run out of tiles, 2 spare warps of a GEMM CTA */
+    int32_t rows;      /* unit: rows moved */
+    int32_t chunks;    /* unit: slices per segment in this call */
+    int64_t ns_claim;  /* item: claimed by the pair's scheduler; unit: every ready flag of the segment seen */
+    int64_t ns_ready;  /* item: first operand stage landed, the MMAs can start; unit: same as ns_claim */
+    int64_t ns_done0;  /* item: tile of the pair's first band published (flag or band counter), taken just
+                          before the release store; unit: last row landed in the receive buffer */
+    int64_t ns_done1;  /* item: same for the pair's second band, -1 if absent; unit: same as ns_done0 */
+} moe_ovl_trace_record;
+/* Waits for the last call, then writes its records to HOST memory: items in issue order, then units in
+ * claim order.  *written = bytes written.  host_buf == NULL: only reports the bytes needed.
+ * MOE_OVL_ERR_INVALID_ARG if `bytes` is too small, MOE_OVL_ERR_UNSUPPORTED if the context has no trace. */
+int moe_ovl_get_trace(moe_ovl_ctx *ctx, void *host_buf, size_t bytes, size_t *written);
+
 int moe_ovl_destroy(moe_ovl_ctx *ctx);
 
 /* Return slots without any allocation (the paper has no counterpart: this entry point
@@ -254,9 +305,12 @@ int moe_ovl_destroy(moe_ovl_ctx *ctx);
  * MOE_OVL_STATIC_MAX_WORDS (the array is 512 KiB, and every GPU that loads the library
  * holds it until the process exits); larger problems return MOE_OVL_ERR_UNSUPPORTED and
  * belong to moe_ovl_expert_return with a workspace.
- * The first call on a device resolves the array's device address (one runtime query,
- * with that device made current) and should therefore be made before any stream capture
- * begins on that device.  Every call uses the same array: the kernel clears what it needs
+ * Every call makes `device` the calling thread's current device and leaves it so; `stream`
+ * must belong to that device.  The first call on a device also resolves the array's device
+ * address (one runtime query) and should therefore be made before any stream capture begins
+ * on that device.  There is no status channel: a row whose metadata is out of range, or that
+ * lies beyond the sum of expert_counts, gets slot -1; a duplicate (expert, rank, token) row --
+ * which moe_ovl_expert_return reports as bad routing -- silently gets its twin's slot.  Every call uses the same array: the kernel clears what it needs
  * at its start, but two calls that overlap on one GPU (different streams) race on it and
  * give wrong slots -- keep calls on a device ordered. */
 #define MOE_OVL_STATIC_MAX_GROUPS 1024

@@ -17,9 +17,12 @@ from . import build as _build
 
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_WORKSPACE, ERR_TIMEOUT, ERR_BAD_ROUTING = -1, -2, -3, -4, -5, -6
-MODE_OVERLAP, MODE_NON_OVERLAP = 0, 1
+MODE_OVERLAP, MODE_NON_OVERLAP, MODE_IN_KERNEL, MODE_AUTO = 0, 1, 2, 3
 FLAG_HOST_STAGING = 1
 FLAG_TEST_NO_FLAGS = 2
+FLAG_TRACE = 4
+FLAG_TEST_SKIP_GATHER = 8
+TRACE_ITEM, TRACE_UNIT = 0, 1
 BUF_XA, BUF_H, BUF_Y = 0, 1, 2
 TB_M, TB_N, H_TILE = 128, 256, 128
 
@@ -27,7 +30,7 @@ EXPORTS = [
     "moe_ovl_workspace_bytes", "moe_ovl_limits", "moe_ovl_create", "moe_ovl_expert_return",
     "moe_ovl_expert_return_host", "moe_ovl_host_join", "moe_ovl_query_status", "moe_ovl_get_report", "moe_ovl_get_plan",
     "moe_ovl_get_sm_map", "moe_ovl_get_gemm_time", "moe_ovl_read_buffer", "moe_ovl_destroy", "moe_ovl_strerror", "moe_ovl_last_cuda_error",
-    "moe_ovl_return_slots_static",
+    "moe_ovl_return_slots_static", "moe_ovl_get_trace",
 ]
 
 
@@ -58,11 +61,23 @@ class HostArgs(C.Structure):
 class Report(C.Structure):
     _fields_ = [("padded_rows", C.c_int32), ("num_bands", C.c_int32), ("num_items", C.c_int32),
                 ("num_segments", C.c_int32), ("producer_ctas", C.c_int32), ("consumer_ctas", C.c_int32),
-                ("kernel_launches", C.c_int32), ("segments_by_gemm_ctas", C.c_int32), ("ms_total", C.c_float),
+                ("kernel_launches", C.c_int32), ("segments_by_gemm_ctas", C.c_int32), ("mode_used", C.c_int32),
+                ("timing_valid", C.c_int32), ("ms_total", C.c_float),
                 ("ms_prep", C.c_float), ("ms_expert_return", C.c_float), ("ms_producer", C.c_float),
                 ("ms_mover", C.c_float), ("ms_combine", C.c_float), ("us_first_flag", C.c_float),
                 ("us_gemm_done", C.c_float), ("us_return_done", C.c_float), ("copy_gbs_per_cta", C.c_float),
                 ("overlap_ratio", C.c_float)]
+
+
+class TraceRecord(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("index", C.c_int32), ("cta", C.c_int32), ("who", C.c_int32),
+                ("rows", C.c_int32), ("chunks", C.c_int32), ("ns_claim", C.c_int64), ("ns_ready", C.c_int64),
+                ("ns_done0", C.c_int64), ("ns_done1", C.c_int64)]
+
+
+TRACE_DTYPE = np.dtype([("kind", np.int32), ("index", np.int32), ("cta", np.int32), ("who", np.int32),
+                        ("rows", np.int32), ("chunks", np.int32), ("ns_claim", np.int64), ("ns_ready", np.int64),
+                        ("ns_done0", np.int64), ("ns_done1", np.int64)])
 
 
 class PlanView(C.Structure):
@@ -111,6 +126,7 @@ def load(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moe_ovl_get_gemm_time.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
     lib.moe_ovl_get_sm_map.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     lib.moe_ovl_read_buffer.argtypes = [C.c_void_p, C.c_int32, C.c_size_t, C.c_size_t, C.c_void_p]
+    lib.moe_ovl_get_trace.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
     lib.moe_ovl_destroy.argtypes = [C.c_void_p]
     lib.moe_ovl_last_cuda_error.argtypes = [C.c_void_p]
     lib.moe_ovl_return_slots_static.argtypes = [C.c_int32] * 5 + [C.c_void_p] * 6
@@ -191,6 +207,8 @@ class ReportView:
     us_return_done: float = 0.0
     overlap_ratio: float = 0.0
     copy_gbs_per_cta: float = 0.0
+    mode_used: int = 0
+    timing_valid: int = 1
 
 
 class MoeOvl:
@@ -254,7 +272,7 @@ class MoeOvl:
         return ReportView(r.padded_rows, r.num_bands, r.num_items, r.num_segments, r.producer_ctas, r.consumer_ctas,
                           r.kernel_launches, r.ms_total, r.ms_prep, r.ms_expert_return, r.ms_producer, r.ms_mover,
                           r.ms_combine, r.segments_by_gemm_ctas, r.us_first_flag, r.us_gemm_done, r.us_return_done,
-                          r.overlap_ratio, r.copy_gbs_per_cta)
+                          r.overlap_ratio, r.copy_gbs_per_cta, r.mode_used, r.timing_valid)
 
     def moe_ovl_get_plan(self) -> Dict[str, np.ndarray]:
         rep = self.moe_ovl_get_report()
@@ -274,6 +292,17 @@ class MoeOvl:
         arrs["tok_slot"] = arrs["tok_slot"].reshape(-1, self.kmax)
         arrs["tok_gate"] = arrs["tok_gate"].reshape(-1, self.kmax)
         return arrs
+
+    def moe_ovl_get_trace(self) -> np.ndarray:
+        """Trace records of the last call as a structured array (fields of moe_ovl_trace_record)."""
+        need = C.c_size_t(0)
+        self._check(self.lib.moe_ovl_get_trace(self.ctx, None, 0, C.byref(need)), "moe_ovl_get_trace")
+        assert need.value % C.sizeof(TraceRecord) == 0 and TRACE_DTYPE.itemsize == C.sizeof(TraceRecord)
+        out = np.zeros(need.value // TRACE_DTYPE.itemsize, TRACE_DTYPE)
+        if need.value:
+            self._check(self.lib.moe_ovl_get_trace(self.ctx, out.ctypes.data, need.value, C.byref(need)),
+                        "moe_ovl_get_trace")
+        return out
 
     def moe_ovl_get_gemm_time(self, last_n: int):
         """(mean GEMM kernel duration in ms over the last calls, number of calls averaged)."""

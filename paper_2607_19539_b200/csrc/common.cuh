@@ -24,6 +24,9 @@ enum { STAMP_START_INV = 0, STAMP_FIRST_FLAG_INV, STAMP_LAST_FLAG, STAMP_LAST_SE
 // status[] slots
 enum { ST_CODE = 0, ST_ABORT = 1, ST_DETAIL_LO = 2, ST_DETAIL_HI = 3, ST_COUNT = 4 };
 
+// who moved a unit of the return (trace records)
+enum { TRACE_BY_CONSUMER = 0, TRACE_BY_GEMM_TAIL = 1, TRACE_BY_GEMM_WARPS = 2 };
+
 constexpr int ERR_TIMEOUT = -5;
 constexpr int ERR_BAD_ROUTING = -6;
 
@@ -31,8 +34,10 @@ constexpr int ERR_BAD_ROUTING = -6;
 enum : long long {
     SITE_TMA_EMPTY = 1, SITE_TMA_HCOUNT, SITE_MMA_FULL, SITE_MMA_TEMPTY, SITE_EPI_TFULL, SITE_CONS_FLAG,
     SITE_MMA_DRAIN, SITE_TMA_DRAIN, SITE_CLAIM, SITE_SCHED_GO, SITE_TMA_XREADY,
-    SITE_ROW_RANGE = 16, SITE_ROW_DUP, SITE_COUNT_SUM, SITE_TOK_OVERFLOW
+    SITE_ROW_RANGE = 16, SITE_ROW_DUP, SITE_COUNT_SUM, SITE_TOK_OVERFLOW, SITE_RET_OVERFLOW
 };
+
+struct __align__(32) TraceRec { unsigned long long a, b, c, d; };
 
 struct Params {
     // problem
@@ -42,6 +47,7 @@ struct Params {
     int single;         // single-projection experts: no first GEMM, the output GEMM reads Xa
     int M;
     int mgb;            // bands per middle segment
+    int seg_chunks;     // units a segment is moved in: 1 (whole segments), more when spare warps of GEMM CTAs move them
     int group_bands;    // bands interleaved in one super-band
     int lag_items;      // schedule items between a band's last first-GEMM tile and its first second-GEMM tile
     int words;          // 32-bit words of one (expert, rank) token bitmap = ceil(T / 32)
@@ -86,6 +92,11 @@ struct Params {
     unsigned *hcount;     // [max_bands] first-GEMM tiles finished per band
     unsigned *flags;      // [max_bands*n2] epoch of the call that finished the tile
     int *meta;            // [META_COUNT]
+    // optional trace (null when off), raw %globaltimer values: one record per schedule item {claimed, first
+    // operands landed, published by CTA 0 of the pair, published by CTA 1} plus the leader CTA's index, and
+    // one per moved unit {who << 32 | CTA, flags seen, copy done, rows}
+    TraceRec *trace_items, *trace_units;
+    int *trace_item_cta;
     int *status;          // [ST_COUNT]
 };
 

@@ -24,6 +24,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 constexpr size_t ALIGN = 1024;
+constexpr int MAX_SEG_CHUNKS = 8;     // slices a segment is moved in when spare warps of GEMM CTAs move the return
 inline size_t align_up(size_t v, size_t a = ALIGN) { return (v + a - 1) / a * a; }
 
 struct Layout {
@@ -34,6 +35,7 @@ struct Layout {
     size_t wordpfx, group_rows, group_start, group_slot, pos, slot, row_at, xready;
     size_t band_expert, band_dest, band_valid, band_slot0, sched_band, items, segs, seg_slot0;
     size_t tok_gate, flags, meta;
+    size_t trace_items, trace_units, trace_item_cta, trace_bytes;   // MOE_OVL_FLAG_TRACE
     size_t sb[6];
     // host staging (MOE_OVL_FLAG_HOST_STAGING)
     size_t st_x[2], st_counts[2], st_rank[2], st_token[2], st_gate[2], st_out[2], st_ret;   // two staging slots
@@ -120,6 +122,13 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->smid = take(2 * 1024 * 4);            // SM of every GEMM CTA, then of every consumer CTA
     for (int i = 0; i < 6; ++i) L->sb[i] = take((size_t)L->max_bands * 4);
     L->st_ret_rows = (long long)c->tokens_per_rank * L->kmax;
+    L->trace_bytes = 0;
+    if (c->flags & MOE_OVL_FLAG_TRACE) {
+        L->trace_items = take((size_t)L->max_items * sizeof(TraceRec));
+        L->trace_units = take((size_t)L->max_bands * MAX_SEG_CHUNKS * sizeof(TraceRec));
+        L->trace_item_cta = take((size_t)L->max_items * 4);
+        L->trace_bytes = off - L->trace_items;
+    }
     if (c->flags & MOE_OVL_FLAG_HOST_STAGING) {
         for (int s = 0; s < 2; ++s) {
             L->st_x[s] = take((size_t)std::max(c->max_rows, 1) * d * 2);
@@ -156,7 +165,9 @@ struct moe_ovl_ctx {
     unsigned long long calls;
     cudaStream_t last_stream;
     bool ran;
-    int last_mode, last_prod_ctas, last_cons_ctas, last_launches, last_rows;
+    int last_mode, last_prod_ctas, last_cons_ctas, last_launches, last_rows, last_chunks;
+    bool last_timed;                                  // false when the last call was captured into a graph
+    bool hist_timed[MOE_OVL_TIMING_HISTORY];
     int last_cuda_error;
     EncodeTiledFn encode;
     CUtensorMap map_xa, map_h;
@@ -228,7 +239,35 @@ Params make_params(moe_ovl_ctx *ctx)
     p.flags = at<unsigned>(ctx, L.flags);
     p.epoch_rw = at<unsigned>(ctx, L.meta) + META_COUNT;     // the word after meta[], cleared at creation only
     p.epoch = p.epoch_rw; p.meta = at<int>(ctx, L.meta); p.status = at<int>(ctx, L.status);
+    p.seg_chunks = 1;
+    if (c.flags & MOE_OVL_FLAG_TRACE) {
+        p.trace_items = at<TraceRec>(ctx, L.trace_items);
+        p.trace_units = at<TraceRec>(ctx, L.trace_units);
+        p.trace_item_cta = at<int>(ctx, L.trace_item_cta);
+    }
     return p;
+}
+
+// Consumer budget for MODE_OVERLAP with consumer_sm_count = 0 (Section 3.3.3: too few consumer SMs and the
+// transfer falls behind, too many and the GEMM loses capacity).  Every SM given up costs 1/SMs of the GEMM
+// time; the return it hides is worth t_return.  About half of the break-even count SMs * t_return / t_gemm,
+// with t_return = 4*d bytes per row at ~5 TB/s and t_gemm = 6*d*F flop per row at ~1.2 PFLOP/s.
+int choose_consumer_sms(const moe_ovl_ctx *ctx)
+{
+    const moe_ovl_config &c = ctx->cfg;
+    const Layout &L = ctx->L;
+    const double t_ret = 4.0 * L.dout / 5.0e12;
+    const double t_gemm = (L.single ? 2.0 * c.d_model * (double)L.dout : 6.0 * c.d_model * (double)c.d_ffn) / 1.2e15;
+    const double breakeven = ctx->num_sms * t_ret / t_gemm;
+    return std::min(16, std::max(2, 2 * (int)(breakeven / 4.0 + 0.5)));
+}
+
+// MODE_AUTO: which of the three ways to run the return, and with how many consumer SMs.
+void choose_mode(const moe_ovl_ctx *ctx, int num_rows, int *mode, int *consumer_sms)
+{
+    (void)num_rows;
+    *mode = MOE_OVL_MODE_IN_KERNEL;
+    *consumer_sms = choose_consumer_sms(ctx);
 }
 
 int sync_last(moe_ovl_ctx *ctx)
@@ -383,38 +422,41 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     if (!a->expert_counts || !a->w1 || (!a->w2 && !L.single) || !a->ret || !a->out) return MOE_OVL_ERR_INVALID_ARG;
     if (a->num_rows > 0 && (!a->x || !a->src_rank || !a->src_token || !a->gate)) return MOE_OVL_ERR_INVALID_ARG;
     if (a->ret_rows_per_rank < (int64_t)c.tokens_per_rank * L.kmax) return MOE_OVL_ERR_INVALID_ARG;
-    if (a->mode != MOE_OVL_MODE_OVERLAP && a->mode != MOE_OVL_MODE_NON_OVERLAP) return MOE_OVL_ERR_INVALID_ARG;
+    if (a->mode < MOE_OVL_MODE_OVERLAP || a->mode > MOE_OVL_MODE_AUTO) return MOE_OVL_ERR_INVALID_ARG;
     const uintptr_t align16 = reinterpret_cast<uintptr_t>(a->x) | reinterpret_cast<uintptr_t>(a->w1) |
                               reinterpret_cast<uintptr_t>(a->w2) | reinterpret_cast<uintptr_t>(a->ret) |
                               reinterpret_cast<uintptr_t>(a->out);
     if (align16 & 15u) return MOE_OVL_ERR_INVALID_ARG;
-    const bool overlap = a->mode == MOE_OVL_MODE_OVERLAP;
+    int mode = a->mode, want = a->consumer_sm_count;
+    if (mode == MOE_OVL_MODE_AUTO) choose_mode(ctx, a->num_rows, &mode, &want);
+    const bool dedicated = mode == MOE_OVL_MODE_OVERLAP, in_kernel = mode == MOE_OVL_MODE_IN_KERNEL;
     int prod_ctas, cons_ctas = 0;
-    if (overlap) {
-        if (a->consumer_sm_count < 0 || a->consumer_sm_count > ctx->num_sms / 2) return MOE_OVL_ERR_INVALID_ARG;
-        int want = a->consumer_sm_count;
-        if (want == 0) {
-            // Automatic budget (Section 3.3.3: too few consumer SMs and the transfer falls behind, too many and
-            // the GEMM loses capacity).  Every SM given up costs 1/SMs of the GEMM time; the return it hides is
-            // worth t_return.  Take about half of the break-even count SMs * t_return / t_gemm, with
-            // t_return = 4*d bytes per row at ~5 TB/s and t_gemm = 6*d*F flop per row at ~1.2 PFLOP/s.
-            const double t_ret = 4.0 * L.dout / 5.0e12;
-            const double t_gemm = (L.single ? 2.0 * c.d_model * (double)L.dout : 6.0 * c.d_model * (double)c.d_ffn) / 1.2e15;
-            const double breakeven = ctx->num_sms * t_ret / t_gemm;
-            want = std::min(16, std::max(2, 2 * (int)(breakeven / 4.0 + 0.5)));
-        }
+    if (dedicated) {
+        if (want < 0 || want > ctx->num_sms / 2) return MOE_OVL_ERR_INVALID_ARG;
+        if (want == 0) want = choose_consumer_sms(ctx);
         cons_ctas = (want + 1) & ~1;                        // whole SM pairs: the GEMM's CTAs work in pairs
         prod_ctas = (ctx->num_sms - cons_ctas) & ~1;        // disjoint SM sets: grids sum to the SM count
     } else {
-        prod_ctas = (c.producer_sm_limit > 0 ? std::min(c.producer_sm_limit, ctx->num_sms) : ctx->num_sms) & ~1;
+        const bool limited = mode == MOE_OVL_MODE_NON_OVERLAP && c.producer_sm_limit > 0;
+        prod_ctas = (limited ? std::min(c.producer_sm_limit, ctx->num_sms) : ctx->num_sms) & ~1;
         if (prod_ctas < 2) return MOE_OVL_ERR_INVALID_ARG;
     }
     CU_CHECK(ctx, cudaSetDevice(c.device));
     cudaStream_t st = static_cast<cudaStream_t>(a->stream);
+    // Events recorded while a stream is being captured carry no time: a captured call records none of the
+    // timing events, and the report says so.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    CU_CHECK(ctx, cudaStreamIsCapturing(st, &cap));
+    const bool timed = cap == cudaStreamCaptureStatusNone;
+#define TIME_POINT(ev, stream)                                      \
+    do {                                                            \
+        if (timed) CU_CHECK(ctx, cudaEventRecord((ev), (stream)));  \
+    } while (0)
 
     Params p = make_params(ctx);
     p.M = a->num_rows;
     p.lag_items = prod_ctas;                        // two rounds of the prod_ctas / 2 CTA pairs
+    p.seg_chunks = in_kernel ? MAX_SEG_CHUNKS : 1;
     p.ret_rows_per_rank = a->ret_rows_per_rank;
     p.x = static_cast<const uint16_t *>(a->x);
     p.expert_counts = a->expert_counts; p.src_rank = a->src_rank; p.src_token = a->src_token; p.gate = a->gate;
@@ -441,9 +483,13 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
 
     int launches = 0;
     const int hist = (int)(ctx->calls % MOE_OVL_TIMING_HISTORY);
-    CU_CHECK(ctx, cudaEventRecord(ctx->t_begin, st));
-    // ---- plan + gather (8a-1 .. 8a-3): integer kernels on the caller's stream
+    int kflags = (c.flags & MOE_OVL_FLAG_TEST_SKIP_GATHER) ? PROD_SKIP_FIRST_BAND : 0;
+    if (mode != MOE_OVL_MODE_NON_OVERLAP && !(c.flags & MOE_OVL_FLAG_TEST_NO_FLAGS)) kflags |= PROD_RAISE_FLAGS;
+    if (in_kernel) kflags |= PROD_WARP_MOVERS;
+    TIME_POINT(ctx->t_begin, st);
+    // ---- plan (row layout, tile schedule, combine plan): integer kernels on the caller's stream
     CU_CHECK(ctx, cudaMemsetAsync(ctx->ws + L.zero_begin, 0, L.zero_end - L.zero_begin, st));
+    if (L.trace_bytes) CU_CHECK(ctx, cudaMemsetAsync(ctx->ws + L.trace_items, 0, L.trace_bytes, st));
     plan_mark_build_kernel<<<std::max(1, (p.M + PLAN_THREADS - 1) / PLAN_THREADS), PLAN_THREADS, 0, st>>>(p, sc);
     ++launches;
     if (p.M > 0) {
@@ -451,51 +497,64 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
         ++launches;
     }
     CU_CHECK(ctx, cudaGetLastError());
-    CU_CHECK(ctx, cudaEventRecord(ctx->t_prep, st));
+    TIME_POINT(ctx->t_prep, st);
 
-    if (overlap) {
+    if (dedicated) {
         // ---- two persistent kernels on two streams, disjoint SM sets (Section 3.3.3)
         CU_CHECK(ctx, cudaEventRecord(ctx->ev_fork, st));
         CU_CHECK(ctx, cudaStreamWaitEvent(ctx->s_cons, ctx->ev_fork, 0));
         CU_CHECK(ctx, cudaStreamWaitEvent(ctx->s_prod, ctx->ev_fork, 0));
-        CU_CHECK(ctx, cudaEventRecord(ctx->t_m0, ctx->s_cons));
-        consumer_kernel<<<cons_ctas, MOVER_THREADS, CONSUMER_SMEM_BYTES, ctx->s_cons>>>(p);
-        CU_CHECK(ctx, cudaEventRecord(ctx->t_m1, ctx->s_cons));
-        CU_CHECK(ctx, cudaEventRecord(ctx->ev_cons_done, ctx->s_cons));
-        CU_CHECK(ctx, cudaEventRecord(ctx->t_p0, ctx->s_prod));
-        CU_CHECK(ctx, cudaEventRecord(ctx->h_p0[hist], ctx->s_prod));
-        producer_kernel<<<prod_ctas, PROD_THREADS, PROD_SMEM_BYTES, ctx->s_prod>>>(
-            maps, p, (c.flags & MOE_OVL_FLAG_TEST_NO_FLAGS) ? 0 : 1);
-        CU_CHECK(ctx, cudaEventRecord(ctx->t_p1, ctx->s_prod));
-        CU_CHECK(ctx, cudaEventRecord(ctx->h_p1[hist], ctx->s_prod));
+        // The GEMM is enqueued first: if anything serialises the two kernels (a profiler, blocking launches, a
+        // GPU whose free SMs do not hold both grids), the GEMM runs to completion, its own CTAs drain every
+        // segment at the end, and the consumer then finds nothing left -- instead of a consumer that waits for
+        // flags nobody can raise.  With both grids resident the order makes no difference.
+        TIME_POINT(ctx->t_p0, ctx->s_prod);
+        TIME_POINT(ctx->h_p0[hist], ctx->s_prod);
+        producer_kernel<<<prod_ctas, PROD_THREADS, PROD_SMEM_BYTES, ctx->s_prod>>>(maps, p, kflags);
+        TIME_POINT(ctx->t_p1, ctx->s_prod);
+        TIME_POINT(ctx->h_p1[hist], ctx->s_prod);
         CU_CHECK(ctx, cudaEventRecord(ctx->ev_prod_done, ctx->s_prod));
+        TIME_POINT(ctx->t_m0, ctx->s_cons);
+        consumer_kernel<<<cons_ctas, MOVER_THREADS, CONSUMER_SMEM_BYTES, ctx->s_cons>>>(p);
+        TIME_POINT(ctx->t_m1, ctx->s_cons);
+        CU_CHECK(ctx, cudaEventRecord(ctx->ev_cons_done, ctx->s_cons));
         CU_CHECK(ctx, cudaStreamWaitEvent(st, ctx->ev_cons_done, 0));
         CU_CHECK(ctx, cudaStreamWaitEvent(st, ctx->ev_prod_done, 0));
+        launches += 2;
     } else {
-        // ---- comparison baseline: the GEMM runs to completion, then a separate scatter kernel
-        CU_CHECK(ctx, cudaEventRecord(ctx->t_p0, st));
-        CU_CHECK(ctx, cudaEventRecord(ctx->h_p0[hist], st));
-        producer_kernel<<<prod_ctas, PROD_THREADS, PROD_SMEM_BYTES, st>>>(maps, p, 0);
-        CU_CHECK(ctx, cudaEventRecord(ctx->t_p1, st));
-        CU_CHECK(ctx, cudaEventRecord(ctx->h_p1[hist], st));
-        CU_CHECK(ctx, cudaEventRecord(ctx->t_m0, st));
-        scatter_kernel<<<ctx->scatter_blocks_per_sm * ctx->num_sms, 256, 0, st>>>(p);
-        CU_CHECK(ctx, cudaEventRecord(ctx->t_m1, st));
+        // ---- one GEMM kernel on every SM.  IN_KERNEL: its spare warps move the finished segments while the
+        //      tensor cores work.  NON_OVERLAP (the comparison baseline): it runs to completion, then a separate
+        //      scatter kernel moves all rows.
+        TIME_POINT(ctx->t_p0, st);
+        TIME_POINT(ctx->h_p0[hist], st);
+        producer_kernel<<<prod_ctas, PROD_THREADS, PROD_SMEM_BYTES, st>>>(maps, p, kflags);
+        ++launches;
+        TIME_POINT(ctx->t_p1, st);
+        TIME_POINT(ctx->h_p1[hist], st);
+        TIME_POINT(ctx->t_m0, st);
+        if (!in_kernel) {
+            scatter_kernel<<<ctx->scatter_blocks_per_sm * ctx->num_sms, 256, 0, st>>>(p);
+            ++launches;
+        }
+        TIME_POINT(ctx->t_m1, st);
     }
-    launches += 2;                               // GEMM + consumer or scatter
     combine_kernel<<<ctx->combine_blocks_per_sm * ctx->num_sms, 256, 0, st>>>(p);
     ++launches;
     CU_CHECK(ctx, cudaGetLastError());
-    CU_CHECK(ctx, cudaEventRecord(ctx->t_end, st));
+    TIME_POINT(ctx->t_end, st);
+#undef TIME_POINT
 
     ctx->last_stream = st;
     ctx->ran = true;
+    ctx->hist_timed[hist] = timed;
     ++ctx->calls;
-    ctx->last_mode = a->mode;
+    ctx->last_timed = timed;
+    ctx->last_mode = mode;
     ctx->last_prod_ctas = prod_ctas;
     ctx->last_cons_ctas = cons_ctas;
     ctx->last_launches = launches;
     ctx->last_rows = p.M;
+    ctx->last_chunks = p.seg_chunks;
     return MOE_OVL_OK;
 }
 
@@ -592,16 +651,20 @@ int moe_ovl_get_report(moe_ovl_ctx *ctx, moe_ovl_report *r)
     r->producer_ctas = ctx->last_prod_ctas;
     r->consumer_ctas = ctx->last_cons_ctas;
     r->kernel_launches = ctx->last_launches;
-    float prod_end = 0.f, mover_end = 0.f;
-    CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_total, ctx->t_begin, ctx->t_end));
-    CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_prep, ctx->t_begin, ctx->t_prep));
-    CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_producer, ctx->t_p0, ctx->t_p1));
-    CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_mover, ctx->t_m0, ctx->t_m1));
-    CU_CHECK(ctx, cudaEventElapsedTime(&prod_end, ctx->t_prep, ctx->t_p1));
-    CU_CHECK(ctx, cudaEventElapsedTime(&mover_end, ctx->t_prep, ctx->t_m1));
-    r->ms_expert_return = std::max(prod_end, mover_end);
-    r->ms_combine = r->ms_total - r->ms_prep - r->ms_expert_return;
-    if (ctx->last_mode == MOE_OVL_MODE_OVERLAP && meta[META_SEGS] > 0) {
+    r->mode_used = ctx->last_mode;
+    r->timing_valid = ctx->last_timed ? 1 : 0;
+    if (ctx->last_timed) {
+        float prod_end = 0.f, mover_end = 0.f;
+        CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_total, ctx->t_begin, ctx->t_end));
+        CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_prep, ctx->t_begin, ctx->t_prep));
+        CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_producer, ctx->t_p0, ctx->t_p1));
+        CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_mover, ctx->t_m0, ctx->t_m1));
+        CU_CHECK(ctx, cudaEventElapsedTime(&prod_end, ctx->t_prep, ctx->t_p1));
+        CU_CHECK(ctx, cudaEventElapsedTime(&mover_end, ctx->t_prep, ctx->t_m1));
+        r->ms_expert_return = std::max(prod_end, mover_end);
+        r->ms_combine = r->ms_total - r->ms_prep - r->ms_expert_return;
+    }
+    if (ctx->last_mode != MOE_OVL_MODE_NON_OVERLAP && meta[META_SEGS] > 0) {
         unsigned long long st[STAMP_COUNT];
         int misc[4];
         CU_CHECK(ctx, cudaMemcpy(st, ctx->ws + ctx->L.stamps, sizeof(st), cudaMemcpyDeviceToHost));
@@ -661,14 +724,17 @@ int moe_ovl_get_gemm_time(moe_ovl_ctx *ctx, int32_t last_n, float *avg_ms, int32
     const int have = (int)std::min<unsigned long long>(ctx->calls, MOE_OVL_TIMING_HISTORY);
     const int n = std::min<int>(last_n, have);
     double sum = 0;
+    int used = 0;
     for (int k = 1; k <= n; ++k) {
         const int i = (int)((ctx->calls - k) % MOE_OVL_TIMING_HISTORY);
+        if (!ctx->hist_timed[i]) continue;          // a captured call: its events carry no time
         float ms = 0.f;
         CU_CHECK(ctx, cudaEventElapsedTime(&ms, ctx->h_p0[i], ctx->h_p1[i]));
         sum += ms;
+        ++used;
     }
-    *avg_ms = n ? (float)(sum / n) : 0.f;
-    if (n_used) *n_used = n;
+    *avg_ms = used ? (float)(sum / used) : 0.f;
+    if (n_used) *n_used = used;
     return MOE_OVL_OK;
 }
 
@@ -702,6 +768,62 @@ int moe_ovl_read_buffer(moe_ovl_ctx *ctx, int32_t which, size_t offset, size_t b
     int rc = sync_last(ctx);
     if (rc != MOE_OVL_OK) return rc;
     if (bytes) CU_CHECK(ctx, cudaMemcpy(host_dst, ctx->ws + base + offset, bytes, cudaMemcpyDeviceToHost));
+    return MOE_OVL_OK;
+}
+
+int moe_ovl_get_trace(moe_ovl_ctx *ctx, void *host_buf, size_t bytes, size_t *written)
+{
+    if (!ctx || !written) return MOE_OVL_ERR_INVALID_ARG;
+    *written = 0;
+    const Layout &L = ctx->L;
+    if (!L.trace_bytes) return MOE_OVL_ERR_UNSUPPORTED;
+    if (!ctx->ran) return MOE_OVL_OK;
+    int rc = sync_last(ctx);
+    if (rc != MOE_OVL_OK) return rc;
+    int meta[META_COUNT];
+    unsigned long long st[STAMP_COUNT];
+    CU_CHECK(ctx, cudaMemcpy(meta, ctx->ws + L.meta, sizeof(meta), cudaMemcpyDeviceToHost));
+    CU_CHECK(ctx, cudaMemcpy(st, ctx->ws + L.stamps, sizeof(st), cudaMemcpyDeviceToHost));
+    const size_t n_items = (size_t)meta[META_ITEMS];
+    const size_t n_units = ctx->last_mode == MOE_OVL_MODE_NON_OVERLAP ? 0 : (size_t)meta[META_SEGS] * ctx->last_chunks;
+    const size_t need = (n_items + n_units) * sizeof(moe_ovl_trace_record);
+    if (!host_buf) { *written = need; return MOE_OVL_OK; }
+    if (bytes < need) return MOE_OVL_ERR_INVALID_ARG;
+    TraceRec *items = new (std::nothrow) TraceRec[n_items + n_units + 1];
+    int *ctas = new (std::nothrow) int[n_items + 1];
+    if (!items || !ctas) { delete[] items; delete[] ctas; return MOE_OVL_ERR_INVALID_ARG; }
+    cudaError_t e = cudaSuccess;
+    if (n_items) e = cudaMemcpy(items, ctx->ws + L.trace_items, n_items * sizeof(TraceRec), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && n_items)
+        e = cudaMemcpy(ctas, ctx->ws + L.trace_item_cta, n_items * 4, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && n_units)
+        e = cudaMemcpy(items + n_items, ctx->ws + L.trace_units, n_units * sizeof(TraceRec), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) {
+        delete[] items; delete[] ctas;
+        ctx->last_cuda_error = (int)e;
+        return MOE_OVL_ERR_CUDA;
+    }
+    const unsigned long long t0 = ~st[STAMP_START_INV];
+    auto rel = [&](unsigned long long t) -> int64_t { return t ? (int64_t)(t - t0) : -1; };
+    moe_ovl_trace_record *out = static_cast<moe_ovl_trace_record *>(host_buf);
+    for (size_t i = 0; i < n_items; ++i) {
+        moe_ovl_trace_record &r = out[i];
+        std::memset(&r, 0, sizeof(r));
+        r.kind = MOE_OVL_TRACE_ITEM; r.index = (int32_t)i; r.cta = ctas[i];
+        r.ns_claim = rel(items[i].a); r.ns_ready = rel(items[i].b);
+        r.ns_done0 = rel(items[i].c); r.ns_done1 = rel(items[i].d);
+    }
+    for (size_t u = 0; u < n_units; ++u) {
+        const TraceRec &t = items[n_items + u];
+        moe_ovl_trace_record &r = out[n_items + u];
+        std::memset(&r, 0, sizeof(r));
+        r.kind = MOE_OVL_TRACE_UNIT; r.index = (int32_t)u; r.cta = (int32_t)(t.a & 0xffffffffu);
+        r.who = (int32_t)(t.a >> 32); r.rows = (int32_t)t.d; r.chunks = ctx->last_chunks;
+        r.ns_claim = r.ns_ready = rel(t.b);
+        r.ns_done0 = r.ns_done1 = rel(t.c);
+    }
+    delete[] items; delete[] ctas;
+    *written = need;
     return MOE_OVL_OK;
 }
 

@@ -33,47 +33,78 @@ __device__ __forceinline__ void copy_rows_16B(const uint16_t *src, uint16_t *dst
     for (; v < nvec; v += nthr) __stcs(d + v, __ldcg(s + v));
 }
 
-// Segment mover shared by the consumer CTAs and by GEMM CTAs that have run out of tiles: claim the next
-// segment in schedule order, wait (bounded, acquire) until every tile of every one of its bands is flagged,
-// then move its valid rows into the owner rank's receive buffer with one contiguous copy.
-// s_seg: two ints of shared memory.  All threads of the CTA must call this together.
-__device__ __forceinline__ void move_segments(const Params &p, volatile int *s_seg, bool gemm_cta)
+// A group of threads that moves segments: a whole CTA (barrier 0) or some warps of a GEMM CTA (their own
+// named barrier).  tid counts inside the group; the group's first warp claims and polls.
+struct MoverGroup {
+    int tid, nthr, bar;
+    int *s_unit;          // two ints of shared memory owned by the group
+    int who;              // TRACE_BY_* of the trace record
+    __device__ __forceinline__ void sync() const
+    {
+        asm volatile("bar.sync %0, %1;" ::"r"(bar), "r"(nthr) : "memory");
+    }
+};
+
+// Segment mover shared by the consumer CTAs, by GEMM CTAs that have run out of tiles and by the spare warps of
+// GEMM CTAs (in-kernel return): claim the next unit in schedule order, wait (bounded, acquire) until every tile
+// of every band of its segment is flagged, then move the unit's valid rows into the owner rank's receive buffer
+// with one contiguous copy.  A unit is one of p.seg_chunks equal row slices of a segment (1 = whole segments,
+// the transfer unit of Section 3.3.2).  All threads of the group must call this together.
+__device__ __forceinline__ void move_segments(const Params &p, const MoverGroup &g)
 {
     const int nseg = p.meta[META_SEGS];
-    const int lane = threadIdx.x & 31;
+    const int chunks = p.seg_chunks;
+    const int nunits = nseg * chunks;
+    const int lane = g.tid & 31;
     const unsigned epoch = *p.epoch;
+    volatile int *s_unit = g.s_unit;
     for (;;) {
-        __syncthreads();
-        if (threadIdx.x < 32) {
-            int s = 0;
-            if (lane == 0) s = atomicAdd(p.next_seg, 1);
-            s = __shfl_sync(0xffffffffu, s, 0);
+        g.sync();
+        if (g.tid < 32) {
+            int u = 0;
+            if (lane == 0) u = atomicAdd(p.next_seg, 1);
+            u = __shfl_sync(0xffffffffu, u, 0);
             bool ok = true;
-            if (s < nseg) {
-                const int4 seg = p.segs[s];          // {first band, bands, dest, rows}
+            if (u < nunits) {
+                const int4 seg = p.segs[u / chunks];          // {first band, bands, dest, rows}
                 const int nflags = seg.y * p.n2;
                 const unsigned *f = p.flags + (size_t)seg.x * p.n2;
                 for (int i = lane; i < nflags && ok; i += 32)
                     ok = wait_global(f + i, epoch, false, p, SITE_CONS_FLAG, (long long)seg.x * p.n2 + i, 2048);
                 ok = __all_sync(0xffffffffu, ok);
             }
-            if (lane == 0) { s_seg[0] = s; s_seg[1] = ok ? 1 : 0; }
+            if (lane == 0) { s_unit[0] = u; s_unit[1] = ok ? 1 : 0; }
         }
-        __syncthreads();
-        const int s = s_seg[0];
-        if (s >= nseg || !s_seg[1]) return;
+        g.sync();
+        const int u = s_unit[0];
+        if (u >= nunits || !s_unit[1]) return;
+        const int s = u / chunks, c = u % chunks;
         const int4 seg = p.segs[s];
+        const int per = (seg.w + chunks - 1) / chunks;         // rows per unit
+        const int r0 = c * per, rows = min(per, seg.w - r0);
+        const long long slot0 = (long long)p.seg_slot0[s] + r0;
         const unsigned long long t_copy = globaltimer_ns();
-        const uint16_t *src = p.Y + (size_t)seg.x * TB_M * p.dout;
-        uint16_t *dst = p.ret + ((size_t)seg.z * p.ret_rows_per_rank + p.seg_slot0[s]) * p.dout;
-        copy_rows_16B(src, dst, (size_t)seg.w * p.dout / 8, threadIdx.x, blockDim.x);
-        __syncthreads();
-        if (threadIdx.x == 0) {
+        // rows that would not fit into the rank's receive region (malformed routing, already reported) stay put
+        if (rows > 0 && slot0 + rows <= p.ret_rows_per_rank) {
+            const uint16_t *src = p.Y + ((size_t)seg.x * TB_M + r0) * p.dout;
+            uint16_t *dst = p.ret + ((size_t)seg.z * p.ret_rows_per_rank + slot0) * p.dout;
+            copy_rows_16B(src, dst, (size_t)rows * p.dout / 8, g.tid, g.nthr);
+        }
+        g.sync();
+        if (g.tid == 0) {
             const unsigned long long now = globaltimer_ns();
             stamp_max(&p.stamps[STAMP_LAST_SEG], now);
-            atomicAdd(&p.stamps[STAMP_COPY_NS], now - t_copy);                       // time one CTA spent copying
-            atomicAdd(&p.stamps[STAMP_COPY_BYTES], (unsigned long long)seg.w * p.dout * 2);
-            if (gemm_cta) atomicAdd(p.assist_segs, 1);
+            atomicAdd(&p.stamps[STAMP_COPY_NS], now - t_copy);                       // time one group spent copying
+            atomicAdd(&p.stamps[STAMP_COPY_BYTES], (unsigned long long)max(rows, 0) * p.dout * 2);
+            if (g.who != TRACE_BY_CONSUMER) atomicAdd(p.assist_segs, 1);
+            if (p.trace_units) {
+                TraceRec rec;
+                rec.a = ((unsigned long long)(unsigned)g.who << 32) | (unsigned)blockIdx.x;
+                rec.b = t_copy;                  // every flag of the segment seen
+                rec.c = now;                     // last row of the unit landed
+                rec.d = (unsigned long long)max(rows, 0);
+                p.trace_units[u] = rec;
+            }
         }
     }
 }
@@ -83,9 +114,10 @@ __device__ __forceinline__ void move_segments(const Params &p, volatile int *s_s
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MOVER_THREADS, 1) consumer_kernel(const Params p)
 {
     extern __shared__ uint8_t unused_smem[];
-    __shared__ int s_seg[2];
+    __shared__ int s_unit[2];
     if (threadIdx.x == 0) p.smid_cons[blockIdx.x] = (int)smid();
-    move_segments(p, s_seg, false);
+    MoverGroup g{(int)threadIdx.x, (int)blockDim.x, 0, s_unit, TRACE_BY_CONSUMER};
+    move_segments(p, g);
 }
 
 // One CTA per (band, chunk of rows): grid-stride over bands x chunks.
@@ -100,6 +132,8 @@ __global__ void __launch_bounds__(256) scatter_kernel(const Params p)
         const int r0 = chunk * rows_per_chunk;
         if (r0 >= valid) continue;
         const int rows = min(rows_per_chunk, valid - r0);
+        // malformed routing can ask for more rows than the region holds: reported by the plan, skipped here
+        if ((long long)p.band_slot0[band] + r0 + rows > p.ret_rows_per_rank) continue;
         const uint16_t *src = p.Y + ((size_t)band * TB_M + r0) * p.dout;
         uint16_t *dst = p.ret + ((size_t)p.band_dest[band] * p.ret_rows_per_rank + p.band_slot0[band] + r0) * p.dout;
         copy_rows_16B(src, dst, (size_t)rows * p.dout / 8, threadIdx.x, blockDim.x);

@@ -168,6 +168,9 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
             acc += n[e * R + r];
         }
         if (p.rows_per_rank_out) p.rows_per_rank_out[r] = acc;
+        // Only malformed routing (a token in more than min(k, El) local experts) can ask for more rows than
+        // the rank's receive region holds.  It is reported here; the copies below skip what does not fit.
+        if (acc > p.ret_rows_per_rank) report_error(p.status, ERR_BAD_ROUTING, SITE_RET_OVERFLOW, r);
     }
     __syncthreads();
     if (tid == 0) {
@@ -361,7 +364,7 @@ __global__ void __launch_bounds__(256) plan_rows_kernel(Params p)
     p.row_at[pos] = i;
     p.slot[i] = slot;
     if (p.slot_out) p.slot_out[i] = slot;
-    if (j < p.kmax) {
+    if (j < p.kmax && slot < p.ret_rows_per_rank) {
         const size_t at = ((size_t)r * p.T + t) * p.kmax + j;
         p.tok_slot[at] = slot + 1;            // 0 (the cleared state) means "no row"
         p.tok_gate[at] = p.gate[i];

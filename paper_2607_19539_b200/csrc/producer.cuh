@@ -48,6 +48,10 @@ constexpr int GATHER_ROWS = 8;                         // rows per gather unit
 constexpr int GATHER_HEAD_ROWS = 2;                    // ... in the first super-band of the schedule
 constexpr int PROD_RING = 16;                          // claimed-item ring; roles are never more than 5 items apart
 constexpr int PROD_TMEM_COLS = 512;
+// kernel flags
+constexpr int PROD_RAISE_FLAGS = 1;    // publish a ready flag per finished output tile; idle CTAs help drain segments
+constexpr int PROD_WARP_MOVERS = 2;    // in-kernel return: the gather warps move finished segments once Xa is complete
+constexpr int PROD_SKIP_FIRST_BAND = 4; // test hook: the first band of the schedule is never gathered
 constexpr int PROD_SMEM_BYTES = PROD_STAGES * PROD_STAGE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers, ring*/;
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -288,8 +292,10 @@ struct ProducerMaps {
 };
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PROD_THREADS, 1)
-producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const int raise_flags)
+producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const int kflags)
 {
+    const bool raise_flags = (kflags & PROD_RAISE_FLAGS) != 0;
+    const bool warp_movers = (kflags & PROD_WARP_MOVERS) != 0;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bars = smem_base + PROD_STAGES * PROD_STAGE_BYTES;
@@ -300,6 +306,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
     const uint32_t bar_go = tmem_slot + 8;                         // TMA thread -> scheduler: "started an item"
     const uint32_t bar_ring = bar_go + 8;                          // PROD_RING barriers: slot filled
     const uint32_t ring = bar_ring + 8 * PROD_RING;                // PROD_RING claimed item indices
+    const uint32_t mover_ints = ring + 4 * PROD_RING;              // two ints of the in-kernel movers
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     volatile uint32_t *tmem_slot_gen = reinterpret_cast<volatile uint32_t *>(smem_gen + (tmem_slot - smem_base));
     volatile int *ring_gen = reinterpret_cast<volatile int *>(smem_gen + (ring - smem_base));
@@ -433,6 +440,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 for (int ks = 0; ks < ksteps; ++ks) {
                     ok = mbar_wait(bar_full + 8 * stage, phase, p, SITE_MMA_FULL, it);
                     if (!ok) break;
+                    if (ks == 0 && p.trace_items) p.trace_items[it].b = globaltimer_ns();
                     tc_fence_after();
                     const uint32_t sa = smem_base + stage * PROD_STAGE_BYTES, sb = sa + PROD_A_BYTES;
                     const uint64_t adesc = umma_smem_desc(sa), bdesc = umma_smem_desc(sb);
@@ -462,6 +470,10 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 // latency is hidden and no role can fall a whole ring behind
                 if (n >= 1 && !mbar_wait(bar_go, (uint32_t)(n - 1) & 1u, p, SITE_SCHED_GO, n)) break;
                 const int it = atomicAdd(p.next_item, 1);
+                if (p.trace_items && it < n_items) {
+                    p.trace_items[it].a = globaltimer_ns();
+                    p.trace_item_cta[it] = (int)blockIdx.x;
+                }
                 const int slot = n % PROD_RING;
                 ring_gen[slot] = it;
                 asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_ring + 4 * slot), "r"(it) : "memory");
@@ -487,7 +499,9 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
         while (unit < nunits) {
             int next = 0;
             if (lane == 0) next = atomicAdd(p.next_gather, 1);      // claimed while this unit's rows are moving
-            if (unit < head_units) {
+            if ((kflags & PROD_SKIP_FIRST_BAND) && unit < TB_M / GATHER_HEAD_ROWS) {
+                // test hook: leave band 0 of the schedule ungathered, so that the wait for it runs out
+            } else if (unit < head_units) {
                 const int per = TB_M / GATHER_HEAD_ROWS;
                 gather_unit<GATHER_HEAD_ROWS, 16 / GATHER_HEAD_ROWS>(p, p.sched_band[unit / per],
                                                                      (unit % per) * GATHER_HEAD_ROWS, lane);
@@ -497,6 +511,14 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                                                            (u % per) * GATHER_ROWS, lane);
             }
             unit = __shfl_sync(0xffffffffu, next, 0);
+        }
+        // In-kernel return: with Xa complete these warps have nothing left to do, so they take over the
+        // consumer's job on this SM -- no SM is taken from the GEMM.  They only ever wait on tile flags, which
+        // the epilogue warps raise without waiting on anybody.
+        if (warp_movers) {
+            MoverGroup g{(int)threadIdx.x - 224, 32 * PROD_GATHER_WARPS, 3,
+                         reinterpret_cast<int *>(smem_gen + (mover_ints - smem_base)), TRACE_BY_GEMM_WARPS};
+            move_segments(p, g);
         }
     } else {
         // ---------------- epilogue: warps 2..5 own tensor-memory lanes 32*(warp % 4) .. +31
@@ -566,6 +588,11 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             __threadfence();
             if (kind == KIND_G1) asm volatile("fence.proxy.async;" ::: "memory");   // H is re-read through TMA
             bar_sync_epilogue();
+            if (leader && present && p.trace_items) {
+                // taken before the release below, so that no observer of the flag can carry an earlier time
+                const unsigned long long now = globaltimer_ns();
+                if (rank == 0) p.trace_items[it].c = now; else p.trace_items[it].d = now;
+            }
             if (leader && present) {
                 if (kind == KIND_G1) red_release_add_u32(&p.hcount[band], 1u);
                 else if (raise_flags) {
@@ -590,7 +617,10 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
     }
     // Out of tiles: help the consumer drain what is left, so that the last segments do not wait for the few
     // consumer SMs (the tail Section 3.3.3 warns about when the consumer budget is small).
-    if (raise_flags) move_segments(p, reinterpret_cast<volatile int *>(smem_gen), true);
+    if (raise_flags) {
+        MoverGroup g{(int)threadIdx.x, (int)blockDim.x, 0, reinterpret_cast<int *>(smem_gen), TRACE_BY_GEMM_TAIL};
+        move_segments(p, g);
+    }
 }
 
 }  // namespace moe_ovl

@@ -5,7 +5,19 @@ from oracle import value_oracle as VO
 from oracle.index_oracle import build_plan
 from paper_2607_19539_b200 import inputs as I
 
-TOL_REL = 2e-2   # max relative distance on values (bf16 output, fp32 accumulate), stated by the benchmark spec
+TOL_REL = 2e-2    # max relative error on values (bf16 output, fp32 accumulate), stated by the benchmark spec: asserted
+                  # element by element as |a - b| <= TOL_REL * (|b| + rms of b's row)
+TOL_NORM = 5e-3   # per-token 2-norm distance: what the rounding model supports (both sides round H, Y and out to
+                  # bf16 at the same points; they differ where fp32 summation order flips a rounding, one bf16
+                  # ulp = 2^-8..2^-7 relative on a fraction of the elements)
+
+
+def elem_err(a, b):
+    """Element-wise |a - b| / (|b| + rms(b_row)), float64; rows of zeros must match exactly."""
+    a = a.astype(np.float64)
+    b = b.astype(np.float64)
+    rms = np.sqrt((b * b).mean(axis=-1, keepdims=True))
+    return np.abs(a - b) / (np.abs(b) + rms + 1e-300)
 
 
 def rel_dist(a, b):
@@ -91,23 +103,46 @@ def oracle_values(inp, tokens):
 
 
 def check_values(shape, dsp, plan, tokens, o_out, o_y, o_yexp, gpu_out_bits, gpu_ret_bits):
-    """out and the returned rows of the given tokens against the oracle, within TOL_REL."""
+    """out and the returned rows of the given tokens against the oracle: every element within TOL_REL of
+    (|b| + rms of its row), every row within TOL_NORM in the 2-norm."""
     tokens = np.asarray(tokens)
     got = I.bf16_bits_to_f32(gpu_out_bits[tokens])
     ref = I.bf16_bits_to_f32(o_out)
     none = (o_yexp < 0).all(axis=1)
     assert (gpu_out_bits[tokens][none] == 0).all()                 # no local expert: +0
-    worst = float(rel_dist(got[~none], ref[~none]).max()) if (~none).any() else 0.0
-    assert worst <= TOL_REL, worst
+    worst = worst_el = 0.0
+    if (~none).any():
+        worst = float(rel_dist(got[~none], ref[~none]).max())
+        worst_el = float(elem_err(got[~none], ref[~none]).max())
+    assert worst <= TOL_NORM, worst
+    assert worst_el <= TOL_REL, worst_el
     # returned rows: ret[r][slot] holds the unscaled expert output of that (token, expert)
-    worst_y = 0.0
-    for s, tok in enumerate(tokens.tolist()):
-        r = tok // shape.T
-        slots = plan.tok_slot[tok]
-        assert len(slots) == int((o_yexp[s] >= 0).sum())
-        for j, slot in enumerate(slots):
-            a = I.bf16_bits_to_f32(gpu_ret_bits[r, slot])[None]
-            b = I.bf16_bits_to_f32(o_y[s, j])[None]
-            worst_y = max(worst_y, float(rel_dist(a, b)[0]))
-    assert worst_y <= TOL_REL, worst_y
-    return worst, worst_y
+    kmax = o_yexp.shape[1]
+    nrows = np.asarray([len(plan.tok_slot[t]) for t in tokens.tolist()])
+    assert (nrows == (o_yexp >= 0).sum(axis=1)).all()
+    slot = np.full((len(tokens), kmax), -1, np.int64)
+    for s, t in enumerate(tokens.tolist()):
+        slot[s, :nrows[s]] = plan.tok_slot[t]
+    si, ji = np.nonzero(slot >= 0)
+    worst_y = worst_y_el = 0.0
+    step = 4096
+    for lo in range(0, len(si), step):
+        s_, j_ = si[lo:lo + step], ji[lo:lo + step]
+        a = I.bf16_bits_to_f32(gpu_ret_bits[tokens[s_] // shape.T, slot[s_, j_]])
+        b = I.bf16_bits_to_f32(o_y[s_, j_])
+        worst_y = max(worst_y, float(rel_dist(a, b).max()))
+        worst_y_el = max(worst_y_el, float(elem_err(a, b).max()))
+    assert worst_y <= TOL_NORM, worst_y
+    assert worst_y_el <= TOL_REL, worst_y_el
+    return worst, worst_y, worst_el, worst_y_el
+
+
+def check_aligned_input(shape, dsp, plan, xa_bits):
+    """The gather into the aligned layout (Section 3.2.1): Xa[pos[i]] is input row i, bit for bit, and every
+    other position of the padded buffer is zero."""
+    pos = np.asarray(plan.pos)
+    assert xa_bits.shape[0] == plan.P
+    assert (xa_bits[pos] == dsp.x_rows).all()
+    pad = np.ones(plan.P, bool)
+    pad[pos] = False
+    assert (xa_bits[pad] == 0).all()

@@ -34,11 +34,11 @@ SMALL = ["tiny", "tiny_zipf", "small", "small_zipf_rot", "single_small", "many_g
 
 
 @pytest.mark.parametrize("name", SMALL)
-@pytest.mark.parametrize("mode,csm", [(0, 2), (0, 8), (0, 32), (1, 0)])
+@pytest.mark.parametrize("mode,csm", [(0, 2), (0, 8), (0, 32), (1, 0), (2, 0), (3, 0)])
 def test_small_shapes_full_parity(name, mode, csm):
     torch, B, Hn = _gpu()
     shape = I.SHAPES[name]
-    inp, dsp, ctx, prob = _run_case(shape, mode, csm, shuffle=None if mode else 17)
+    inp, dsp, ctx, prob = _run_case(shape, mode, csm, shuffle=None if mode == 1 else 17)
     plan = U.oracle_plan(shape, dsp)
     U.check_indices(shape, dsp, plan, ctx.moe_ovl_get_plan(), prob.slot_out.cpu().numpy(),
                     prob.rows_per_rank_out.cpu().numpy(), prob.segs_per_rank_out.cpu().numpy(),
@@ -47,6 +47,7 @@ def test_small_shapes_full_parity(name, mode, csm):
     o_out, o_y, o_yexp = U.oracle_values(inp, toks)
     U.check_values(shape, dsp, plan, toks, o_out, o_y, o_yexp, Hn.device_to_bits(prob.out),
                    Hn.device_to_bits(prob.ret))
+    U.check_aligned_input(shape, dsp, plan, ctx.moe_ovl_read_buffer(B.BUF_XA, 0, plan.P))
     # rows of ret beyond rows_per_rank are untouched (still the NaN fill of the harness)
     ret = prob.ret.float().cpu().numpy()
     for r in range(shape.R):
@@ -89,12 +90,12 @@ def test_overlap_equals_non_overlap_bitwise(name):
         torch.cuda.synchronize()
         refs.append((base, base.out.clone(), base.ret.clone()))
     assert not torch.equal(refs[0][1].view(torch.int16), refs[1][1].view(torch.int16))
-    for it in range(24):
-        csm = (2, 4, 8, 16, 32)[it % 5]
+    for it in range(30):
+        csm = (2, 4, 8, 16, 32, 0)[it % 6]                      # 0: the return moved inside the GEMM kernel
         inp, dsp = probs[it % 2]
         base, ref_out, ref_ret = refs[it % 2]
         prob = Hn.upload(inp, dsp, w1=base.w1, w2=base.w2)
-        Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=csm)
+        Hn.run(ctx, prob, mode=B.MODE_OVERLAP if csm else B.MODE_IN_KERNEL, consumer_sm_count=csm)
         torch.cuda.synchronize()
         assert ctx.moe_ovl_query_status()[0] == 0
         assert torch.equal(prob.out.view(torch.int16), ref_out.view(torch.int16))
@@ -340,7 +341,7 @@ def test_random_shapes_full_parity(seed):
                        N_out=int(rng.choice([256, 768])) if single else 0,
                        router=str(rng.choice(["uniform", "zipf", "zipf_rot"])), seed=seed,
                        self_rank=int(rng.integers(0, R)), first_local=int(rng.integers(0, groups)) * El)
-    mode = B.MODE_NON_OVERLAP if seed % 5 == 4 else B.MODE_OVERLAP
+    mode = (B.MODE_OVERLAP, B.MODE_IN_KERNEL, B.MODE_OVERLAP, B.MODE_AUTO, B.MODE_NON_OVERLAP)[seed % 5]
     csm = int(rng.choice([0, 1, 2, 6, 24]))
     mgb = int(rng.integers(1, 4))
     gb = int(rng.choice([0, 2, 4, 5, 64]))
@@ -393,3 +394,171 @@ def test_call_can_be_captured_in_a_cuda_graph_and_replayed():
         torch.cuda.synchronize()
         assert torch.equal(prob.out.view(torch.int16), ref.out.view(torch.int16)), scale
         assert torch.equal(prob.ret.view(torch.int16), ref.ret.view(torch.int16)), scale
+    # a captured call records no timing events: the report says so instead of failing, the plan sizes and the
+    # device stamps of the last replay are still there, and the GEMM-time average skips the captured call
+    rep = ctx.moe_ovl_get_report()
+    assert rep.timing_valid == 0 and rep.ms_total == 0.0 and rep.ms_producer == 0.0
+    assert rep.num_bands > 0 and rep.us_return_done > 0.0
+    ms, n = ctx.moe_ovl_get_gemm_time(1)
+    assert n == 0 and ms == 0.0
+    ms, n = ctx.moe_ovl_get_gemm_time(2)          # the warm-up call before the capture was timed
+    assert n == 1 and ms > 0.0
+
+
+@pytest.mark.parametrize("mode,csm", [(0, 4), (2, 0), (1, 0)])
+def test_trace_records_every_item_and_unit(mode, csm):
+    """The device trace: one record per schedule item (claimed <= first operands landed <= published) and one
+    per moved unit of the return; a segment is never seen ready before the last of its tiles was published."""
+    torch, B, Hn = _gpu()
+    shape = I.SHAPES["small_zipf_rot"]
+    inp = I.make_inputs(shape)
+    dsp = I.dispatch(inp)
+    ctx = Hn.make_context(shape, max_rows=dsp.M, flags=B.FLAG_TRACE)
+    prob = Hn.upload(inp, dsp)
+    for _ in range(2):                                   # the second call must not see the first call's records
+        Hn.run(ctx, prob, mode=mode, consumer_sm_count=csm)
+        torch.cuda.synchronize()
+        assert ctx.moe_ovl_query_status()[0] == 0
+    rep = ctx.moe_ovl_get_report()
+    plan = ctx.moe_ovl_get_plan()
+    tr = ctx.moe_ovl_get_trace()
+    items, units = tr[tr["kind"] == B.TRACE_ITEM], tr[tr["kind"] == B.TRACE_UNIT]
+    assert len(items) == rep.num_items and items["index"].tolist() == list(range(rep.num_items))
+    assert (items["ns_claim"] >= 0).all()
+    assert (items["ns_claim"] <= items["ns_ready"]).all() and (items["ns_ready"] <= items["ns_done0"]).all()
+    second = plan["item"][:, 2] >= 0                     # the pair's second band exists
+    assert (items["ns_done1"][second] >= items["ns_ready"][second]).all() and (items["ns_done1"][~second] == -1).all()
+    assert (items["cta"] % 2 == 0).all() and items["cta"].max() < rep.producer_ctas
+    # claims are handed out in issue order (each pair stamps its own claim, hence the slack)
+    assert (np.diff(items["ns_claim"]) >= -5000).all()
+    if mode == B.MODE_NON_OVERLAP:
+        assert len(units) == 0
+        return
+    chunks = 1 if mode == B.MODE_OVERLAP else 8
+    assert len(units) == rep.num_segments * chunks and (units["chunks"] == chunks).all()
+    assert (units["who"] == 2).all() if mode == B.MODE_IN_KERNEL else set(units["who"].tolist()) <= {0, 1}
+    assert (units["ns_done0"] >= units["ns_claim"]).all()
+    seg_rows = plan["seg"][:, 3]
+    assert units["rows"].reshape(-1, chunks).sum(axis=1).tolist() == seg_rows.tolist()
+    # latest publication time of any output tile of each band (second-GEMM items only)
+    n_bands = rep.num_bands
+    band_done = np.zeros(n_bands, np.int64)
+    for (x, b0, b1, _tile), rec in zip(plan["item"].tolist(), items):
+        if x & 0xff == 1:
+            band_done[b0] = max(band_done[b0], rec["ns_done0"])
+            if b1 >= 0:
+                band_done[b1] = max(band_done[b1], rec["ns_done1"])
+    for u, rec in enumerate(units):
+        first, nb = plan["seg"][u // chunks, 0], plan["seg"][u // chunks, 1]
+        assert rec["ns_claim"] >= band_done[first:first + nb].max()
+    assert abs(rep.us_return_done * 1e3 - units["ns_done0"].max()) < 2e3
+
+
+def test_trace_is_refused_without_the_flag():
+    torch, B, Hn = _gpu()
+    shape = I.SHAPES["tiny"]
+    inp, dsp, ctx, prob = _run_case(shape, 0, 2)
+    with pytest.raises(B.MoeOvlError) as e:
+        ctx.moe_ovl_get_trace()
+    assert e.value.code == B.ERR_UNSUPPORTED
+
+
+def test_serialised_kernels_degrade_instead_of_timing_out():
+    """With launches made blocking the two kernels of the overlap mode cannot run side by side.  The GEMM is
+    enqueued first, so it runs to completion, its own CTAs move every segment, and the consumer finds nothing
+    left: the call succeeds (a profiler that serialises kernels sees the same)."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    child = r"""
+import sys
+sys.path.insert(0, %r)
+import numpy as np, torch
+from paper_2607_19539_b200 import binding as B, harness as Hn, inputs as I
+shape = I.SHAPES["tiny"]
+inp = I.make_inputs(shape); dsp = I.dispatch(inp)
+ctx = Hn.make_context(shape, max_rows=dsp.M, wait_timeout_us=50_000)
+ref = Hn.upload(inp, dsp)
+Hn.run(ctx, ref, mode=B.MODE_NON_OVERLAP); torch.cuda.synchronize()
+for csm in (2, 8):
+    prob = Hn.upload(inp, dsp, w1=ref.w1, w2=ref.w2)
+    Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=csm); torch.cuda.synchronize()
+    code, detail = ctx.moe_ovl_query_status()
+    assert code == 0, (code, hex(detail))
+    assert torch.equal(prob.out.view(torch.int16), ref.out.view(torch.int16))
+    assert torch.equal(prob.ret.view(torch.int16), ref.ret.view(torch.int16))
+    assert ctx.moe_ovl_get_report().segments_by_gemm_ctas == ctx.moe_ovl_get_report().num_segments
+print("serialised ok")
+""" % root
+    env = dict(os.environ, CUDA_LAUNCH_BLOCKING="1")
+    r = subprocess.run([sys.executable, "-c", child], env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and "serialised ok" in r.stdout, r.stdout + r.stderr
+
+
+def test_gemm_kernel_gives_up_cleanly_when_its_input_never_arrives():
+    """The bounded waits inside the GEMM kernel: a test hook leaves the first band of the schedule ungathered, so
+    the load warp's wait for it runs out.  The kernel must report the timeout, let its copies land, free its
+    tensor memory and return; the context and the device stay usable."""
+    torch, B, Hn = _gpu()
+    shape = I.SHAPES["small"]
+    inp = I.make_inputs(shape)
+    dsp = I.dispatch(inp)
+    ctx = Hn.make_context(shape, max_rows=dsp.M, wait_timeout_us=20_000, flags=B.FLAG_TEST_SKIP_GATHER)
+    prob = Hn.upload(inp, dsp)
+    for mode, csm in ((B.MODE_NON_OVERLAP, 0), (B.MODE_OVERLAP, 4), (B.MODE_IN_KERNEL, 0)):
+        Hn.run(ctx, prob, mode=mode, consumer_sm_count=csm)
+        torch.cuda.synchronize()
+        code, detail = ctx.moe_ovl_query_status()
+        assert code == B.ERR_TIMEOUT, (mode, code)
+        # the wait that gave up: the load warp waiting for gathered rows (11); with a mover polling flags at
+        # the same time, its wait (6) may run out a few microseconds earlier
+        assert detail >> 48 in ((11,) if mode == B.MODE_NON_OVERLAP else (11, 6)), hex(detail)
+    ok = Hn.make_context(shape, max_rows=dsp.M)
+    ref = Hn.upload(inp, dsp, w1=prob.w1, w2=prob.w2)
+    Hn.run(ok, ref, mode=B.MODE_NON_OVERLAP)
+    prob2 = Hn.upload(inp, dsp, w1=prob.w1, w2=prob.w2)
+    Hn.run(ok, prob2, mode=B.MODE_OVERLAP, consumer_sm_count=4)
+    torch.cuda.synchronize()
+    assert ok.moe_ovl_query_status()[0] == 0
+    assert torch.equal(prob2.out.view(torch.int16), ref.out.view(torch.int16))
+    plan = U.oracle_plan(shape, dsp)
+    assert prob2.slot_out.cpu().numpy()[:dsp.M].tolist() == plan.slot
+
+
+def test_rows_beyond_the_receive_region_are_reported_and_never_written():
+    """Malformed routing with more local experts than top-k: every token is routed to all three local experts, so
+    a rank would need 3T receive rows where the region holds min(k, El) * T = 2T.  The call must report bad
+    routing and write nothing outside the regions: the receive buffer is over-allocated with a canary tail, so
+    that even an unguarded write would stay in owned memory."""
+    torch, B, Hn = _gpu()
+    shape = I.MoEShape("overflow", R=2, T=200, Eg=6, k=2, El=3, d=256, F=128, seed=11)
+    inp = I.make_inputs(shape)
+    T, R, El, d = shape.T, shape.R, shape.El, shape.d
+    M = El * R * T
+    rng = np.random.Generator(np.random.PCG64(5))
+    rows = I.f32_to_bf16_bits(rng.standard_normal((M, d), dtype=np.float32))
+    r_idx = np.tile(np.repeat(np.arange(R, dtype=np.int32), T), El)
+    t_idx = np.tile(np.arange(T, dtype=np.int32), El * R)
+    bad = I.Dispatched(rows, np.full(El, R * T, np.int32), r_idx, t_idx, np.full(M, 0.5, np.float32),
+                       np.repeat(np.arange(El, dtype=np.int32), R * T))
+    ctx = Hn.make_context(shape, max_rows=M)
+    prob = Hn.upload(inp, bad)
+    region = T * shape.kmax
+    big = torch.full((R * El * T + 64, d), float("nan"), dtype=torch.bfloat16, device="cuda:0")
+    for mode, csm in ((B.MODE_NON_OVERLAP, 0), (B.MODE_OVERLAP, 4), (B.MODE_IN_KERNEL, 0)):
+        big.fill_(float("nan"))
+        ctx.moe_ovl_expert_return(x=prob.x, expert_counts=prob.expert_counts, src_rank=prob.src_rank,
+                                  src_token=prob.src_token, gate=prob.gate, w1=prob.w1, w2=prob.w2,
+                                  ret=big[:R * region].view(R, region, d), out=prob.out, consumer_sm_count=csm,
+                                  mode=mode, num_rows=M)
+        torch.cuda.synchronize()
+        code, detail = ctx.moe_ovl_query_status()
+        assert code == B.ERR_BAD_ROUTING, (mode, code)
+        assert torch.isnan(big[R * region:].float()).all()           # nothing past the last rank's region
+    # the context stays usable with well-formed routing
+    dsp = I.dispatch(inp)
+    good = Hn.upload(inp, dsp, w1=prob.w1, w2=prob.w2)
+    Hn.run(ctx, good, mode=B.MODE_OVERLAP, consumer_sm_count=4)
+    torch.cuda.synchronize()
+    assert ctx.moe_ovl_query_status()[0] == 0

@@ -11,6 +11,8 @@ import pytest
 
 from paper_2607_19539_b200 import inputs as I
 
+from .parity_util import oracle_plan
+
 pytestmark = pytest.mark.gpu
 
 
@@ -49,6 +51,50 @@ def test_static_scratch_entry_point_matches_workspace_entry_point():
             torch.cuda.synchronize()
             assert torch.equal(slot, want_slot)          # integer work: bit-exact
             assert torch.equal(rows, want_rows)
+            # and against the CPU oracle's plan, which shares nothing with either entry point
+            plan = oracle_plan(shape, dsp)
+            assert slot.cpu().tolist() == plan.slot and rows.cpu().tolist() == plan.rows_per_rank
+
+
+def test_static_scratch_entry_point_edge_cases():
+    """No rows at all; no rows-per-rank output wanted; rows the metadata does not cover get slot -1."""
+    import torch
+    from paper_2607_19539_b200 import binding as B
+    dev = torch.device("cuda:0")
+    shape = I.SHAPES["tiny"]
+    dsp = I.dispatch(I.make_inputs(shape, weights=False))
+    common = dict(device=0, num_src_ranks=shape.R, tokens_per_rank=shape.T, num_local_experts=shape.El)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, np.int32)).to(dev)
+    # (a) M = 0
+    rows = torch.full((shape.R,), -9, dtype=torch.int32, device=dev)
+    empty = torch.zeros(0, dtype=torch.int32, device=dev)
+    B.moe_ovl_return_slots_static(expert_counts=i32(np.zeros(shape.El)), src_rank=empty, src_token=empty,
+                                  slot_out=empty, rows_per_rank_out=rows, **common)
+    torch.cuda.synchronize()
+    assert rows.tolist() == [0] * shape.R
+    # (b) rows_per_rank_out = NULL, right after a call that left the array full of another problem's bits
+    plan = oracle_plan(shape, dsp)
+    slot = torch.full((dsp.M,), -9, dtype=torch.int32, device=dev)
+    B.moe_ovl_return_slots_static(expert_counts=i32(dsp.expert_counts), src_rank=i32(dsp.src_rank),
+                                  src_token=i32(dsp.src_token), slot_out=slot, rows_per_rank_out=None, **common)
+    torch.cuda.synchronize()
+    assert slot.cpu().tolist() == plan.slot
+    # (c) one row with an out-of-range rank, and counts that cover one row fewer than passed: both get -1,
+    #     every other row keeps the slot it has without them
+    sr = dsp.src_rank.copy()
+    sr[3] = shape.R
+    counts = dsp.expert_counts.copy()
+    counts[-1] -= 1
+    keep = np.ones(dsp.M, bool)
+    keep[3] = keep[-1] = False
+    sub = I.Dispatched(dsp.x_rows[keep], np.bincount(dsp.row_expert[keep], minlength=shape.El).astype(np.int32),
+                       dsp.src_rank[keep], dsp.src_token[keep], dsp.gate[keep], dsp.row_expert[keep])
+    want = np.full(dsp.M, -1, np.int64)
+    want[keep] = oracle_plan(shape, sub).slot
+    B.moe_ovl_return_slots_static(expert_counts=i32(counts), src_rank=i32(sr), src_token=i32(dsp.src_token),
+                                  slot_out=slot, rows_per_rank_out=rows, **common)
+    torch.cuda.synchronize()
+    assert slot.cpu().tolist() == want.tolist()
 
 
 def test_static_scratch_limits_are_rejected():
