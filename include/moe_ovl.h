@@ -275,6 +275,13 @@ typedef struct {
     int64_t ns_done0;  /* item: tile of the pair's first band published (flag or band counter), taken just
                           before the release store; unit: last row landed in the receive buffer */
     int64_t ns_done1;  /* item: same for the pair's second band, -1 if absent; unit: same as ns_done0 */
+    int64_t ns_operand_wait; /* item: time the MMA-issuing thread spent waiting for operand stages after the
+                          item's first stage (pipeline stalls, not start-up); unit: 0 */
+    int64_t ns_epilogue_start;     /* item: the epilogue warps of the pair's first CTA saw the finished accumulator */
+    int64_t ns_first_operand_wait; /* item: time the MMA-issuing thread waited for the item's first operand stage
+                                      (the bubble between two items, or the kernel's start-up) */
+    int64_t ns_accumulator_wait;   /* item: time it waited for a free accumulator buffer, i.e. for the epilogue of
+                                      the item before the previous one: non-zero means the epilogue is the bound */
 } moe_ovl_trace_record;
 /* Waits for the last call, then writes its records to HOST memory: items in issue order, then units in
  * claim order.  *written = bytes written.  host_buf == NULL: only reports the bytes needed.

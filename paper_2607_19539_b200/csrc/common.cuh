@@ -93,10 +93,12 @@ struct Params {
     unsigned *flags;      // [max_bands*n2] epoch of the call that finished the tile
     int *meta;            // [META_COUNT]
     // optional trace (null when off), raw %globaltimer values: one record per schedule item {claimed, first
-    // operands landed, published by CTA 0 of the pair, published by CTA 1} plus the leader CTA's index, and
+    // operands landed, published by CTA 0 of the pair, published by CTA 1} plus trace_item_aux, and
     // one per moved unit {who << 32 | CTA, flags seen, copy done, rows}
     TraceRec *trace_items, *trace_units;
-    int *trace_item_cta;
+    int2 *trace_item_aux;   // {leader CTA, ns the MMA-issuing thread waited for operand stages during the item}
+    TraceRec *trace_items2; // {epilogue of CTA 0 saw the accumulator, ns the MMA thread waited for the item's first
+                            //  stage, ns it waited for a free accumulator, unused}
     int *status;          // [ST_COUNT]
 };
 

@@ -35,7 +35,7 @@ struct Layout {
     size_t wordpfx, group_rows, group_start, group_slot, pos, slot, row_at, xready;
     size_t band_expert, band_dest, band_valid, band_slot0, sched_band, items, segs, seg_slot0;
     size_t tok_gate, flags, meta;
-    size_t trace_items, trace_units, trace_item_cta, trace_bytes;   // MOE_OVL_FLAG_TRACE
+    size_t trace_items, trace_items2, trace_units, trace_item_aux, trace_bytes;   // MOE_OVL_FLAG_TRACE
     size_t sb[6];
     // host staging (MOE_OVL_FLAG_HOST_STAGING)
     size_t st_x[2], st_counts[2], st_rank[2], st_token[2], st_gate[2], st_out[2], st_ret;   // two staging slots
@@ -125,8 +125,9 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->trace_bytes = 0;
     if (c->flags & MOE_OVL_FLAG_TRACE) {
         L->trace_items = take((size_t)L->max_items * sizeof(TraceRec));
+        L->trace_items2 = take((size_t)L->max_items * sizeof(TraceRec));
         L->trace_units = take((size_t)L->max_bands * MAX_SEG_CHUNKS * sizeof(TraceRec));
-        L->trace_item_cta = take((size_t)L->max_items * 4);
+        L->trace_item_aux = take((size_t)L->max_items * 8);
         L->trace_bytes = off - L->trace_items;
     }
     if (c->flags & MOE_OVL_FLAG_HOST_STAGING) {
@@ -243,7 +244,8 @@ Params make_params(moe_ovl_ctx *ctx)
     if (c.flags & MOE_OVL_FLAG_TRACE) {
         p.trace_items = at<TraceRec>(ctx, L.trace_items);
         p.trace_units = at<TraceRec>(ctx, L.trace_units);
-        p.trace_item_cta = at<int>(ctx, L.trace_item_cta);
+        p.trace_items2 = at<TraceRec>(ctx, L.trace_items2);
+        p.trace_item_aux = at<int2>(ctx, L.trace_item_aux);
     }
     return p;
 }
@@ -789,13 +791,16 @@ int moe_ovl_get_trace(moe_ovl_ctx *ctx, void *host_buf, size_t bytes, size_t *wr
     const size_t need = (n_items + n_units) * sizeof(moe_ovl_trace_record);
     if (!host_buf) { *written = need; return MOE_OVL_OK; }
     if (bytes < need) return MOE_OVL_ERR_INVALID_ARG;
-    TraceRec *items = new (std::nothrow) TraceRec[n_items + n_units + 1];
-    int *ctas = new (std::nothrow) int[n_items + 1];
+    TraceRec *items = new (std::nothrow) TraceRec[2 * n_items + n_units + 1];
+    TraceRec *items2 = items ? items + n_items + n_units : nullptr;
+    int2 *ctas = new (std::nothrow) int2[n_items + 1];
     if (!items || !ctas) { delete[] items; delete[] ctas; return MOE_OVL_ERR_INVALID_ARG; }
     cudaError_t e = cudaSuccess;
     if (n_items) e = cudaMemcpy(items, ctx->ws + L.trace_items, n_items * sizeof(TraceRec), cudaMemcpyDeviceToHost);
     if (e == cudaSuccess && n_items)
-        e = cudaMemcpy(ctas, ctx->ws + L.trace_item_cta, n_items * 4, cudaMemcpyDeviceToHost);
+        e = cudaMemcpy(ctas, ctx->ws + L.trace_item_aux, n_items * 8, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && n_items)
+        e = cudaMemcpy(items2, ctx->ws + L.trace_items2, n_items * sizeof(TraceRec), cudaMemcpyDeviceToHost);
     if (e == cudaSuccess && n_units)
         e = cudaMemcpy(items + n_items, ctx->ws + L.trace_units, n_units * sizeof(TraceRec), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) {
@@ -809,9 +814,12 @@ int moe_ovl_get_trace(moe_ovl_ctx *ctx, void *host_buf, size_t bytes, size_t *wr
     for (size_t i = 0; i < n_items; ++i) {
         moe_ovl_trace_record &r = out[i];
         std::memset(&r, 0, sizeof(r));
-        r.kind = MOE_OVL_TRACE_ITEM; r.index = (int32_t)i; r.cta = ctas[i];
+        r.kind = MOE_OVL_TRACE_ITEM; r.index = (int32_t)i; r.cta = ctas[i].x; r.ns_operand_wait = ctas[i].y;
         r.ns_claim = rel(items[i].a); r.ns_ready = rel(items[i].b);
         r.ns_done0 = rel(items[i].c); r.ns_done1 = rel(items[i].d);
+        r.ns_epilogue_start = rel(items2[i].a);
+        r.ns_first_operand_wait = (int64_t)items2[i].b;
+        r.ns_accumulator_wait = (int64_t)items2[i].c;
     }
     for (size_t u = 0; u < n_units; ++u) {
         const TraceRec &t = items[n_items + u];

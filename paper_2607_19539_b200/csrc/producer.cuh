@@ -82,6 +82,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
+// Non-blocking probe of a phase (try_wait may suspend the thread for a while before it answers).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // Same test with acquire semantics at cluster scope: for barriers the peer CTA arrives on.
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
 {
@@ -433,12 +446,27 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 if (it < 0 || it >= n_items) break;
                 const int kind = p.items[it].x & 0xff;
                 const int ksteps = (kind == KIND_G1 ? p.d : p.k2) / TB_K;
-                ok = mbar_wait<true>(bar_tempty + 8 * acc, acc_phase ^ 1u, p, SITE_MMA_TEMPTY, it);
+                unsigned long long w_acc = 0, w_first = 0;    // trace only
+                if (p.trace_items && !mbar_try_wait_cluster(bar_tempty + 8 * acc, acc_phase ^ 1u)) {
+                    const unsigned long long w0 = globaltimer_ns();
+                    ok = mbar_wait<true>(bar_tempty + 8 * acc, acc_phase ^ 1u, p, SITE_MMA_TEMPTY, it);
+                    w_acc = globaltimer_ns() - w0;
+                } else {
+                    ok = mbar_wait<true>(bar_tempty + 8 * acc, acc_phase ^ 1u, p, SITE_MMA_TEMPTY, it);
+                }
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * TB_N;
+                unsigned long long stall_ns = 0;              // trace only: time spent waiting for operand stages
                 for (int ks = 0; ks < ksteps; ++ks) {
-                    ok = mbar_wait(bar_full + 8 * stage, phase, p, SITE_MMA_FULL, it);
+                    if (p.trace_items && !mbar_test_wait(bar_full + 8 * stage, phase)) {
+                        const unsigned long long w0 = globaltimer_ns();
+                        ok = mbar_wait(bar_full + 8 * stage, phase, p, SITE_MMA_FULL, it);
+                        if (ks > 0) stall_ns += globaltimer_ns() - w0;   // the first stage is the item's start-up
+                        else w_first = globaltimer_ns() - w0;
+                    } else {
+                        ok = mbar_wait(bar_full + 8 * stage, phase, p, SITE_MMA_FULL, it);
+                    }
                     if (!ok) break;
                     if (ks == 0 && p.trace_items) p.trace_items[it].b = globaltimer_ns();
                     tc_fence_after();
@@ -452,6 +480,11 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
+                if (p.trace_items) {
+                    p.trace_item_aux[it].y = (int)stall_ns;
+                    p.trace_items2[it].b = w_first;
+                    p.trace_items2[it].c = w_acc;
+                }
                 umma_commit_pair(bar_tfull + 8 * acc);        // accumulator complete, in both CTAs
                 acc ^= 1;
                 if (acc == 0) acc_phase ^= 1u;
@@ -472,7 +505,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 const int it = atomicAdd(p.next_item, 1);
                 if (p.trace_items && it < n_items) {
                     p.trace_items[it].a = globaltimer_ns();
-                    p.trace_item_cta[it] = (int)blockIdx.x;
+                    p.trace_item_aux[it].x = (int)blockIdx.x;
                 }
                 const int slot = n % PROD_RING;
                 ring_gen[slot] = it;
@@ -540,6 +573,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             ok = epilogue_all(ok);
             if (!ok) break;
             tc_fence_after();
+            if (leader && rank == 0 && p.trace_items) p.trace_items2[it].a = globaltimer_ns();
             const uint32_t taddr = tmem_base + (uint32_t)acc * TB_N + ((uint32_t)(q * 32) << 16);
             const size_t grow = (size_t)(present ? band : 0) * TB_M + row;
             if (!present) {

@@ -42,3 +42,20 @@ def test_two_rank_gloo_aggregate():
 def test_single_process_is_identity():
     from paper_2607_19539_b200 import dist as D
     assert D.aggregate_throughput(10.0, 2.0) == (5.0, 2.0)
+
+
+def test_bench_starts_its_own_ranks():
+    """`bench.py --gpus 2` without a launcher in the environment starts two ranks of itself; --dry-run keeps the
+    run on CPU (gloo) and exercises the barrier / max-over-ranks / whole-job aggregate of the real bench."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run", "--steps", "4",
+                        "--workload", "tiny"], env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stdout + r.stderr
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                   # rank 0 alone prints
+    line = lines[0]
+    assert line["n_gpus"] == 2 and line["steps"] == 4 and line["scaling"] == "weak"
+    # rank r pretends a step takes (r + 1) ms: the job's time is the slowest rank's, its work the sum
+    assert abs(line["ms_per_step"] - 2.0) < 1e-9 and abs(line["value"] - 8 / 8e-3) < 1e-6
+    assert line["config"]["parallelism"] == "replicas x2"
