@@ -263,11 +263,14 @@ def dry_run(args, shape):
 
 
 def interleaved_medians(torch, run_variant, names, rounds):
-    """Variants measured call by call in alternating order (the GPU is power-limited under this load, so a block
+    """Variants measured call by call, interleaved (the GPU is power-limited under this load, so a block
     of steps measured later runs slower than one measured earlier); returns the median ms of each."""
     evs = {n: [] for n in names}
+    rng = np.random.Generator(np.random.PCG64(7))
     for r in range(rounds + 2):
-        for name in (names if r % 2 == 0 else names[::-1]):
+        # a fresh random order every round: under the power cap a call runs a little faster right after a variant
+        # that draws less power, so a fixed order would favour the neighbours of the light variants
+        for name in [names[i] for i in rng.permutation(len(names))]:
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
             run_variant(name)

@@ -264,12 +264,38 @@ int choose_consumer_sms(const moe_ovl_ctx *ctx)
     return std::min(16, std::max(2, 2 * (int)(breakeven / 4.0 + 0.5)));
 }
 
-// MODE_AUTO: which of the three ways to run the return, and with how many consumer SMs.
+// MODE_AUTO: which of the three ways to run the return, and with how many consumer SMs (Section 3.3.3 names
+// the trade-off and leaves the choice to future work).  A three-line cost model over what the host knows --
+// the shape and the number of rows -- with coefficients measured on a B200 at its power cap:
+//   GEMM      padded flop / (8.6 TFLOP/s per GEMM CTA): 148 CTAs reach about 1270 TFLOP/s sustained
+//   scatter   non-overlap only: a launch boundary (about 6 us) + 4*dout bytes per row at 5.5 TB/s
+//   tail      what is left to move after the last tile is flagged: one segment per mover.  A consumer CTA
+//             moves about 35 GB/s of payload, the four spare warps of a GEMM CTA about 15 GB/s of a unit that
+//             is an eighth of a segment
+//   stolen    dedicated consumer SMs are not GEMM SMs: the GEMM term grows by SMs / (SMs - c)
+//   drag      movers inside the GEMM CTAs share their load/store path: about 0.4 % of the GEMM term
+// Padding is estimated as half a band per (expert, rank) group.
 void choose_mode(const moe_ovl_ctx *ctx, int num_rows, int *mode, int *consumer_sms)
 {
-    (void)num_rows;
-    *mode = MOE_OVL_MODE_IN_KERNEL;
+    const moe_ovl_config &c = ctx->cfg;
+    const Layout &L = ctx->L;
     *consumer_sms = choose_consumer_sms(ctx);
+    if (num_rows == 0) { *mode = MOE_OVL_MODE_NON_OVERLAP; return; }       // nothing to return
+    const double sms = ctx->num_sms;
+    const double groups = (double)c.num_local_experts * c.num_src_ranks;
+    const double padded = num_rows + 0.5 * TB_M * groups;
+    const double flop_row = L.single ? 2.0 * c.d_model * L.dout : 6.0 * (double)c.d_model * c.d_ffn;
+    const double gemm_all = padded * flop_row / (8.6e12 * sms);            // seconds on every SM
+    const double row_bytes = 2.0 * L.dout;
+    const double seg_bytes = (double)std::max(1, c.mid_seg_bands) * TB_M * row_bytes;
+    const double t_non = gemm_all + 6e-6 + 2.0 * row_bytes * num_rows / 5.5e12;
+    const double t_in = gemm_all * 1.004 + (seg_bytes / MAX_SEG_CHUNKS) / 15e9;
+    const double cs = *consumer_sms;
+    const double t_ded = gemm_all * sms / (sms - cs) + seg_bytes / 35e9 / std::max(1.0, cs / 4.0);
+    *mode = MOE_OVL_MODE_IN_KERNEL;
+    double best = t_in;
+    if (t_non < best) { best = t_non; *mode = MOE_OVL_MODE_NON_OVERLAP; }
+    if (t_ded < best) { best = t_ded; *mode = MOE_OVL_MODE_OVERLAP; }
 }
 
 int sync_last(moe_ovl_ctx *ctx)

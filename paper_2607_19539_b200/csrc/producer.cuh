@@ -46,7 +46,8 @@ constexpr int PROD_GATHER_WARPS = 4;
 constexpr int PROD_THREADS = 224 + 32 * PROD_GATHER_WARPS;   // TMA, MMA, 4 epilogue warps, scheduler, gather warps
 constexpr int GATHER_ROWS = 8;                         // rows per gather unit
 constexpr int GATHER_HEAD_ROWS = 2;                    // ... in the first super-band of the schedule
-constexpr int PROD_RING = 16;                          // claimed-item ring; roles are never more than 5 items apart
+constexpr int PROD_RING = 16;                          // claimed-item ring; roles are never more than 6 items apart
+constexpr int PROD_LOOKAHEAD = 5;                      // stages before an item's last load at which the next item is looked up
 constexpr int PROD_TMEM_COLS = 512;
 // kernel flags
 constexpr int PROD_RAISE_FLAGS = 1;    // publish a ready flag per finished output tile; idle CTAs help drain segments
@@ -374,41 +375,63 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             uint32_t phase = 0;
             long long fills = 0;
             bool ok = true;
-            for (int n = 0; ok; ++n) {
+            // What the loads of one schedule item need.  It is looked up -- ring slot, item record, the counter the
+            // item depends on -- a few stages BEFORE the previous item's last load, so that these dependent
+            // round trips to L2 do not open a bubble between two items.
+            struct Job {
+                int it, a_row, b_row, ksteps, dep_index;
+                const CUtensorMap *amap, *bmap;
+                const unsigned *dep;        // counter that must reach dep_want before the item's first load
+                unsigned dep_want;
+                long long dep_site;
+                bool dep_ok;
+            };
+            // 1 = item n is in `j`, 0 = schedule exhausted, -1 = gave up
+            auto fetch = [&](int n, Job &j) -> int {
                 const int it = claimed(n);
-                if (it < 0 || it >= n_items) { ok = it >= 0; break; }
+                if (it < 0) return -1;
+                if (it >= n_items) return 0;
                 if (rank == 0) mbar_arrive(bar_go);  // lets the scheduler claim the item after this one
                 const int4 item = p.items[it];       // {kind | expert << 8, band 0, band 1 or -1, tile}
                 const int kind = item.x & 0xff, e = item.x >> 8, tile = item.w;
                 const int band = (rank == 0 || item.z < 0) ? item.y : item.z;
-                const CUtensorMap *amap, *bmap;
-                int b_row, ksteps;
+                j.it = it;
+                j.a_row = band * TB_M;
+                j.dep_index = band;
                 if (kind == KIND_G1) {
-                    amap = &maps.xa; bmap = &maps.w1;
+                    j.amap = &maps.xa; j.bmap = &maps.w1;
                     // rank 0 holds the gate-projection rows of the tile, rank 1 the matching up-projection rows
-                    b_row = e * 2 * p.F + tile * H_TILE + (int)rank * p.F;
-                    ksteps = p.d / TB_K;
+                    j.b_row = e * 2 * p.F + tile * H_TILE + (int)rank * p.F;
+                    j.ksteps = p.d / TB_K;
                     // all 128 rows of the band (padding included) must have been gathered into Xa
-                    ok = wait_global(&p.xready[band], (unsigned)TB_M, true, p, SITE_TMA_XREADY, band);
-                    if (!ok) break;
-                    asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
+                    j.dep = &p.xready[band]; j.dep_want = (unsigned)TB_M; j.dep_site = SITE_TMA_XREADY;
                 } else {
                     // single-projection experts: the output GEMM reads the aligned input itself
-                    amap = p.single ? &maps.xa : &maps.h; bmap = &maps.w2;
-                    b_row = e * p.dout + tile * TB_N + (int)rank * (TB_N / 2);
-                    ksteps = p.k2 / TB_K;
-                    if (p.n1 > 0) {
-                        // every first-GEMM tile of this band must have landed in H
-                        ok = wait_global(&p.hcount[band], (unsigned)p.n1, true, p, SITE_TMA_HCOUNT, band);
+                    j.amap = p.single ? &maps.xa : &maps.h; j.bmap = &maps.w2;
+                    j.b_row = e * p.dout + tile * TB_N + (int)rank * (TB_N / 2);
+                    j.ksteps = p.k2 / TB_K;
+                    if (p.n1 > 0) {   // every first-GEMM tile of this band must have landed in H
+                        j.dep = &p.hcount[band]; j.dep_want = (unsigned)p.n1; j.dep_site = SITE_TMA_HCOUNT;
                     } else {
-                        ok = wait_global(&p.xready[band], (unsigned)TB_M, true, p, SITE_TMA_XREADY, band);
+                        j.dep = &p.xready[band]; j.dep_want = (unsigned)TB_M; j.dep_site = SITE_TMA_XREADY;
                     }
-                    if (!ok) break;
-                    asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
                 }
-                const int a_row = band * TB_M;
-                for (int ks = 0; ks < ksteps; ++ks) {
-                    ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, p, SITE_TMA_EMPTY, it);
+                j.dep_ok = ld_acquire_u32(j.dep) >= j.dep_want;      // the counters only grow
+                return 1;
+            };
+            Job cur, nxt;
+            int have = fetch(0, cur);
+            ok = have >= 0;
+            for (int n = 0; ok && have == 1; ++n) {
+                if (!cur.dep_ok) {
+                    ok = wait_global(cur.dep, cur.dep_want, true, p, cur.dep_site, cur.dep_index);
+                    if (!ok) break;
+                }
+                asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
+                const int look = cur.ksteps > PROD_LOOKAHEAD ? cur.ksteps - PROD_LOOKAHEAD : 0;
+                int have_next = 0;
+                for (int ks = 0; ks < cur.ksteps; ++ks) {
+                    ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, p, SITE_TMA_EMPTY, cur.it);
                     if (!ok) break;
                     const uint32_t sa = smem_base + stage * PROD_STAGE_BYTES, sb = sa + PROD_A_BYTES;
                     const uint32_t full = lead_full + 8 * stage;
@@ -417,11 +440,17 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     // The peer can only refill a stage after the leader's MMAs have consumed (hence completed)
                     // its previous phase, so bytes never leak into the wrong phase.
                     if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * PROD_STAGE_BYTES);
-                    tma_load_2d(sa, amap, full, ks * TB_K, a_row);
-                    tma_load_2d(sb, bmap, full, ks * TB_K, b_row);
+                    tma_load_2d(sa, cur.amap, full, ks * TB_K, cur.a_row);
+                    tma_load_2d(sb, cur.bmap, full, ks * TB_K, cur.b_row);
                     ++fills;
                     if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
+                    if (ks == look) {
+                        have_next = fetch(n + 1, nxt);
+                        if (have_next < 0) { ok = false; break; }
+                    }
                 }
+                cur = nxt;
+                have = have_next;
             }
             if (!ok && rank == 0) {
                 // give-up path: let the copies already issued land before the shared memory goes away
