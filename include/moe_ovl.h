@@ -97,6 +97,8 @@ typedef struct {
                                          bounded wait runs out and the call ends with MOE_OVL_ERR_TIMEOUT */
 #define MOE_OVL_FLAG_TRACE 4u         /* reserve workspace for, and record, the per-item / per-unit device trace
                                          (moe_ovl_get_trace); off by default, costs nothing when off */
+#define MOE_OVL_FLAG_NO_SMALL_GROUP_TILES 16u /* never issue the swapped-operand items that runs of small (expert, rank)
+                                         groups otherwise get (see moe_ovl_plan_view.item); for comparisons */
 #define MOE_OVL_FLAG_TEST_SKIP_GATHER 8u /* test hook: the first band of the schedule is never gathered, so the GEMM's
                                          own bounded wait for it runs out (exercises the give-up path inside the GEMM
                                          kernel: copies drained, tensor memory freed, MOE_OVL_ERR_TIMEOUT) */
@@ -188,8 +190,14 @@ typedef struct {
     int32_t *band_valid;
     int32_t *band_slot0;
     int32_t *sched_band;      /* [bands] band ids in schedule order */
-    int32_t *item;            /* [items][4] = {kind (0 first GEMM, 1 second) | expert << 8, band, second band of the
-                                 pair or -1, tile} in issue order */
+    int32_t *item;            /* [items][4] in issue order.  Kinds 0 (first GEMM) and 1 (second GEMM): {kind | expert << 8,
+                                 band, second band of the pair or -1, tile}, a 256-row x 256-column tile of two bands
+                                 (128 hidden columns per band for kind 0).  Kinds 2 and 3, the same two GEMMs for a
+                                 run whose (expert, rank) groups hold at most 64 rows each: {kind | expert << 8,
+                                 position of the first band in sched_band, bands | rows << 8, tile} -- the valid rows
+                                 of up to 8 consecutive bands (each rounded up to 16, at most 128 together) against a
+                                 tile of 256 weight rows with the operands swapped, so that the tensor cores do not
+                                 multiply padding (tile = 256 hidden columns for kind 2, 256 output columns for 3) */
     int32_t *seg;             /* [segments][4] = {first band, bands, dest rank, rows} in schedule order */
     int32_t *tok_slot;        /* [R*T*min(k,El)] slots of each token's rows, ascending expert, -1 = none */
     float *tok_gate;          /* [R*T*min(k,El)] matching gates */

@@ -15,6 +15,15 @@ constexpr int H_TILE = 128;   // hidden columns per first-GEMM tile (gate half +
 
 constexpr int KIND_G1 = 0;    // x . W1 (gate | up) -> SiLU * up -> H
 constexpr int KIND_G2 = 1;    // H . W2 -> Y, raises the consumer-visible flag
+// The same two GEMMs with the operands swapped, for runs whose bands hold at most SMALL_BAND_ROWS valid rows each:
+// 256 weight rows are the MMA's M side and the valid rows of a GROUP of such bands (each rounded up to 16, at
+// most SWAP_MAX_N together) its N side, so the tensor cores do not multiply padding and one pass over a weight
+// tile serves the whole group.
+constexpr int KIND_G1S = 2;
+constexpr int KIND_G2S = 3;
+constexpr int SMALL_BAND_ROWS = 64;
+constexpr int SWAP_MAX_N = 128;
+constexpr int SWAP_MAX_BANDS = 8;          // SWAP_MAX_N / 16
 
 // meta[] slots written by the plan kernel
 enum { META_P = 0, META_BANDS, META_ITEMS, META_SEGS, META_SUPERBANDS, META_COUNT = 8 };
@@ -52,6 +61,7 @@ struct Params {
     int lag_items;      // schedule items between a band's last first-GEMM tile and its first second-GEMM tile
     int words;          // 32-bit words of one (expert, rank) token bitmap = ceil(T / 32)
     int n1, n2;         // tiles per band: F / 128 (0 for single-projection experts) and dout / 256
+    int swap_ok;        // small runs may use the swapped-operand items (needs F % 256 == 0 for FFN experts)
     int max_bands, max_items;
     unsigned *epoch_rw;      // same word, for the plan kernel
     const unsigned *epoch;   // device word: number of this call; the plan kernel bumps it once per call
@@ -91,6 +101,7 @@ struct Params {
     unsigned *xready;     // [max_bands] rows of the band gathered into Xa (128 = ready)
     unsigned *hcount;     // [max_bands] first-GEMM tiles finished per band
     unsigned *flags;      // [max_bands*n2] epoch of the call that finished the tile
+    unsigned *fcount;     // [max_bands*n2] swapped-operand items: CTAs of the pair that have stored their half of the tile
     int *meta;            // [META_COUNT]
     // optional trace (null when off), raw %globaltimer values: one record per schedule item {claimed, first
     // operands landed, published by CTA 0 of the pair, published by CTA 1} plus trace_item_aux, and

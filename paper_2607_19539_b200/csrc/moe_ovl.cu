@@ -30,13 +30,13 @@ inline size_t align_up(size_t v, size_t a = ALIGN) { return (v + a - 1) / a * a;
 struct Layout {
     // offsets into the workspace, in bytes
     size_t Xa, H, Y;
-    size_t zero_begin, bitmap, hcount, status, next_item, stamps, tok_slot, zero_end;   // cleared at the start of every call
+    size_t zero_begin, bitmap, hcount, fcount, status, next_item, stamps, tok_slot, zero_end;   // cleared at the start of every call
     size_t smid;
     size_t wordpfx, group_rows, group_start, group_slot, pos, slot, row_at, xready;
     size_t band_expert, band_dest, band_valid, band_slot0, sched_band, items, segs, seg_slot0;
     size_t tok_gate, flags, meta;
     size_t trace_items, trace_items2, trace_units, trace_item_aux, trace_bytes;   // MOE_OVL_FLAG_TRACE
-    size_t sb[6];
+    size_t sb[10];
     // host staging (MOE_OVL_FLAG_HOST_STAGING)
     size_t st_x[2], st_counts[2], st_rank[2], st_token[2], st_gate[2], st_out[2], st_ret;   // two staging slots
     size_t total;
@@ -95,6 +95,7 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->zero_begin = off;
     L->bitmap = take((size_t)G * L->words * 4);
     L->hcount = take((size_t)L->max_bands * 4);
+    L->fcount = take((size_t)L->max_bands * L->n2 * 4);
     L->status = take(ST_COUNT * 4);
     L->next_item = take(32);                 // next_item, plan_ticket, next_seg, assist_segs, next_gather
     L->stamps = take(STAMP_COUNT * 8);
@@ -120,7 +121,7 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->flags = take((size_t)L->max_bands * L->n2 * 4);
     L->meta = take(META_COUNT * 4 + 4);      // meta[] and the call counter
     L->smid = take(2 * 1024 * 4);            // SM of every GEMM CTA, then of every consumer CTA
-    for (int i = 0; i < 6; ++i) L->sb[i] = take((size_t)L->max_bands * 4);
+    for (int i = 0; i < 10; ++i) L->sb[i] = take((size_t)L->max_bands * 4);
     L->st_ret_rows = (long long)c->tokens_per_rank * L->kmax;
     L->trace_bytes = 0;
     if (c->flags & MOE_OVL_FLAG_TRACE) {
@@ -171,7 +172,7 @@ struct moe_ovl_ctx {
     bool hist_timed[MOE_OVL_TIMING_HISTORY];
     int last_cuda_error;
     EncodeTiledFn encode;
-    CUtensorMap map_xa, map_h;
+    CUtensorMap map_xa, map_h, map_xa8, map_h8;
 };
 
 namespace {
@@ -185,12 +186,12 @@ namespace {
         }                                                    \
     } while (0)
 
-// 2-D bf16 row-major tensor [rows, cols], box = 64 columns x 128 rows, 128-byte swizzle
-int encode_map(moe_ovl_ctx *ctx, CUtensorMap *map, const void *base, size_t rows, size_t cols)
+// 2-D bf16 row-major tensor [rows, cols], box = 64 columns x box_rows rows (128 unless stated), 128-byte swizzle
+int encode_map(moe_ovl_ctx *ctx, CUtensorMap *map, const void *base, size_t rows, size_t cols, int box_rows = TB_M)
 {
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)std::max<size_t>(rows, 1)};
     const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {TB_K, TB_M};
+    const cuuint32_t box[2] = {TB_K, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides,
                                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -227,6 +228,8 @@ Params make_params(moe_ovl_ctx *ctx)
     p.sched_band = at<int>(ctx, L.sched_band); p.items = at<int4>(ctx, L.items); p.segs = at<int4>(ctx, L.segs);
     p.seg_slot0 = at<int>(ctx, L.seg_slot0); p.tok_slot = at<int>(ctx, L.tok_slot);
     p.tok_gate = at<float>(ctx, L.tok_gate); p.hcount = at<unsigned>(ctx, L.hcount);
+    p.fcount = at<unsigned>(ctx, L.fcount);
+    p.swap_ok = !(c.flags & MOE_OVL_FLAG_NO_SMALL_GROUP_TILES) && (L.single || c.d_ffn % (2 * H_TILE) == 0);
     p.next_item = at<int>(ctx, L.next_item);
     p.plan_ticket = at<int>(ctx, L.next_item) + 1;
     p.next_seg = at<int>(ctx, L.next_item) + 2;
@@ -408,6 +411,9 @@ int moe_ovl_create(moe_ovl_ctx **out, const moe_ovl_config *cfg, void *workspace
     const size_t P = (size_t)L.max_bands * TB_M;
     rc = encode_map(ctx, &ctx->map_xa, ctx->ws + L.Xa, P, cfg->d_model);
     if (rc == MOE_OVL_OK) rc = encode_map(ctx, &ctx->map_h, ctx->ws + L.H, P, L.f_eff);
+    // the same buffers in boxes of 8 rows, for the token side of the swapped-operand items
+    if (rc == MOE_OVL_OK) rc = encode_map(ctx, &ctx->map_xa8, ctx->ws + L.Xa, P, cfg->d_model, 8);
+    if (rc == MOE_OVL_OK) rc = encode_map(ctx, &ctx->map_h8, ctx->ws + L.H, P, L.f_eff, 8);
     if (rc != MOE_OVL_OK) return fail(rc);
     // flags hold the epoch of the call that finished the tile: clear them once, never again
     CREATE_CHECK(cudaMemset(ctx->ws + L.flags, 0, (size_t)L.max_bands * L.n2 * 4));
@@ -494,6 +500,8 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     ProducerMaps maps;
     maps.xa = ctx->map_xa;
     maps.h = ctx->map_h;
+    maps.xa8 = ctx->map_xa8;
+    maps.h8 = ctx->map_h8;
     int rc;
     if (L.single) {
         // one projection per expert: W[El, N, d] is the B operand of the GEMM that writes Y
@@ -508,6 +516,8 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     PlanScratch sc;
     sc.sb_start = at<int>(ctx, L.sb[0]); sc.sb_nb = at<int>(ctx, L.sb[1]); sc.sb_expert = at<int>(ctx, L.sb[2]);
     sc.sb_g1off = at<int>(ctx, L.sb[3]); sc.sb_g2off = at<int>(ctx, L.sb[4]); sc.sb_g1end = at<int>(ctx, L.sb[5]);
+    sc.sb_kind = at<int>(ctx, L.sb[6]); sc.sb_ntok = at<int>(ctx, L.sb[7]);
+    sc.sb_c1 = at<int>(ctx, L.sb[8]); sc.sb_c2 = at<int>(ctx, L.sb[9]);
 
     int launches = 0;
     const int hist = (int)(ctx->calls % MOE_OVL_TIMING_HISTORY);

@@ -25,7 +25,13 @@ struct PlanScratch {
     int *sb_g1off;   // item index of the super-band's first-GEMM block
     int *sb_g2off;   // item index of its second-GEMM block
     int *sb_g1end;
+    int *sb_kind;    // 0: band pairs (KIND_G1 / KIND_G2 items), 1: one group of small bands (KIND_G1S / KIND_G2S)
+    int *sb_ntok;    // group of small bands: valid rows, each band rounded up to 16
+    int *sb_c1;      // items of the super-band's first-GEMM block
+    int *sb_c2;      // ... of its second-GEMM block
 };
+
+__device__ __forceinline__ int ceil16(int v) { return (v + 15) & ~15; }
 
 __device__ __forceinline__ int expert_of_row(const int *pre, int El, int i)
 {
@@ -100,11 +106,12 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     __shared__ int key[PLAN_MAX_EXPERTS], eorder[PLAN_MAX_EXPERTS];
     __shared__ int run_start[2 * PLAN_MAX_EXPERTS], run_nb[2 * PLAN_MAX_EXPERTS], run_sb0[2 * PLAN_MAX_EXPERTS + 1];
     __shared__ int run_exp[2 * PLAN_MAX_EXPERTS], run_segs[2 * PLAN_MAX_EXPERTS];
+    __shared__ int run_nsb[2 * PLAN_MAX_EXPERTS];     // groups of small bands in the run, or -1: issued as band pairs
     __shared__ int esize[PLAN_MAX_EXPERTS];
     __shared__ int s_total;
     __shared__ int segs_per_rank[PLAN_MAX_GROUPS];
     __shared__ int s_nsb;
-    __shared__ int s_sb_nb[PLAN_SB_STAGE], s_sb_end[PLAN_SB_STAGE];
+    __shared__ int s_sb_c1[PLAN_SB_STAGE], s_sb_c2[PLAN_SB_STAGE], s_sb_end[PLAN_SB_STAGE];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
     const int G = p.El * p.R;
@@ -202,6 +209,10 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
         const bool remote = run < El;
         const int e = remote ? eorder[run] : run - El;
         int nbands = 0, nsegs = 0;
+        // A run whose groups all fit in half a band is issued as groups of small bands with swapped operands:
+        // consecutive bands while their rows, each band rounded up to 16, stay within SWAP_MAX_N.
+        bool small = p.swap_ok != 0;
+        int sgroups = 0, acc_tok = SWAP_MAX_N + 1;
         for (int q = remote ? 0 : R - 1; q < (remote ? R - 1 : R); ++q) {
             const int r = q < R - 1 ? (q < self ? q : q + 1) : self;
             const int g = e * R + r;
@@ -211,10 +222,16 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
             nbands += nb[g];
             nsegs += ns;
             atomicAdd(&segs_per_rank[r], ns);
+            small = small && n[g] <= SMALL_BAND_ROWS;
+            if (n[g] > 0) {
+                if (acc_tok + ceil16(n[g]) > SWAP_MAX_N) { ++sgroups; acc_tok = 0; }
+                acc_tok += ceil16(n[g]);
+            }
         }
         run_exp[run] = e;
         run_nb[run] = nbands;
         run_segs[run] = nsegs;
+        run_nsb[run] = (small && nbands > 0) ? sgroups : -1;
     }
     __syncthreads();
     if (tid == 0) {
@@ -226,9 +243,10 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
             run_segs[run] = segoff;             // now the run's first segment
             segoff += nsegs;
             run_sb0[run] = sbcount;
-            // super-bands are made of whole band pairs (the GEMM works on two bands at a time)
+            // super-bands are made of whole band pairs (the GEMM works on two bands at a time); a run of small
+            // bands has one super-band per group instead
             const int pairs = (run_nb[run] + 1) / 2, pairs_per_sb = max(1, p.group_bands / 2);
-            sbcount += (pairs + pairs_per_sb - 1) / pairs_per_sb;
+            sbcount += run_nsb[run] >= 0 ? run_nsb[run] : (pairs + pairs_per_sb - 1) / pairs_per_sb;
         }
         run_sb0[2 * El] = sbcount;
         s_nsb = sbcount;
@@ -280,6 +298,33 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     for (int run = tid; run < 2 * El; run += blockDim.x) {
         const int nsb = run_sb0[run + 1] - run_sb0[run];
         const int pairs = (run_nb[run] + 1) / 2;
+        if (run_nsb[run] >= 0) {
+            // one super-band per group of small bands; every group of the run holds at most one band, so the
+            // run's bands are its non-empty groups in layout order
+            const bool remote = run < El;
+            const int e = run_exp[run];
+            int sb = run_sb0[run] - 1, acc_tok = SWAP_MAX_N + 1, pos = run_start[run];
+            for (int q = remote ? 0 : R - 1; q < (remote ? R - 1 : R); ++q) {
+                const int r = q < R - 1 ? (q < self ? q : q + 1) : self;
+                const int g = e * R + r;
+                if (n[g] == 0) continue;
+                if (acc_tok + ceil16(n[g]) > SWAP_MAX_N) {
+                    ++sb;
+                    acc_tok = 0;
+                    sc.sb_start[sb] = pos;
+                    sc.sb_nb[sb] = 0;
+                    sc.sb_expert[sb] = e;
+                    sc.sb_kind[sb] = 1;
+                    sc.sb_c1[sb] = p.n1 / 2;          // tiles of 256 hidden columns
+                    sc.sb_c2[sb] = p.n2;
+                }
+                acc_tok += ceil16(n[g]);
+                sc.sb_nb[sb] += 1;
+                sc.sb_ntok[sb] = acc_tok;
+                ++pos;
+            }
+            continue;
+        }
         for (int q = 0; q < nsb; ++q) {
             // spread the run's band pairs evenly; only the run's last super-band can end on a single band
             const int base = pairs / nsb, rem = pairs % nsb;
@@ -288,6 +333,10 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
             sc.sb_start[sb] = run_start[run] + 2 * pair0;
             sc.sb_nb[sb] = min(2 * npairs, run_nb[run] - 2 * pair0);
             sc.sb_expert[sb] = run_exp[run];
+            sc.sb_kind[sb] = 0;
+            sc.sb_ntok[sb] = 0;
+            sc.sb_c1[sb] = ((sc.sb_nb[sb] + 1) / 2) * p.n1;
+            sc.sb_c2[sb] = ((sc.sb_nb[sb] + 1) / 2) * p.n2;
         }
     }
     __syncthreads();
@@ -302,21 +351,21 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
         const int nsb = s_nsb;
         const bool staged = nsb <= PLAN_SB_STAGE;
         if (staged)
-            for (int i = tid; i < nsb; i += blockDim.x) s_sb_nb[i] = sc.sb_nb[i];
+            for (int i = tid; i < nsb; i += blockDim.x) { s_sb_c1[i] = sc.sb_c1[i]; s_sb_c2[i] = sc.sb_c2[i]; }
         __syncthreads();
         if (tid == 0) {
-            int *nbv = staged ? s_sb_nb : sc.sb_nb;
+            int *c1v = staged ? s_sb_c1 : sc.sb_c1, *c2v = staged ? s_sb_c2 : sc.sb_c2;
             int *endv = staged ? s_sb_end : sc.sb_g1end;
             int ng1 = 0, off = 0;
             for (int ng2 = 0; ng2 < nsb; ++ng2) {
                 while (ng1 < nsb && (ng1 <= ng2 || off - endv[ng2] < p.lag_items)) {
                     sc.sb_g1off[ng1] = off;
-                    off += ((nbv[ng1] + 1) / 2) * p.n1;
+                    off += c1v[ng1];
                     endv[ng1] = off;
                     ++ng1;
                 }
                 sc.sb_g2off[ng2] = off;
-                off += ((nbv[ng2] + 1) / 2) * p.n2;
+                off += c2v[ng2];
             }
             p.meta[META_ITEMS] = off;
         }
@@ -328,6 +377,16 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
         const int start = sc.sb_start[sb], cnt = sc.sb_nb[sb], e = sc.sb_expert[sb];
         const int np = (cnt + 1) / 2;
         const int o1 = sc.sb_g1off[sb], o2 = sc.sb_g2off[sb];
+        if (sc.sb_kind[sb]) {
+            // group of small bands: {kind | expert << 8, first schedule position, bands | rows << 8, tile}
+            const int c1 = sc.sb_c1[sb], desc = cnt | (sc.sb_ntok[sb] << 8);
+            for (int idx = lane; idx < c1 + p.n2; idx += 32) {
+                const bool g1 = idx < c1;
+                p.items[g1 ? o1 + idx : o2 + idx - c1] =
+                    make_int4((g1 ? KIND_G1S : KIND_G2S) | (e << 8), start, desc, g1 ? idx : idx - c1);
+            }
+            continue;
+        }
         for (int idx = lane; idx < np * (p.n1 + p.n2); idx += 32) {
             const bool g1 = idx < np * p.n1;
             const int k = g1 ? idx : idx - np * p.n1;

@@ -53,7 +53,8 @@ constexpr int PROD_TMEM_COLS = 512;
 constexpr int PROD_RAISE_FLAGS = 1;    // publish a ready flag per finished output tile; idle CTAs help drain segments
 constexpr int PROD_WARP_MOVERS = 2;    // in-kernel return: the gather warps move finished segments once Xa is complete
 constexpr int PROD_SKIP_FIRST_BAND = 4; // test hook: the first band of the schedule is never gathered
-constexpr int PROD_SMEM_BYTES = PROD_STAGES * PROD_STAGE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers, ring*/;
+constexpr int PROD_AUX_BYTES = 1792;   // barriers, claim ring, mover ints, tables of the swapped-operand items
+constexpr int PROD_SMEM_BYTES = PROD_STAGES * PROD_STAGE_BYTES + 1024 /*alignment slack*/ + PROD_AUX_BYTES;
 
 // ------------------------------------------------------------------ PTX wrappers
 
@@ -243,6 +244,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
+__device__ __forceinline__ int ceil16_rows(int v) { return (v + 15) & ~15; }
 __device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
 
 __device__ __forceinline__ void bar_sync_epilogue() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -303,7 +305,21 @@ __device__ __forceinline__ void gather_unit(const Params &p, int band, int r0, i
 
 struct ProducerMaps {
     CUtensorMap xa, h, w1, w2;   // all 2-D bf16 row-major, box 64 x 128, 128-byte swizzle
+    CUtensorMap xa8, h8;         // Xa and H again in boxes of 64 x 8: token rows of the swapped-operand items
 };
+
+// Instruction descriptor of a swapped-operand MMA: 256 weight rows over the CTA pair, N = rows of the band group.
+__device__ __forceinline__ uint32_t umma_idesc_n(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)((2 * TB_M) >> 4) << 24);
+}
+// acq_rel add that returns the old value: the second CTA of a pair to finish a tile learns that it is the second
+__device__ __forceinline__ unsigned atom_add_acq_rel_u32(unsigned *p, unsigned v)
+{
+    unsigned old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PROD_THREADS, 1)
 producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const int kflags)
@@ -321,6 +337,12 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
     const uint32_t bar_ring = bar_go + 8;                          // PROD_RING barriers: slot filled
     const uint32_t ring = bar_ring + 8 * PROD_RING;                // PROD_RING claimed item indices
     const uint32_t mover_ints = ring + 4 * PROD_RING;              // two ints of the in-kernel movers
+    // swapped-operand items: the load thread's band tables (this item and the next: band, rows per CTA) and the
+    // epilogue's column -> buffer row maps (one per accumulator buffer, SWAP_MAX_N columns each)
+    const uint32_t swap_tab = mover_ints + 8;                      // [2][SWAP_MAX_BANDS] int2
+    const uint32_t swap_rowmap = swap_tab + 2 * SWAP_MAX_BANDS * 8;   // [2][SWAP_MAX_N] int
+    static_assert(16 * PROD_STAGES + 16 + 16 + 8 + 8 + 8 + 8 * PROD_RING + 4 * PROD_RING + 8 + 2 * SWAP_MAX_BANDS * 8 +
+                  2 * SWAP_MAX_N * 4 <= PROD_AUX_BYTES, "auxiliary shared memory");
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     volatile uint32_t *tmem_slot_gen = reinterpret_cast<volatile uint32_t *>(smem_gen + (tmem_slot - smem_base));
     volatile int *ring_gen = reinterpret_cast<volatile int *>(smem_gen + (ring - smem_base));
@@ -350,6 +372,8 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
         prefetch_tmap(&maps.h);
         prefetch_tmap(&maps.w1);
         prefetch_tmap(&maps.w2);
+        prefetch_tmap(&maps.xa8);
+        prefetch_tmap(&maps.h8);
     }
     if (warp == 1) tmem_alloc(tmem_slot, PROD_TMEM_COLS);
     tc_fence_before();
@@ -385,7 +409,12 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 unsigned dep_want;
                 long long dep_site;
                 bool dep_ok;
+                // swapped-operand items: weight rows are the A side; nb bands of tokens the B side (table in
+                // shared memory, slot tab); gate and up projection take separate stage fills (fills = 2 * ksteps)
+                int swap, nb, tab, half_rows, w_row, w_row_up;
+                const CUtensorMap *tokmap;
             };
+            volatile int2 *tabs = reinterpret_cast<volatile int2 *>(smem_gen + (swap_tab - smem_base));
             // 1 = item n is in `j`, 0 = schedule exhausted, -1 = gave up
             auto fetch = [&](int n, Job &j) -> int {
                 const int it = claimed(n);
@@ -394,8 +423,38 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 if (rank == 0) mbar_arrive(bar_go);  // lets the scheduler claim the item after this one
                 const int4 item = p.items[it];       // {kind | expert << 8, band 0, band 1 or -1, tile}
                 const int kind = item.x & 0xff, e = item.x >> 8, tile = item.w;
-                const int band = (rank == 0 || item.z < 0) ? item.y : item.z;
                 j.it = it;
+                j.swap = kind >= KIND_G1S;
+                if (j.swap) {
+                    // {kind | expert << 8, first schedule position, bands | rows << 8, tile}
+                    j.nb = item.z & 0xff;
+                    j.tab = n & 1;
+                    j.half_rows = (item.z >> 8) / 2;
+                    const bool g1 = kind == KIND_G1S;
+                    if (g1) {
+                        // this CTA's 128 of the tile's 256 hidden columns: gate rows, and the matching up rows
+                        j.w_row = e * 2 * p.F + tile * 2 * H_TILE + (int)rank * H_TILE;
+                        j.w_row_up = j.w_row + p.F;
+                        j.amap = &maps.w1; j.tokmap = &maps.xa8; j.ksteps = p.d / TB_K;
+                    } else {
+                        j.w_row = e * p.dout + tile * TB_N + (int)rank * (TB_N / 2);
+                        j.w_row_up = j.w_row;
+                        j.amap = &maps.w2; j.tokmap = p.single ? &maps.xa8 : &maps.h8; j.ksteps = p.k2 / TB_K;
+                    }
+                    const bool on_x = g1 || p.n1 == 0;     // depends on gathered rows, else on finished hidden tiles
+                    j.dep_site = on_x ? SITE_TMA_XREADY : SITE_TMA_HCOUNT;
+                    j.dep_want = on_x ? (unsigned)TB_M : (unsigned)p.n1;
+                    j.dep_ok = true;
+                    for (int i = 0; i < j.nb; ++i) {
+                        const int b = p.sched_band[item.y + i];
+                        tabs[j.tab * SWAP_MAX_BANDS + i].x = b;
+                        tabs[j.tab * SWAP_MAX_BANDS + i].y = ceil16_rows(p.band_valid[b]) / 2;
+                        j.dep_ok = j.dep_ok && ld_acquire_u32(on_x ? &p.xready[b] : &p.hcount[b]) >= j.dep_want;
+                    }
+                    j.dep = on_x ? p.xready : p.hcount;
+                    return 1;
+                }
+                const int band = (rank == 0 || item.z < 0) ? item.y : item.z;
                 j.a_row = band * TB_M;
                 j.dep_index = band;
                 if (kind == KIND_G1) {
@@ -423,13 +482,52 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             int have = fetch(0, cur);
             ok = have >= 0;
             for (int n = 0; ok && have == 1; ++n) {
-                if (!cur.dep_ok) {
+                if (!cur.dep_ok && cur.swap) {
+                    for (int i = 0; i < cur.nb && ok; ++i) {
+                        const int b = tabs[cur.tab * SWAP_MAX_BANDS + i].x;
+                        ok = wait_global(cur.dep + b, cur.dep_want, true, p, cur.dep_site, b);
+                    }
+                    if (!ok) break;
+                } else if (!cur.dep_ok) {
                     ok = wait_global(cur.dep, cur.dep_want, true, p, cur.dep_site, cur.dep_index);
                     if (!ok) break;
                 }
                 asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
-                const int look = cur.ksteps > PROD_LOOKAHEAD ? cur.ksteps - PROD_LOOKAHEAD : 0;
                 int have_next = 0;
+                if (cur.swap) {
+                    // Stage fill = 128 weight rows (A slot) + the group's token rows (B slot, this CTA's half of every
+                    // band, boxes of 8 rows).  First-GEMM items alternate gate and up rows against the same tokens.
+                    const int per_k = cur.w_row_up != cur.w_row ? 2 : 1, fills_item = per_k * cur.ksteps;
+                    const int look = fills_item > PROD_LOOKAHEAD ? fills_item - PROD_LOOKAHEAD : 0;
+                    const uint32_t tx = 2u * (uint32_t)(PROD_A_BYTES + cur.half_rows * TB_K * 2);
+                    for (int f = 0; f < fills_item; ++f) {
+                        const int ks = f / per_k;
+                        ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, p, SITE_TMA_EMPTY, cur.it);
+                        if (!ok) break;
+                        const uint32_t sa = smem_base + stage * PROD_STAGE_BYTES, sb = sa + PROD_A_BYTES;
+                        const uint32_t full = lead_full + 8 * stage;
+                        if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, tx);
+                        tma_load_2d(sa, cur.amap, full, ks * TB_K, (f % per_k) ? cur.w_row_up : cur.w_row);
+                        uint32_t dst = sb;
+                        for (int i = 0; i < cur.nb; ++i) {
+                            const int2 t = make_int2(tabs[cur.tab * SWAP_MAX_BANDS + i].x,
+                                                     tabs[cur.tab * SWAP_MAX_BANDS + i].y);
+                            const int row0 = t.x * TB_M + (int)rank * t.y;
+                            for (int r8 = 0; r8 < t.y; r8 += 8, dst += 8 * TB_K * 2)
+                                tma_load_2d(dst, cur.tokmap, full, ks * TB_K, row0 + r8);
+                        }
+                        ++fills;
+                        if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
+                        if (f == look) {
+                            have_next = fetch(n + 1, nxt);
+                            if (have_next < 0) { ok = false; break; }
+                        }
+                    }
+                    cur = nxt;
+                    have = have_next;
+                    continue;
+                }
+                const int look = cur.ksteps > PROD_LOOKAHEAD ? cur.ksteps - PROD_LOOKAHEAD : 0;
                 for (int ks = 0; ks < cur.ksteps; ++ks) {
                     ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, p, SITE_TMA_EMPTY, cur.it);
                     if (!ok) break;
@@ -473,8 +571,14 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             for (int n = 0; ok; ++n) {
                 const int it = claimed(n);
                 if (it < 0 || it >= n_items) break;
-                const int kind = p.items[it].x & 0xff;
-                const int ksteps = (kind == KIND_G1 ? p.d : p.k2) / TB_K;
+                const int4 item = p.items[it];
+                const int kind = item.x & 0xff;
+                const bool swap = kind >= KIND_G1S;
+                const bool first_gemm = kind == KIND_G1 || kind == KIND_G1S;
+                const int per_k = kind == KIND_G1S ? 2 : 1;           // gate and up rows take separate stage fills
+                const int ksteps = per_k * ((first_gemm ? p.d : p.k2) / TB_K);
+                const int ntok = swap ? item.z >> 8 : 0;
+                const uint32_t idesc = swap ? umma_idesc_n(ntok) : UMMA_IDESC;
                 unsigned long long w_acc = 0, w_first = 0;    // trace only
                 if (p.trace_items && !mbar_try_wait_cluster(bar_tempty + 8 * acc, acc_phase ^ 1u)) {
                     const unsigned long long w0 = globaltimer_ns();
@@ -501,10 +605,14 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     tc_fence_after();
                     const uint32_t sa = smem_base + stage * PROD_STAGE_BYTES, sb = sa + PROD_A_BYTES;
                     const uint64_t adesc = umma_smem_desc(sa), bdesc = umma_smem_desc(sb);
+                    // swapped first GEMM: even fills accumulate the gate half in columns [0, ntok), odd fills the
+                    // up half in [ntok, 2 ntok)
+                    const uint32_t d_col = d_tmem + (uint32_t)((ks % per_k) * ntok);
+                    const int kk = ks / per_k;
 #pragma unroll
                     for (int k = 0; k < TB_K / 16; ++k)      // 16 bf16 = 32 bytes per MMA along K
-                        umma_bf16(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), UMMA_IDESC,
-                                  (ks | k) != 0 ? 1u : 0u);
+                        umma_bf16(d_col, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
+                                  (kk | k) != 0 ? 1u : 0u);
                     umma_commit_pair(bar_empty + 8 * stage);  // both CTAs may refill the stage once it has been read
                     if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -596,7 +704,9 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             if (it >= n_items) break;
             const int4 item = p.items[it];
             const int kind = item.x & 0xff, tile = item.w;
-            const bool present = (rank == 0) || item.z >= 0;        // the pair's second band may be absent
+            const bool swap = kind >= KIND_G1S;
+            const bool first_gemm = kind == KIND_G1 || kind == KIND_G1S;
+            const bool present = swap || (rank == 0) || item.z >= 0;     // the pair's second band may be absent
             const int band = rank == 0 ? item.y : item.z;
             ok = mbar_wait(bar_tfull + 8 * acc, acc_phase, p, SITE_EPI_TFULL, it);
             ok = epilogue_all(ok);
@@ -605,7 +715,47 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             if (leader && rank == 0 && p.trace_items) p.trace_items2[it].a = globaltimer_ns();
             const uint32_t taddr = tmem_base + (uint32_t)acc * TB_N + ((uint32_t)(q * 32) << 16);
             const size_t grow = (size_t)(present ? band : 0) * TB_M + row;
-            if (!present) {
+            if (swap) {
+                // Swapped operands: lane = one of this CTA's 128 weight rows, i.e. one hidden / output column;
+                // accumulator column n = row n of the band group (first halves of all bands from CTA 0's token
+                // rows, then the second halves from CTA 1's).  A table maps n to the row of H / Y (-1: padding).
+                const int nb = item.z & 0xff, ntok = item.z >> 8, nh = ntok / 2;
+                volatile int *rowmap =
+                    reinterpret_cast<volatile int *>(smem_gen + (swap_rowmap - smem_base)) + acc * SWAP_MAX_N;
+                if (row < ntok) {
+                    const int half = row >= nh ? 1 : 0, np = row - half * nh;
+                    int off = 0, val = -1;
+                    for (int i = 0; i < nb; ++i) {
+                        const int b = p.sched_band[item.y + i];
+                        const int v = p.band_valid[b], h = ceil16_rows(v) / 2;
+                        if (np >= off && np < off + h) {
+                            const int rib = half * h + (np - off);
+                            val = rib < v ? b * TB_M + rib : -1;
+                        }
+                        off += h;
+                    }
+                    rowmap[row] = val;
+                }
+                bar_sync_epilogue();
+                const size_t width = first_gemm ? (size_t)p.F : (size_t)p.dout;
+                uint16_t *dst = (first_gemm ? p.H : p.Y) + (size_t)tile * TB_N + rank * (TB_N / 2) + row;
+#pragma unroll 1
+                for (int c = 0; c < ntok; c += 32) {
+                    uint32_t g[32], u[32];
+                    tmem_ld32(taddr + c, g);
+                    if (first_gemm) tmem_ld32(taddr + ntok + c, u);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int r = c + j < ntok ? rowmap[c + j] : -1;          // the same for every lane
+                        if (r >= 0) {
+                            const float val = first_gemm ? silu_mul(__uint_as_float(g[j]), __uint_as_float(u[j]))
+                                                         : __uint_as_float(g[j]);
+                            dst[(size_t)r * width] = (uint16_t)(pack_bf16x2(val, 0.f) & 0xffffu);
+                        }
+                    }
+                }
+            } else if (!present) {
                 // nothing to store: the accumulator of an absent band is discarded
             } else if (kind == KIND_G1) {
                 uint16_t *dst = p.H + grow * p.F + (size_t)tile * H_TILE;
@@ -649,14 +799,30 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             }
             // publish (Section 3.3.1): stores, fence, then one release per tile
             __threadfence();
-            if (kind == KIND_G1) asm volatile("fence.proxy.async;" ::: "memory");   // H is re-read through TMA
+            if (first_gemm) asm volatile("fence.proxy.async;" ::: "memory");   // H is re-read through TMA
             bar_sync_epilogue();
             if (leader && present && p.trace_items) {
                 // taken before the release below, so that no observer of the flag can carry an earlier time
                 const unsigned long long now = globaltimer_ns();
                 if (rank == 0) p.trace_items[it].c = now; else p.trace_items[it].d = now;
             }
-            if (leader && present) {
+            if (leader && swap) {
+                // Both CTAs of the pair hold half of the columns of every band's tile.  Hidden tiles: each CTA counts
+                // once per band (two per 256 columns, as two 128-column tiles would).  Output tiles: the CTA that
+                // arrives second publishes the flag.
+                const int nb = item.z & 0xff;
+                for (int i = 0; i < nb; ++i) {
+                    const int b = p.sched_band[item.y + i];
+                    if (first_gemm) {
+                        red_release_add_u32(&p.hcount[b], 1u);
+                    } else if (raise_flags && atom_add_acq_rel_u32(&p.fcount[(size_t)b * p.n2 + tile], 1u) == 1u) {
+                        st_release_u32(&p.flags[(size_t)b * p.n2 + tile], epoch);
+                        const unsigned long long now = globaltimer_ns();
+                        stamp_max(&p.stamps[STAMP_FIRST_FLAG_INV], ~now);
+                        stamp_max(&p.stamps[STAMP_LAST_FLAG], now);
+                    }
+                }
+            } else if (leader && present) {
                 if (kind == KIND_G1) red_release_add_u32(&p.hcount[band], 1u);
                 else if (raise_flags) {
                     st_release_u32(&p.flags[(size_t)band * p.n2 + tile], epoch);

@@ -76,6 +76,11 @@ SHAPES: Dict[str, MoEShape] = {
                                   router="zipf"),
     # many (expert, rank) groups with few rows each: 512 groups, almost every band partial
     "many_groups": MoEShape("many_groups", R=16, T=300, Eg=64, k=4, El=32, d=256, F=128, self_rank=5, seed=4),
+    # the same with a hidden width the swapped-operand items accept (every run is a run of small bands), and a
+    # decode-sized batch: a handful of rows per (expert, rank) group
+    "many_small_groups": MoEShape("many_small_groups", R=16, T=300, Eg=64, k=4, El=32, d=256, F=256, self_rank=5, seed=4),
+    "decode": MoEShape("decode", R=4, T=64, Eg=16, k=2, El=4, d=512, F=768, self_rank=1, seed=6),
+    "decode_single": MoEShape("decode_single", R=4, T=96, Eg=24, k=2, El=6, d=320, F=0, N_out=768, self_rank=3, seed=8),
     "single_small": MoEShape("single_small", R=3, T=600, Eg=6, k=2, El=2, d=192, F=0, N_out=512, self_rank=2, seed=2),
     # mid-size shapes for parity tests (several bands per group, ragged tails)
     "small": MoEShape("small", R=3, T=700, Eg=6, k=2, El=3, d=512, F=384, self_rank=1),

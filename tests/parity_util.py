@@ -61,12 +61,25 @@ def check_indices(shape, dsp, plan, gpu_plan, slot_out, rows_per_rank, segs_per_
     # issue order: the library interleaves the tiles of neighbouring bands (so that they share weight tiles in
     # L2) and adds the first-GEMM tiles, so the list is not Algorithm 1's literally; what is unique must hold:
     # an item is {kind | expert << 8, band, second band of the pair or -1, tile}: expand pairs to single bands
+    # (kinds 2 and 3 -- a group of small bands against 256 weight rows, operands swapped -- expand to the same
+    # per-band tiles: {kind | expert << 8, first schedule position, bands | rows << 8, tile}, where a first-GEMM
+    # tile of 256 hidden columns stands for two of 128)
     raw = gpu_plan["item"]
     rows = []
+    sched = gpu_plan["sched_band"].tolist()
+    valid = gpu_plan["band_valid"].tolist()
     for x, b0, b1, tile in raw.tolist():
-        rows.append((x & 0xff, b0, tile, x >> 8))
+        kind, e = x & 0xff, x >> 8
+        if kind >= 2:
+            group = sched[b0:b0 + (b1 & 0xff)]
+            assert 1 <= len(group) <= 8 and all(valid[b] <= 64 for b in group)
+            assert (b1 >> 8) == sum(-(-valid[b] // 16) * 16 for b in group) <= 128
+            for b in group:
+                rows += [(0, b, 2 * tile, e), (0, b, 2 * tile + 1, e)] if kind == 2 else [(1, b, tile, e)]
+            continue
+        rows.append((kind, b0, tile, e))
         if b1 >= 0:
-            rows.append((x & 0xff, b1, tile, x >> 8))
+            rows.append((kind, b1, tile, e))
     items = np.asarray(rows, np.int64).reshape(-1, 4)
     n1, n2 = (0 if shape.N_out else shape.F // 128), shape.dout // 256
     g2 = items[items[:, 0] == 1]

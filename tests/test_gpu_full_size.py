@@ -42,6 +42,7 @@ def all_tokens_with_rows(shape, dsp):
     ("mixtral", 8, None), ("fine", 8, None), ("mixtral_zipf", 8, 8), ("paper_op_e16_zipf", 14, 16),
     # points of the sweep grid: 4 local experts of 16, d=4096; (tokens per local expert, ffn, router)
     ((1024, 1024, "uniform"), 2, 16), ((128, 2816, "zipf"), 16, 8), ((4096, 1024, "zipf"), 32, 8),
+    ((128, 14336, "uniform"), 8, 32),       # decode-sized batch: every run is a run of small groups
     ((16384, 14336, "uniform"), 4, 4),      # the largest point of the grid: 65893 rows, 6.5 GB of workspace
 ])
 def test_full_size_parity(name, csm, per_rank):

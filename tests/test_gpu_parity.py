@@ -30,7 +30,8 @@ def _run_case(shape, mode, csm, shuffle=None, mgb=1, group_bands=0, inp=None, ds
     return inp, dsp, ctx, prob
 
 
-SMALL = ["tiny", "tiny_zipf", "small", "small_zipf_rot", "single_small", "many_groups"]
+SMALL = ["tiny", "tiny_zipf", "small", "small_zipf_rot", "single_small", "many_groups", "many_small_groups", "decode",
+         "decode_single"]
 
 
 @pytest.mark.parametrize("name", SMALL)
@@ -69,7 +70,7 @@ def test_segment_and_group_knobs(name, mgb, gb):
     U.check_values(shape, dsp, plan, toks, *o, Hn.device_to_bits(prob.out), Hn.device_to_bits(prob.ret))
 
 
-@pytest.mark.parametrize("name", ["tiny", "small_zipf_rot"])
+@pytest.mark.parametrize("name", ["tiny", "small_zipf_rot", "decode"])
 def test_overlap_equals_non_overlap_bitwise(name):
     """Both modes run the same GEMM code on the same tiles: any difference is a protocol bug, not rounding.
     Two different problems alternate on one context, so that before every overlapped run the internal buffers
@@ -564,3 +565,31 @@ def test_rows_beyond_the_receive_region_are_reported_and_never_written():
     Hn.run(ctx, good, mode=B.MODE_OVERLAP, consumer_sm_count=4)
     torch.cuda.synchronize()
     assert ctx.moe_ovl_query_status()[0] == 0
+
+
+@pytest.mark.parametrize("name", ["decode", "many_small_groups", "tiny"])
+def test_small_group_items_can_be_switched_off(name):
+    """Runs of small (expert, rank) groups are issued as swapped-operand items; with the flag that forbids them the
+    same problem goes through band-pair items only.  Both must match the oracle, and the plan must show the
+    difference."""
+    torch, B, Hn = _gpu()
+    shape = I.SHAPES[name]
+    inp = I.make_inputs(shape)
+    dsp = I.dispatch(inp)
+    plan = U.oracle_plan(shape, dsp)
+    toks = np.arange(shape.R * shape.T)
+    o = U.oracle_values(inp, toks)
+    kinds = {}
+    for flags in (0, B.FLAG_NO_SMALL_GROUP_TILES):
+        ctx = Hn.make_context(shape, max_rows=dsp.M, flags=flags)
+        prob = Hn.upload(inp, dsp)
+        Hn.run(ctx, prob, mode=B.MODE_IN_KERNEL)
+        torch.cuda.synchronize()
+        assert ctx.moe_ovl_query_status()[0] == 0
+        gp = ctx.moe_ovl_get_plan()
+        U.check_indices(shape, dsp, plan, gp, prob.slot_out.cpu().numpy(), prob.rows_per_rank_out.cpu().numpy(),
+                        prob.segs_per_rank_out.cpu().numpy(), ctx.moe_ovl_get_report())
+        U.check_values(shape, dsp, plan, toks, *o, Hn.device_to_bits(prob.out), Hn.device_to_bits(prob.ret))
+        kinds[flags] = set((gp["item"][:, 0] & 0xff).tolist())
+    assert kinds[B.FLAG_NO_SMALL_GROUP_TILES] <= {0, 1}
+    assert kinds[0] & {2, 3}                      # every one of these problems has at least one run of small groups
