@@ -99,6 +99,8 @@ typedef struct {
                                          (moe_ovl_get_trace); off by default, costs nothing when off */
 #define MOE_OVL_FLAG_NO_SMALL_GROUP_TILES 16u /* never issue the swapped-operand items that runs of small (expert, rank)
                                          groups otherwise get (see moe_ovl_plan_view.item); for comparisons */
+#define MOE_OVL_FLAG_TEST_ALL_SMALL_GROUP_TILES 32u /* test hook: every eligible run of small groups gets swapped-operand
+                                         items, also where the plan's cost rule would keep band pairs */
 #define MOE_OVL_FLAG_TEST_SKIP_GATHER 8u /* test hook: the first band of the schedule is never gathered, so the GEMM's
                                          own bounded wait for it runs out (exercises the give-up path inside the GEMM
                                          kernel: copies drained, tensor memory freed, MOE_OVL_ERR_TIMEOUT) */
@@ -196,8 +198,10 @@ typedef struct {
                                  run whose (expert, rank) groups hold at most 64 rows each: {kind | expert << 8,
                                  position of the first band in sched_band, bands | rows << 8, tile} -- the valid rows
                                  of up to 8 consecutive bands (each rounded up to 16, at most 128 together) against a
-                                 tile of 256 weight rows with the operands swapped, so that the tensor cores do not
-                                 multiply padding (tile = 256 hidden columns for kind 2, 256 output columns for 3) */
+                                 tile of 256 weight rows with the operands swapped, so that one pass over a weight
+                                 tile serves the whole group (tile = 256 hidden columns for kind 2, 256 output columns
+                                 for 3).  Issued only where a run's groups are fewer than its band pairs and the
+                                 schedule holds several such items per CTA pair. */
     int32_t *seg;             /* [segments][4] = {first band, bands, dest rank, rows} in schedule order */
     int32_t *tok_slot;        /* [R*T*min(k,El)] slots of each token's rows, ascending expert, -1 = none */
     float *tok_gate;          /* [R*T*min(k,El)] matching gates */

@@ -61,7 +61,8 @@ struct Params {
     int lag_items;      // schedule items between a band's last first-GEMM tile and its first second-GEMM tile
     int words;          // 32-bit words of one (expert, rank) token bitmap = ceil(T / 32)
     int n1, n2;         // tiles per band: F / 128 (0 for single-projection experts) and dout / 256
-    int swap_ok;        // small runs may use the swapped-operand items (needs F % 256 == 0 for FFN experts)
+    int swap_ok;        // runs of small groups may use the swapped-operand items (needs F % 256 == 0 for FFN experts):
+                        // 0 never, 1 where the plan's cost rule says so, 2 every eligible run (test hook)
     int max_bands, max_items;
     unsigned *epoch_rw;      // same word, for the plan kernel
     const unsigned *epoch;   // device word: number of this call; the plan kernel bumps it once per call

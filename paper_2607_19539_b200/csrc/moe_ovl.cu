@@ -229,7 +229,8 @@ Params make_params(moe_ovl_ctx *ctx)
     p.seg_slot0 = at<int>(ctx, L.seg_slot0); p.tok_slot = at<int>(ctx, L.tok_slot);
     p.tok_gate = at<float>(ctx, L.tok_gate); p.hcount = at<unsigned>(ctx, L.hcount);
     p.fcount = at<unsigned>(ctx, L.fcount);
-    p.swap_ok = !(c.flags & MOE_OVL_FLAG_NO_SMALL_GROUP_TILES) && (L.single || c.d_ffn % (2 * H_TILE) == 0);
+    p.swap_ok = (!(c.flags & MOE_OVL_FLAG_NO_SMALL_GROUP_TILES) && (L.single || c.d_ffn % (2 * H_TILE) == 0))
+                    ? ((c.flags & MOE_OVL_FLAG_TEST_ALL_SMALL_GROUP_TILES) ? 2 : 1) : 0;
     p.next_item = at<int>(ctx, L.next_item);
     p.plan_ticket = at<int>(ctx, L.next_item) + 1;
     p.next_seg = at<int>(ctx, L.next_item) + 2;

@@ -231,10 +231,21 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
         run_exp[run] = e;
         run_nb[run] = nbands;
         run_segs[run] = nsegs;
-        run_nsb[run] = (small && nbands > 0) ? sgroups : -1;
+        // Worth it only if the groups are fewer than the band pairs they replace: an MMA costs the same whether its
+        // 256 rows are two bands of tokens or 256 weight rows against one group of tokens.  (swap_ok == 2: a
+        // test hook that takes every eligible run.)
+        const bool fewer = sgroups < (nbands + 1) / 2 || p.swap_ok == 2;
+        run_nsb[run] = (small && nbands > 0 && fewer) ? sgroups : -1;
     }
     __syncthreads();
     if (tid == 0) {
+        // Groups make fewer, longer items than band pairs.  That pays when there are at least two such items per CTA pair;
+        // with few, the pairs that find no item idle while the long items run, and band pairs are faster.
+        int group_items = 0;
+        for (int run = 0; run < 2 * El; ++run)
+            if (run_nsb[run] >= 0) group_items += run_nsb[run] * (p.n1 / 2 + p.n2);
+        if (group_items < p.lag_items && p.swap_ok != 2)
+            for (int run = 0; run < 2 * El; ++run) run_nsb[run] = -1;
         int spos = 0, segoff = 0, sbcount = 0;
         for (int run = 0; run < 2 * El; ++run) {
             run_start[run] = spos;

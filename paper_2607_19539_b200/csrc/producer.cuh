@@ -393,173 +393,207 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
     };
 
     if (warp == 0) {
-        // ---------------- TMA producer (both CTAs)
-        if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            long long fills = 0;
-            bool ok = true;
-            // What the loads of one schedule item need.  It is looked up -- ring slot, item record, the counter the
-            // item depends on -- a few stages BEFORE the previous item's last load, so that these dependent
-            // round trips to L2 do not open a bubble between two items.
-            struct Job {
-                int it, a_row, b_row, ksteps, dep_index;
-                const CUtensorMap *amap, *bmap;
-                const unsigned *dep;        // counter that must reach dep_want before the item's first load
-                unsigned dep_want;
-                long long dep_site;
-                bool dep_ok;
-                // swapped-operand items: weight rows are the A side; nb bands of tokens the B side (table in
-                // shared memory, slot tab); gate and up projection take separate stage fills (fills = 2 * ksteps)
-                int swap, nb, tab, half_rows, w_row, w_row_up;
-                const CUtensorMap *tokmap;
-            };
-            volatile int2 *tabs = reinterpret_cast<volatile int2 *>(smem_gen + (swap_tab - smem_base));
-            // 1 = item n is in `j`, 0 = schedule exhausted, -1 = gave up
-            auto fetch = [&](int n, Job &j) -> int {
-                const int it = claimed(n);
-                if (it < 0) return -1;
-                if (it >= n_items) return 0;
-                if (rank == 0) mbar_arrive(bar_go);  // lets the scheduler claim the item after this one
-                const int4 item = p.items[it];       // {kind | expert << 8, band 0, band 1 or -1, tile}
-                const int kind = item.x & 0xff, e = item.x >> 8, tile = item.w;
-                j.it = it;
-                j.swap = kind >= KIND_G1S;
-                if (j.swap) {
-                    // {kind | expert << 8, first schedule position, bands | rows << 8, tile}
-                    j.nb = item.z & 0xff;
-                    j.tab = n & 1;
-                    j.half_rows = (item.z >> 8) / 2;
-                    const bool g1 = kind == KIND_G1S;
-                    if (g1) {
-                        // this CTA's 128 of the tile's 256 hidden columns: gate rows, and the matching up rows
-                        j.w_row = e * 2 * p.F + tile * 2 * H_TILE + (int)rank * H_TILE;
-                        j.w_row_up = j.w_row + p.F;
-                        j.amap = &maps.w1; j.tokmap = &maps.xa8; j.ksteps = p.d / TB_K;
-                    } else {
-                        j.w_row = e * p.dout + tile * TB_N + (int)rank * (TB_N / 2);
-                        j.w_row_up = j.w_row;
-                        j.amap = &maps.w2; j.tokmap = p.single ? &maps.xa8 : &maps.h8; j.ksteps = p.k2 / TB_K;
-                    }
-                    const bool on_x = g1 || p.n1 == 0;     // depends on gathered rows, else on finished hidden tiles
-                    j.dep_site = on_x ? SITE_TMA_XREADY : SITE_TMA_HCOUNT;
-                    j.dep_want = on_x ? (unsigned)TB_M : (unsigned)p.n1;
-                    j.dep_ok = true;
-                    for (int i = 0; i < j.nb; ++i) {
-                        const int b = p.sched_band[item.y + i];
-                        tabs[j.tab * SWAP_MAX_BANDS + i].x = b;
-                        tabs[j.tab * SWAP_MAX_BANDS + i].y = ceil16_rows(p.band_valid[b]) / 2;
-                        j.dep_ok = j.dep_ok && ld_acquire_u32(on_x ? &p.xready[b] : &p.hcount[b]) >= j.dep_want;
-                    }
-                    j.dep = on_x ? p.xready : p.hcount;
-                    return 1;
-                }
-                const int band = (rank == 0 || item.z < 0) ? item.y : item.z;
-                j.a_row = band * TB_M;
-                j.dep_index = band;
-                if (kind == KIND_G1) {
-                    j.amap = &maps.xa; j.bmap = &maps.w1;
-                    // rank 0 holds the gate-projection rows of the tile, rank 1 the matching up-projection rows
-                    j.b_row = e * 2 * p.F + tile * H_TILE + (int)rank * p.F;
-                    j.ksteps = p.d / TB_K;
-                    // all 128 rows of the band (padding included) must have been gathered into Xa
-                    j.dep = &p.xready[band]; j.dep_want = (unsigned)TB_M; j.dep_site = SITE_TMA_XREADY;
+        // ---------------- load warp (both CTAs).  Lane 0 looks the items up and issues the loads of band-pair
+        // items; for swapped-operand items, whose token side is many small boxes, lanes 1..8 issue one box each
+        // (one thread gets about one tensor copy per 0.1 us out of the door).
+        int stage = 0;
+        uint32_t phase = 0;
+        long long fills = 0;
+        bool ok = true;
+        // What the loads of one schedule item need.  It is looked up -- ring slot, item record, the counter the
+        // item depends on -- a few stages BEFORE the previous item's last load, so that these dependent
+        // round trips to L2 do not open a bubble between two items.
+        struct Job {
+            int it, a_row, b_row, ksteps, dep_index;
+            const CUtensorMap *amap, *bmap;
+            const unsigned *dep;        // counter that must reach dep_want before the item's first load
+            unsigned dep_want;
+            long long dep_site;
+            bool dep_ok;
+            // swapped-operand items: weight rows are the A side; nb bands of tokens the B side (table in
+            // shared memory, slot tab); gate and up projection take separate stage fills (fills = 2 * ksteps)
+            int swap, nb, tab, half_rows, w_row, w_row_up, tok_is_x;
+        };
+        volatile int2 *tabs = reinterpret_cast<volatile int2 *>(smem_gen + (swap_tab - smem_base));
+        // 1 = item n is in `j`, 0 = schedule exhausted, -1 = gave up.  Lane 0 only.
+        auto fetch = [&](int n, Job &j) -> int {
+            const int it = claimed(n);
+            if (it < 0) return -1;
+            if (it >= n_items) return 0;
+            if (rank == 0) mbar_arrive(bar_go);  // lets the scheduler claim the item after this one
+            const int4 item = p.items[it];       // {kind | expert << 8, band 0, band 1 or -1, tile}
+            const int kind = item.x & 0xff, e = item.x >> 8, tile = item.w;
+            j.it = it;
+            j.swap = kind >= KIND_G1S;
+            if (j.swap) {
+                // {kind | expert << 8, first schedule position, bands | rows << 8, tile}
+                j.nb = item.z & 0xff;
+                j.tab = n & 1;
+                j.half_rows = (item.z >> 8) / 2;
+                const bool g1 = kind == KIND_G1S;
+                if (g1) {
+                    // this CTA's 128 of the tile's 256 hidden columns: gate rows, and the matching up rows
+                    j.w_row = e * 2 * p.F + tile * 2 * H_TILE + (int)rank * H_TILE;
+                    j.w_row_up = j.w_row + p.F;
+                    j.amap = &maps.w1; j.tok_is_x = 1; j.ksteps = p.d / TB_K;
                 } else {
-                    // single-projection experts: the output GEMM reads the aligned input itself
-                    j.amap = p.single ? &maps.xa : &maps.h; j.bmap = &maps.w2;
-                    j.b_row = e * p.dout + tile * TB_N + (int)rank * (TB_N / 2);
-                    j.ksteps = p.k2 / TB_K;
-                    if (p.n1 > 0) {   // every first-GEMM tile of this band must have landed in H
-                        j.dep = &p.hcount[band]; j.dep_want = (unsigned)p.n1; j.dep_site = SITE_TMA_HCOUNT;
-                    } else {
-                        j.dep = &p.xready[band]; j.dep_want = (unsigned)TB_M; j.dep_site = SITE_TMA_XREADY;
-                    }
+                    j.w_row = e * p.dout + tile * TB_N + (int)rank * (TB_N / 2);
+                    j.w_row_up = j.w_row;
+                    j.amap = &maps.w2; j.tok_is_x = p.single; j.ksteps = p.k2 / TB_K;
                 }
-                j.dep_ok = ld_acquire_u32(j.dep) >= j.dep_want;      // the counters only grow
+                const bool on_x = g1 || p.n1 == 0;     // depends on gathered rows, else on finished hidden tiles
+                j.dep_site = on_x ? SITE_TMA_XREADY : SITE_TMA_HCOUNT;
+                j.dep_want = on_x ? (unsigned)TB_M : (unsigned)p.n1;
+                j.dep_ok = true;
+                for (int i = 0; i < j.nb; ++i) {
+                    const int b = p.sched_band[item.y + i];
+                    tabs[j.tab * SWAP_MAX_BANDS + i].x = b;
+                    tabs[j.tab * SWAP_MAX_BANDS + i].y = ceil16_rows(p.band_valid[b]) / 2;
+                    j.dep_ok = j.dep_ok && ld_acquire_u32(on_x ? &p.xready[b] : &p.hcount[b]) >= j.dep_want;
+                }
+                j.dep = on_x ? p.xready : p.hcount;
                 return 1;
-            };
-            Job cur, nxt;
-            int have = fetch(0, cur);
+            }
+            const int band = (rank == 0 || item.z < 0) ? item.y : item.z;
+            j.a_row = band * TB_M;
+            j.dep_index = band;
+            if (kind == KIND_G1) {
+                j.amap = &maps.xa; j.bmap = &maps.w1;
+                // rank 0 holds the gate-projection rows of the tile, rank 1 the matching up-projection rows
+                j.b_row = e * 2 * p.F + tile * H_TILE + (int)rank * p.F;
+                j.ksteps = p.d / TB_K;
+                // all 128 rows of the band (padding included) must have been gathered into Xa
+                j.dep = &p.xready[band]; j.dep_want = (unsigned)TB_M; j.dep_site = SITE_TMA_XREADY;
+            } else {
+                // single-projection experts: the output GEMM reads the aligned input itself
+                j.amap = p.single ? &maps.xa : &maps.h; j.bmap = &maps.w2;
+                j.b_row = e * p.dout + tile * TB_N + (int)rank * (TB_N / 2);
+                j.ksteps = p.k2 / TB_K;
+                if (p.n1 > 0) {   // every first-GEMM tile of this band must have landed in H
+                    j.dep = &p.hcount[band]; j.dep_want = (unsigned)p.n1; j.dep_site = SITE_TMA_HCOUNT;
+                } else {
+                    j.dep = &p.xready[band]; j.dep_want = (unsigned)TB_M; j.dep_site = SITE_TMA_XREADY;
+                }
+            }
+            j.dep_ok = ld_acquire_u32(j.dep) >= j.dep_want;      // the counters only grow
+            return 1;
+        };
+        Job cur, nxt;
+        cur.swap = 0;
+        int have = 0;
+        if (lane == 0) {
+            have = fetch(0, cur);
             ok = have >= 0;
-            for (int n = 0; ok && have == 1; ++n) {
-                if (!cur.dep_ok && cur.swap) {
+        }
+        for (int n = 0;; ++n) {
+            // item boundary: lanes 1..31 learn from lane 0 whether to go on and whether to help
+            __syncwarp();
+            const int go = __shfl_sync(0xffffffffu, (ok && have == 1) ? (cur.swap ? 2 : 1) : 0, 0);
+            if (go == 0) break;
+            if (go == 2) {
+                // ---- swapped-operand item, all lanes.  Stage fill = 128 weight rows (A slot, lane 0) + the
+                // group's token rows (B slot: this CTA's half of every band in boxes of 8 rows, lane 1 + box).
+                // First-GEMM items alternate gate and up rows against the same tokens.
+                if (lane == 0 && !cur.dep_ok) {
                     for (int i = 0; i < cur.nb && ok; ++i) {
                         const int b = tabs[cur.tab * SWAP_MAX_BANDS + i].x;
                         ok = wait_global(cur.dep + b, cur.dep_want, true, p, cur.dep_site, b);
                     }
-                    if (!ok) break;
-                } else if (!cur.dep_ok) {
-                    ok = wait_global(cur.dep, cur.dep_want, true, p, cur.dep_site, cur.dep_index);
-                    if (!ok) break;
                 }
                 asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
-                int have_next = 0;
-                if (cur.swap) {
-                    // Stage fill = 128 weight rows (A slot) + the group's token rows (B slot, this CTA's half of every
-                    // band, boxes of 8 rows).  First-GEMM items alternate gate and up rows against the same tokens.
-                    const int per_k = cur.w_row_up != cur.w_row ? 2 : 1, fills_item = per_k * cur.ksteps;
-                    const int look = fills_item > PROD_LOOKAHEAD ? fills_item - PROD_LOOKAHEAD : 0;
-                    const uint32_t tx = 2u * (uint32_t)(PROD_A_BYTES + cur.half_rows * TB_K * 2);
-                    for (int f = 0; f < fills_item; ++f) {
-                        const int ks = f / per_k;
-                        ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, p, SITE_TMA_EMPTY, cur.it);
-                        if (!ok) break;
-                        const uint32_t sa = smem_base + stage * PROD_STAGE_BYTES, sb = sa + PROD_A_BYTES;
-                        const uint32_t full = lead_full + 8 * stage;
-                        if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, tx);
-                        tma_load_2d(sa, cur.amap, full, ks * TB_K, (f % per_k) ? cur.w_row_up : cur.w_row);
-                        uint32_t dst = sb;
-                        for (int i = 0; i < cur.nb; ++i) {
-                            const int2 t = make_int2(tabs[cur.tab * SWAP_MAX_BANDS + i].x,
-                                                     tabs[cur.tab * SWAP_MAX_BANDS + i].y);
-                            const int row0 = t.x * TB_M + (int)rank * t.y;
-                            for (int r8 = 0; r8 < t.y; r8 += 8, dst += 8 * TB_K * 2)
-                                tma_load_2d(dst, cur.tokmap, full, ks * TB_K, row0 + r8);
-                        }
-                        ++fills;
-                        if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
-                        if (f == look) {
-                            have_next = fetch(n + 1, nxt);
-                            if (have_next < 0) { ok = false; break; }
-                        }
+                __syncwarp();
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                if (!ok) break;
+                const int nb = __shfl_sync(0xffffffffu, cur.nb, 0), tab = __shfl_sync(0xffffffffu, cur.tab, 0);
+                const int half_rows = __shfl_sync(0xffffffffu, cur.half_rows, 0);
+                const int ksteps = __shfl_sync(0xffffffffu, cur.ksteps, 0);
+                const int per_k = __shfl_sync(0xffffffffu, cur.w_row_up != cur.w_row ? 2 : 1, 0);
+                const int tok_is_x = __shfl_sync(0xffffffffu, cur.tok_is_x, 0);
+                const int it_now = __shfl_sync(0xffffffffu, cur.it, 0);
+                stage = __shfl_sync(0xffffffffu, stage, 0);
+                phase = __shfl_sync(0xffffffffu, phase, 0);
+                const CUtensorMap *tokmap = tok_is_x ? &maps.xa8 : &maps.h8;
+                // lane 1 + j owns box j of the B slot: which rows of which band are they?
+                int my_row = -1;
+                {
+                    int box0 = 0;
+                    for (int i = 0; i < nb; ++i) {
+                        const int b = tabs[tab * SWAP_MAX_BANDS + i].x, h = tabs[tab * SWAP_MAX_BANDS + i].y;
+                        const int j = lane - 1 - box0;
+                        if (j >= 0 && 8 * j < h) my_row = b * TB_M + (int)rank * h + 8 * j;
+                        box0 += h / 8;
                     }
-                    cur = nxt;
-                    have = have_next;
-                    continue;
                 }
-                const int look = cur.ksteps > PROD_LOOKAHEAD ? cur.ksteps - PROD_LOOKAHEAD : 0;
-                for (int ks = 0; ks < cur.ksteps; ++ks) {
-                    ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, p, SITE_TMA_EMPTY, cur.it);
-                    if (!ok) break;
+                const int fills_item = per_k * ksteps;
+                const int look = fills_item > PROD_LOOKAHEAD ? fills_item - PROD_LOOKAHEAD : 0;
+                const uint32_t tx = 2u * (uint32_t)(PROD_A_BYTES + half_rows * TB_K * 2);
+                int have_next = 0;
+                for (int f = 0; f < fills_item; ++f) {
+                    const int ks = f / per_k;
+                    bool fill_ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, p, SITE_TMA_EMPTY, it_now);
+                    fill_ok = __all_sync(0xffffffffu, fill_ok);
+                    if (!fill_ok) { ok = false; break; }
                     const uint32_t sa = smem_base + stage * PROD_STAGE_BYTES, sb = sa + PROD_A_BYTES;
                     const uint32_t full = lead_full + 8 * stage;
-                    // The leader announces the bytes of both CTAs.  The peer's bytes may land before this
-                    // arrival; the phase still cannot complete early because the arrival itself is pending.
-                    // The peer can only refill a stage after the leader's MMAs have consumed (hence completed)
-                    // its previous phase, so bytes never leak into the wrong phase.
-                    if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * PROD_STAGE_BYTES);
-                    tma_load_2d(sa, cur.amap, full, ks * TB_K, cur.a_row);
-                    tma_load_2d(sb, cur.bmap, full, ks * TB_K, cur.b_row);
-                    ++fills;
+                    if (lane == 0) {
+                        if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, tx);
+                        tma_load_2d(sa, cur.amap, full, ks * TB_K, (f % per_k) ? cur.w_row_up : cur.w_row);
+                        ++fills;
+                    } else if (my_row >= 0) {
+                        tma_load_2d(sb + (uint32_t)(lane - 1) * (8 * TB_K * 2), tokmap, full, ks * TB_K, my_row);
+                    }
                     if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
-                    if (ks == look) {
+                    if (f == look && lane == 0) {
                         have_next = fetch(n + 1, nxt);
-                        if (have_next < 0) { ok = false; break; }
+                        if (have_next < 0) ok = false;
                     }
                 }
-                cur = nxt;
-                have = have_next;
-            }
-            if (!ok && rank == 0) {
-                // give-up path: let the copies already issued land before the shared memory goes away
-                const long long pending = fills < PROD_STAGES ? fills : PROD_STAGES;
-                for (long long q = 1; q <= pending; ++q) {
-                    const long long f = fills - q;                       // index of an issued fill
-                    const int s = (int)(f % PROD_STAGES);
-                    const uint32_t par = (uint32_t)((f / PROD_STAGES) & 1);
-                    const unsigned long long t0 = globaltimer_ns();
-                    while (!mbar_try_wait(bar_full + 8 * s, par) && globaltimer_ns() - t0 < p.timeout_ns) {}
+                if (lane == 0) {
+                    cur = nxt;
+                    have = have_next;
                 }
+                continue;
+            }
+            if (lane != 0) continue;
+            // ---- band-pair item, lane 0
+            if (!cur.dep_ok) {
+                ok = wait_global(cur.dep, cur.dep_want, true, p, cur.dep_site, cur.dep_index);
+                if (!ok) continue;
+            }
+            asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
+            int have_next = 0;
+            const int look = cur.ksteps > PROD_LOOKAHEAD ? cur.ksteps - PROD_LOOKAHEAD : 0;
+            for (int ks = 0; ks < cur.ksteps; ++ks) {
+                ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, p, SITE_TMA_EMPTY, cur.it);
+                if (!ok) break;
+                const uint32_t sa = smem_base + stage * PROD_STAGE_BYTES, sb = sa + PROD_A_BYTES;
+                const uint32_t full = lead_full + 8 * stage;
+                // The leader announces the bytes of both CTAs.  The peer's bytes may land before this
+                // arrival; the phase still cannot complete early because the arrival itself is pending.
+                // The peer can only refill a stage after the leader's MMAs have consumed (hence completed)
+                // its previous phase, so bytes never leak into the wrong phase.
+                if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * PROD_STAGE_BYTES);
+                tma_load_2d(sa, cur.amap, full, ks * TB_K, cur.a_row);
+                tma_load_2d(sb, cur.bmap, full, ks * TB_K, cur.b_row);
+                ++fills;
+                if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
+                if (ks == look) {
+                    have_next = fetch(n + 1, nxt);
+                    if (have_next < 0) { ok = false; break; }
+                }
+            }
+            cur = nxt;
+            have = have_next;
+        }
+        if (lane == 0 && !ok && rank == 0) {
+            // give-up path: let the copies already issued land before the shared memory goes away
+            const long long pending = fills < PROD_STAGES ? fills : PROD_STAGES;
+            for (long long q = 1; q <= pending; ++q) {
+                const long long f = fills - q;                       // index of an issued fill
+                const int s = (int)(f % PROD_STAGES);
+                const uint32_t par = (uint32_t)((f / PROD_STAGES) & 1);
+                const unsigned long long t0 = globaltimer_ns();
+                while (!mbar_try_wait(bar_full + 8 * s, par) && globaltimer_ns() - t0 < p.timeout_ns) {}
             }
         }
     } else if (warp == 1) {

@@ -16,12 +16,12 @@ def _gpu():
     return torch, B, Hn
 
 
-def _run_case(shape, mode, csm, shuffle=None, mgb=1, group_bands=0, inp=None, dsp=None):
+def _run_case(shape, mode, csm, shuffle=None, mgb=1, group_bands=0, inp=None, dsp=None, flags=0):
     torch, B, Hn = _gpu()
     inp = inp or I.make_inputs(shape)
     dsp = dsp or I.dispatch(inp, shuffle_seed=shuffle)
     ctx = Hn.make_context(shape, max_rows=max(dsp.M, 1), mid_seg_bands=mgb, group_bands=group_bands,
-                          wait_timeout_us=2_000_000)
+                          wait_timeout_us=2_000_000, flags=flags)
     prob = Hn.upload(inp, dsp)
     Hn.run(ctx, prob, mode=mode, consumer_sm_count=csm)
     torch.cuda.synchronize()
@@ -39,7 +39,10 @@ SMALL = ["tiny", "tiny_zipf", "small", "small_zipf_rot", "single_small", "many_g
 def test_small_shapes_full_parity(name, mode, csm):
     torch, B, Hn = _gpu()
     shape = I.SHAPES[name]
-    inp, dsp, ctx, prob = _run_case(shape, mode, csm, shuffle=None if mode == 1 else 17)
+    # the small shapes hold too few items for the plan to choose swapped-operand items by itself: every other
+    # mode forces them onto all eligible runs
+    inp, dsp, ctx, prob = _run_case(shape, mode, csm, shuffle=None if mode == 1 else 17,
+                                    flags=B.FLAG_TEST_ALL_SMALL_GROUP_TILES if csm in (0, 8) else 0)
     plan = U.oracle_plan(shape, dsp)
     U.check_indices(shape, dsp, plan, ctx.moe_ovl_get_plan(), prob.slot_out.cpu().numpy(),
                     prob.rows_per_rank_out.cpu().numpy(), prob.segs_per_rank_out.cpu().numpy(),
@@ -83,7 +86,7 @@ def test_overlap_equals_non_overlap_bitwise(name):
         inp = I.make_inputs(I.with_seed(shape, seed))
         dsp = I.dispatch(inp)
         probs.append((inp, dsp))
-    ctx = Hn.make_context(shape, max_rows=max(d.M for _, d in probs))
+    ctx = Hn.make_context(shape, max_rows=max(d.M for _, d in probs), flags=B.FLAG_TEST_ALL_SMALL_GROUP_TILES)
     refs = []
     for inp, dsp in probs:
         base = Hn.upload(inp, dsp)
@@ -348,7 +351,8 @@ def test_random_shapes_full_parity(seed):
     gb = int(rng.choice([0, 2, 4, 5, 64]))
     inp = I.make_inputs(shape)
     dsp = I.dispatch(inp, shuffle_seed=int(rng.integers(0, 99)) if seed % 2 else None)
-    ctx = Hn.make_context(shape, max_rows=max(dsp.M, 1) + int(rng.integers(0, 300)), mid_seg_bands=mgb, group_bands=gb)
+    ctx = Hn.make_context(shape, max_rows=max(dsp.M, 1) + int(rng.integers(0, 300)), mid_seg_bands=mgb, group_bands=gb,
+                          flags=B.FLAG_TEST_ALL_SMALL_GROUP_TILES if seed % 3 else 0)
     prob = Hn.upload(inp, dsp)
     Hn.run(ctx, prob, mode=mode, consumer_sm_count=csm)
     torch.cuda.synchronize()
@@ -580,7 +584,7 @@ def test_small_group_items_can_be_switched_off(name):
     toks = np.arange(shape.R * shape.T)
     o = U.oracle_values(inp, toks)
     kinds = {}
-    for flags in (0, B.FLAG_NO_SMALL_GROUP_TILES):
+    for flags in (B.FLAG_TEST_ALL_SMALL_GROUP_TILES, B.FLAG_NO_SMALL_GROUP_TILES):
         ctx = Hn.make_context(shape, max_rows=dsp.M, flags=flags)
         prob = Hn.upload(inp, dsp)
         Hn.run(ctx, prob, mode=B.MODE_IN_KERNEL)
@@ -592,4 +596,5 @@ def test_small_group_items_can_be_switched_off(name):
         U.check_values(shape, dsp, plan, toks, *o, Hn.device_to_bits(prob.out), Hn.device_to_bits(prob.ret))
         kinds[flags] = set((gp["item"][:, 0] & 0xff).tolist())
     assert kinds[B.FLAG_NO_SMALL_GROUP_TILES] <= {0, 1}
-    assert kinds[0] & {2, 3}                      # every one of these problems has at least one run of small groups
+    # every one of these problems has at least one run of small groups
+    assert kinds[B.FLAG_TEST_ALL_SMALL_GROUP_TILES] & {2, 3}
