@@ -302,6 +302,14 @@ void choose_mode(const moe_ovl_ctx *ctx, int num_rows, int *mode, int *consumer_
     if (t_ded < best) { best = t_ded; *mode = MOE_OVL_MODE_OVERLAP; }
 }
 
+// Two builds of the GEMM kernel: the one with the trace bookkeeping compiled in runs only for contexts that asked
+// for a trace, so that the bookkeeping costs nothing otherwise.
+void launch_producer(int ctas, cudaStream_t st, const ProducerMaps &maps, const Params &p, int kflags)
+{
+    if (p.trace_items) producer_kernel<true><<<ctas, PROD_THREADS, PROD_SMEM_BYTES, st>>>(maps, p, kflags);
+    else producer_kernel<false><<<ctas, PROD_THREADS, PROD_SMEM_BYTES, st>>>(maps, p, kflags);
+}
+
 int sync_last(moe_ovl_ctx *ctx)
 {
     if (ctx->ran) CU_CHECK(ctx, cudaStreamSynchronize(ctx->last_stream));
@@ -395,7 +403,8 @@ int moe_ovl_create(moe_ovl_ctx **out, const moe_ovl_config *cfg, void *workspace
         CREATE_CHECK(cudaEventCreate(&ctx->h_p0[i]));
         CREATE_CHECK(cudaEventCreate(&ctx->h_p1[i]));
     }
-    CREATE_CHECK(cudaFuncSetAttribute(producer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PROD_SMEM_BYTES));
+    CREATE_CHECK(cudaFuncSetAttribute(producer_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PROD_SMEM_BYTES));
+    CREATE_CHECK(cudaFuncSetAttribute(producer_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PROD_SMEM_BYTES));
     CREATE_CHECK(cudaFuncSetAttribute(consumer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       CONSUMER_SMEM_BYTES));
     // grid-stride kernels get exactly one resident wave: a partial second wave would run at a fraction of the
@@ -549,7 +558,7 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
         // flags nobody can raise.  With both grids resident the order makes no difference.
         TIME_POINT(ctx->t_p0, ctx->s_prod);
         TIME_POINT(ctx->h_p0[hist], ctx->s_prod);
-        producer_kernel<<<prod_ctas, PROD_THREADS, PROD_SMEM_BYTES, ctx->s_prod>>>(maps, p, kflags);
+        launch_producer(prod_ctas, ctx->s_prod, maps, p, kflags);
         TIME_POINT(ctx->t_p1, ctx->s_prod);
         TIME_POINT(ctx->h_p1[hist], ctx->s_prod);
         CU_CHECK(ctx, cudaEventRecord(ctx->ev_prod_done, ctx->s_prod));
@@ -566,7 +575,7 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
         //      scatter kernel moves all rows.
         TIME_POINT(ctx->t_p0, st);
         TIME_POINT(ctx->h_p0[hist], st);
-        producer_kernel<<<prod_ctas, PROD_THREADS, PROD_SMEM_BYTES, st>>>(maps, p, kflags);
+        launch_producer(prod_ctas, st, maps, p, kflags);
         ++launches;
         TIME_POINT(ctx->t_p1, st);
         TIME_POINT(ctx->h_p1[hist], st);

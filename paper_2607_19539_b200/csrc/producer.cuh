@@ -321,6 +321,46 @@ __device__ __forceinline__ unsigned atom_add_acq_rel_u32(unsigned *p, unsigned v
     return old;
 }
 
+// Main loop of the MMA-issuing thread for one schedule item: per stage fill, wait for the operands, issue the
+// four K=16 MMAs of the 64-wide K slice, free the stage.  This thread's instruction stream is on the kernel's
+// critical path (a few dozen extra instructions per fill cost percents), so everything that varies is a
+// template parameter: kPerK = 2 for the swapped first GEMM, whose gate and up halves take separate fills and
+// accumulate in columns [0, ntok) and [ntok, 2 ntok); kTrace adds the wait-time bookkeeping of the trace.
+template <bool kTrace, int kPerK>
+__device__ __forceinline__ bool mma_mainloop(const Params &p, uint32_t smem_base, uint32_t bar_full, uint32_t bar_empty,
+                                             int &stage, uint32_t &phase, int ksteps, uint32_t d_tmem, uint32_t idesc,
+                                             int ntok, int it, unsigned long long &stall_ns,
+                                             unsigned long long &w_first)
+{
+    for (int kk = 0; kk < ksteps; ++kk) {
+#pragma unroll
+        for (int half = 0; half < kPerK; ++half) {
+            bool ok;
+            if (kTrace && !mbar_test_wait(bar_full + 8 * stage, phase)) {
+                const unsigned long long w0 = globaltimer_ns();
+                ok = mbar_wait(bar_full + 8 * stage, phase, p, SITE_MMA_FULL, it);
+                if (kk > 0 || half > 0) stall_ns += globaltimer_ns() - w0;   // the first fill is the item's start-up
+                else w_first = globaltimer_ns() - w0;
+            } else {
+                ok = mbar_wait(bar_full + 8 * stage, phase, p, SITE_MMA_FULL, it);
+            }
+            if (!ok) return false;
+            if (kTrace && kk == 0 && half == 0) p.trace_items[it].b = globaltimer_ns();
+            tc_fence_after();
+            const uint32_t sa = smem_base + stage * PROD_STAGE_BYTES, sb = sa + PROD_A_BYTES;
+            const uint64_t adesc = umma_smem_desc(sa), bdesc = umma_smem_desc(sb);
+            const uint32_t d_col = d_tmem + (uint32_t)(half * ntok);
+#pragma unroll
+            for (int k = 0; k < TB_K / 16; ++k)      // 16 bf16 = 32 bytes per MMA along K
+                umma_bf16(d_col, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kk | k) != 0 ? 1u : 0u);
+            umma_commit_pair(bar_empty + 8 * stage);  // both CTAs may refill the stage once it has been read
+            if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
+        }
+    }
+    return true;
+}
+
+template <bool kTrace>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PROD_THREADS, 1)
 producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const int kflags)
 {
@@ -609,12 +649,11 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 const int kind = item.x & 0xff;
                 const bool swap = kind >= KIND_G1S;
                 const bool first_gemm = kind == KIND_G1 || kind == KIND_G1S;
-                const int per_k = kind == KIND_G1S ? 2 : 1;           // gate and up rows take separate stage fills
-                const int ksteps = per_k * ((first_gemm ? p.d : p.k2) / TB_K);
+                const int ksteps = (first_gemm ? p.d : p.k2) / TB_K;
                 const int ntok = swap ? item.z >> 8 : 0;
                 const uint32_t idesc = swap ? umma_idesc_n(ntok) : UMMA_IDESC;
-                unsigned long long w_acc = 0, w_first = 0;    // trace only
-                if (p.trace_items && !mbar_try_wait_cluster(bar_tempty + 8 * acc, acc_phase ^ 1u)) {
+                unsigned long long w_acc = 0, w_first = 0, stall_ns = 0;    // trace only
+                if (kTrace && !mbar_try_wait_cluster(bar_tempty + 8 * acc, acc_phase ^ 1u)) {
                     const unsigned long long w0 = globaltimer_ns();
                     ok = mbar_wait<true>(bar_tempty + 8 * acc, acc_phase ^ 1u, p, SITE_MMA_TEMPTY, it);
                     w_acc = globaltimer_ns() - w0;
@@ -624,34 +663,14 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * TB_N;
-                unsigned long long stall_ns = 0;              // trace only: time spent waiting for operand stages
-                for (int ks = 0; ks < ksteps; ++ks) {
-                    if (p.trace_items && !mbar_test_wait(bar_full + 8 * stage, phase)) {
-                        const unsigned long long w0 = globaltimer_ns();
-                        ok = mbar_wait(bar_full + 8 * stage, phase, p, SITE_MMA_FULL, it);
-                        if (ks > 0) stall_ns += globaltimer_ns() - w0;   // the first stage is the item's start-up
-                        else w_first = globaltimer_ns() - w0;
-                    } else {
-                        ok = mbar_wait(bar_full + 8 * stage, phase, p, SITE_MMA_FULL, it);
-                    }
-                    if (!ok) break;
-                    if (ks == 0 && p.trace_items) p.trace_items[it].b = globaltimer_ns();
-                    tc_fence_after();
-                    const uint32_t sa = smem_base + stage * PROD_STAGE_BYTES, sb = sa + PROD_A_BYTES;
-                    const uint64_t adesc = umma_smem_desc(sa), bdesc = umma_smem_desc(sb);
-                    // swapped first GEMM: even fills accumulate the gate half in columns [0, ntok), odd fills the
-                    // up half in [ntok, 2 ntok)
-                    const uint32_t d_col = d_tmem + (uint32_t)((ks % per_k) * ntok);
-                    const int kk = ks / per_k;
-#pragma unroll
-                    for (int k = 0; k < TB_K / 16; ++k)      // 16 bf16 = 32 bytes per MMA along K
-                        umma_bf16(d_col, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
-                                  (kk | k) != 0 ? 1u : 0u);
-                    umma_commit_pair(bar_empty + 8 * stage);  // both CTAs may refill the stage once it has been read
-                    if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
-                }
+                if (kind == KIND_G1S)
+                    ok = mma_mainloop<kTrace, 2>(p, smem_base, bar_full, bar_empty, stage, phase, ksteps, d_tmem, idesc,
+                                                 ntok, it, stall_ns, w_first);
+                else
+                    ok = mma_mainloop<kTrace, 1>(p, smem_base, bar_full, bar_empty, stage, phase, ksteps, d_tmem, idesc,
+                                                 ntok, it, stall_ns, w_first);
                 if (!ok) break;
-                if (p.trace_items) {
+                if (kTrace) {
                     p.trace_item_aux[it].y = (int)stall_ns;
                     p.trace_items2[it].b = w_first;
                     p.trace_items2[it].c = w_acc;
@@ -674,7 +693,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 // latency is hidden and no role can fall a whole ring behind
                 if (n >= 1 && !mbar_wait(bar_go, (uint32_t)(n - 1) & 1u, p, SITE_SCHED_GO, n)) break;
                 const int it = atomicAdd(p.next_item, 1);
-                if (p.trace_items && it < n_items) {
+                if (kTrace && it < n_items) {
                     p.trace_items[it].a = globaltimer_ns();
                     p.trace_item_aux[it].x = (int)blockIdx.x;
                 }
@@ -746,7 +765,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             ok = epilogue_all(ok);
             if (!ok) break;
             tc_fence_after();
-            if (leader && rank == 0 && p.trace_items) p.trace_items2[it].a = globaltimer_ns();
+            if (kTrace && leader && rank == 0) p.trace_items2[it].a = globaltimer_ns();
             const uint32_t taddr = tmem_base + (uint32_t)acc * TB_N + ((uint32_t)(q * 32) << 16);
             const size_t grow = (size_t)(present ? band : 0) * TB_M + row;
             if (swap) {
@@ -835,7 +854,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             __threadfence();
             if (first_gemm) asm volatile("fence.proxy.async;" ::: "memory");   // H is re-read through TMA
             bar_sync_epilogue();
-            if (leader && present && p.trace_items) {
+            if (kTrace && leader && present) {
                 // taken before the release below, so that no observer of the flag can carry an earlier time
                 const unsigned long long now = globaltimer_ns();
                 if (rank == 0) p.trace_items[it].c = now; else p.trace_items[it].d = now;
