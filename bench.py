@@ -505,11 +505,6 @@ def main():
         ctx_lim = Hn.make_context(shape, max_rows=M, device=local_rank,
                                   producer_sm_limit=sms - ((args.consumer_sms + 1) & ~1))
         variants["non_overlap_restricted"] = (ctx_lim, B.MODE_NON_OVERLAP, 0)
-        # the overlapped modes with the weighted reduction kept as a kernel of its own after the return (the
-        # paper's arrangement): separates what hiding the return buys from what hiding the reduction buys
-        ctx_sep = Hn.make_context(shape, max_rows=M, device=local_rank, flags=B.FLAG_SEPARATE_COMBINE)
-        variants["in_kernel_separate_combine"] = (ctx_sep, B.MODE_IN_KERNEL, 0)
-        variants[f"overlap{args.consumer_sms}_separate_combine"] = (ctx_sep, B.MODE_OVERLAP, args.consumer_sms)
         names = list(variants)
 
         def run_variant(nm):
@@ -542,9 +537,7 @@ def main():
                    "vs_non_overlap": med[f"overlap{c}"] / nov} for c in csms]
         sweep.append({"mode": "auto", "chose_mode": rep_auto.mode_used, "chose_consumer_ctas": rep_auto.consumer_ctas,
                       "us_per_layer": med["auto"] * 1e3, "vs_non_overlap": med["auto"] / nov})
-        for nm in ("in_kernel_separate_combine", f"overlap{args.consumer_sms}_separate_combine"):
-            sweep.append({"mode": nm, "us_per_layer": med[nm] * 1e3, "vs_non_overlap": med[nm] / nov})
-        del ctx_lim, ctx_sep
+        del ctx_lim
 
     # ---- end to end through the host-buffer entry point: H2D of the step's inputs and D2H of out inside the timing
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()

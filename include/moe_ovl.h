@@ -53,10 +53,7 @@ enum {
 };
 
 enum {
-    MOE_OVL_MODE_OVERLAP = 0,     /* producer + consumer kernel on consumer_sm_count dedicated SMs (Section 3.3.3).  In this
-                                     mode and in IN_KERNEL the movers also form each rank's weighted sums (Section 2.1
-                                     step 5) as soon as the rank's last segment has landed, instead of a reduction
-                                     kernel after the return (MOE_OVL_FLAG_SEPARATE_COMBINE restores that kernel). */
+    MOE_OVL_MODE_OVERLAP = 0,     /* producer + consumer kernel on consumer_sm_count dedicated SMs (Section 3.3.3) */
     MOE_OVL_MODE_NON_OVERLAP = 1, /* comparison baseline of Section 4.1: GEMM to completion, then scatter */
     MOE_OVL_MODE_IN_KERNEL = 2,   /* same flag protocol and segments, but the finished segments are moved by spare
                                      warps inside the GEMM CTAs: no SM is taken from the GEMM, one kernel, nothing
@@ -102,9 +99,6 @@ typedef struct {
                                          (moe_ovl_get_trace); off by default, costs nothing when off */
 #define MOE_OVL_FLAG_NO_SMALL_GROUP_TILES 16u /* never issue the swapped-operand items that runs of small (expert, rank)
                                          groups otherwise get (see moe_ovl_plan_view.item); for comparisons */
-#define MOE_OVL_FLAG_SEPARATE_COMBINE 64u /* OVERLAP and IN_KERNEL: keep the weighted reduction a kernel of its own after
-                                         the return (as the paper does) instead of letting the movers form each rank's
-                                         sums as soon as the rank's last segment has landed; for comparisons */
 #define MOE_OVL_FLAG_TEST_ALL_SMALL_GROUP_TILES 32u /* test hook: every eligible run of small groups gets swapped-operand
                                          items, also where the plan's cost rule would keep band pairs */
 #define MOE_OVL_FLAG_TEST_SKIP_GATHER 8u /* test hook: the first band of the schedule is never gathered, so the GEMM's
@@ -180,7 +174,6 @@ typedef struct {
     float us_first_flag;      /* first output tile flagged: the consumer's window opens */
     float us_gemm_done;       /* last output tile flagged */
     float us_return_done;     /* last segment landed in ret */
-    float us_combine_done;    /* last weighted sum written, when the movers form them (0 otherwise) */
     float copy_gbs_per_cta;   /* returned bytes / time the moving CTAs spent inside segment copies: the rate one CTA
                                  sustains while the GEMM runs (GB/s, payload counted once) */
     float overlap_ratio;      /* share of the return window that lies before us_gemm_done:
@@ -283,18 +276,15 @@ int moe_ovl_read_buffer(moe_ovl_ctx *ctx, int32_t which, size_t offset, size_t b
  * equal row slices of it when spare warps of the GEMM CTAs move the return); times are nanoseconds of the
  * GPU's global timer after the first GEMM CTA started.  It is what the overlap ratio of Section 4.2.2, the
  * tail after the last tile and the idle time of the consumer (Section 3.3.3) are read from. */
-enum { MOE_OVL_TRACE_ITEM = 0, MOE_OVL_TRACE_UNIT = 1, MOE_OVL_TRACE_COMBINE = 2 };
+enum { MOE_OVL_TRACE_ITEM = 0, MOE_OVL_TRACE_UNIT = 1 };
 typedef struct {
-    int32_t kind;      /* MOE_OVL_TRACE_ITEM, MOE_OVL_TRACE_UNIT (a slice of a segment moved) or MOE_OVL_TRACE_COMBINE
-                          (a block of 32 tokens of one rank reduced by a mover) */
-    int32_t index;     /* item: position in issue order (moe_ovl_plan_view.item); unit: segment * chunks + chunk;
-                          combine: rank * ceil(T / 32) + block */
+    int32_t kind;      /* MOE_OVL_TRACE_ITEM / MOE_OVL_TRACE_UNIT */
+    int32_t index;     /* item: position in issue order (moe_ovl_plan_view.item); unit: segment * chunks + chunk */
     int32_t cta;       /* item: leader CTA of the pair that ran it; unit: CTA that moved it */
     int32_t who;       /* unit: 0 consumer CTA, 1 GEMM CTA that had run out of tiles, 2 spare warps of a GEMM CTA */
-    int32_t rows;      /* unit: rows moved; combine: tokens reduced */
+    int32_t rows;      /* unit: rows moved */
     int32_t chunks;    /* unit: slices per segment in this call */
-    int64_t ns_claim;  /* item: claimed by the pair's scheduler; unit: every ready flag of the segment seen; combine:
-                          every segment of the rank seen landed */
+    int64_t ns_claim;  /* item: claimed by the pair's scheduler; unit: every ready flag of the segment seen */
     int64_t ns_ready;  /* item: first operand stage landed, the MMAs can start; unit: same as ns_claim */
     int64_t ns_done0;  /* item: tile of the pair's first band published (flag or band counter), taken just
                           before the release store; unit: last row landed in the receive buffer */

@@ -24,8 +24,7 @@ FLAG_TRACE = 4
 FLAG_TEST_SKIP_GATHER = 8
 FLAG_NO_SMALL_GROUP_TILES = 16
 FLAG_TEST_ALL_SMALL_GROUP_TILES = 32
-FLAG_SEPARATE_COMBINE = 64
-TRACE_ITEM, TRACE_UNIT, TRACE_COMBINE = 0, 1, 2
+TRACE_ITEM, TRACE_UNIT = 0, 1
 BUF_XA, BUF_H, BUF_Y = 0, 1, 2
 TB_M, TB_N, H_TILE = 128, 256, 128
 
@@ -68,8 +67,7 @@ class Report(C.Structure):
                 ("timing_valid", C.c_int32), ("ms_total", C.c_float),
                 ("ms_prep", C.c_float), ("ms_expert_return", C.c_float), ("ms_producer", C.c_float),
                 ("ms_mover", C.c_float), ("ms_combine", C.c_float), ("us_first_flag", C.c_float),
-                ("us_gemm_done", C.c_float), ("us_return_done", C.c_float), ("us_combine_done", C.c_float),
-                ("copy_gbs_per_cta", C.c_float),
+                ("us_gemm_done", C.c_float), ("us_return_done", C.c_float), ("copy_gbs_per_cta", C.c_float),
                 ("overlap_ratio", C.c_float)]
 
 
@@ -217,7 +215,6 @@ class ReportView:
     copy_gbs_per_cta: float = 0.0
     mode_used: int = 0
     timing_valid: int = 1
-    us_combine_done: float = 0.0
 
 
 class MoeOvl:
@@ -281,7 +278,7 @@ class MoeOvl:
         return ReportView(r.padded_rows, r.num_bands, r.num_items, r.num_segments, r.producer_ctas, r.consumer_ctas,
                           r.kernel_launches, r.ms_total, r.ms_prep, r.ms_expert_return, r.ms_producer, r.ms_mover,
                           r.ms_combine, r.segments_by_gemm_ctas, r.us_first_flag, r.us_gemm_done, r.us_return_done,
-                          r.overlap_ratio, r.copy_gbs_per_cta, r.mode_used, r.timing_valid, r.us_combine_done)
+                          r.overlap_ratio, r.copy_gbs_per_cta, r.mode_used, r.timing_valid)
 
     def moe_ovl_get_plan(self) -> Dict[str, np.ndarray]:
         rep = self.moe_ovl_get_report()

@@ -13,8 +13,6 @@ constexpr int TB_N = 256;     // accumulator width of one tile (both GEMMs)
 constexpr int TB_K = 64;      // K extent of one pipeline stage: 64 bf16 = one 128-byte swizzle row
 constexpr int H_TILE = 128;   // hidden columns per first-GEMM tile (gate half + up half of the accumulator)
 
-constexpr int COMBINE_TOKENS = 32;   // tokens of one combine unit when the movers also do the weighted reduction
-
 constexpr int KIND_G1 = 0;    // x . W1 (gate | up) -> SiLU * up -> H
 constexpr int KIND_G2 = 1;    // H . W2 -> Y, raises the consumer-visible flag
 // The same two GEMMs with the operands swapped, for runs whose bands hold at most SMALL_BAND_ROWS valid rows each:
@@ -28,10 +26,10 @@ constexpr int SWAP_MAX_N = 128;
 constexpr int SWAP_MAX_BANDS = 8;          // SWAP_MAX_N / 16
 
 // meta[] slots written by the plan kernel
-enum { META_P = 0, META_BANDS, META_ITEMS, META_SEGS, META_SUPERBANDS, META_UNITS, META_COUNT = 8 };
+enum { META_P = 0, META_BANDS, META_ITEMS, META_SEGS, META_SUPERBANDS, META_COUNT = 8 };
 // stamps[] slots.  "first" stamps hold ~t so that the cleared state (0) is neutral under atomicMax.
 enum { STAMP_START_INV = 0, STAMP_FIRST_FLAG_INV, STAMP_LAST_FLAG, STAMP_LAST_SEG, STAMP_COPY_NS, STAMP_COPY_BYTES,
-       STAMP_LAST_COMBINE, STAMP_COUNT };
+       STAMP_COUNT };
 // status[] slots
 enum { ST_CODE = 0, ST_ABORT = 1, ST_DETAIL_LO = 2, ST_DETAIL_HI = 3, ST_COUNT = 4 };
 
@@ -44,7 +42,7 @@ constexpr int ERR_BAD_ROUTING = -6;
 // wait sites reported in the high bits of the status detail
 enum : long long {
     SITE_TMA_EMPTY = 1, SITE_TMA_HCOUNT, SITE_MMA_FULL, SITE_MMA_TEMPTY, SITE_EPI_TFULL, SITE_CONS_FLAG,
-    SITE_MMA_DRAIN, SITE_TMA_DRAIN, SITE_CLAIM, SITE_SCHED_GO, SITE_TMA_XREADY, SITE_COMBINE_RANK,
+    SITE_MMA_DRAIN, SITE_TMA_DRAIN, SITE_CLAIM, SITE_SCHED_GO, SITE_TMA_XREADY,
     SITE_ROW_RANGE = 16, SITE_ROW_DUP, SITE_COUNT_SUM, SITE_TOK_OVERFLOW, SITE_RET_OVERFLOW
 };
 
@@ -59,7 +57,6 @@ struct Params {
     int M;
     int mgb;            // bands per middle segment
     int seg_chunks;     // units a segment is moved in: 1 (whole segments), more when spare warps of GEMM CTAs move them
-    int fuse_combine;   // the movers also form the weighted sums, rank by rank as each rank's last segment lands
     int group_bands;    // bands interleaved in one super-band
     int lag_items;      // schedule items between a band's last first-GEMM tile and its first second-GEMM tile
     int words;          // 32-bit words of one (expert, rank) token bitmap = ceil(T / 32)
@@ -106,13 +103,6 @@ struct Params {
     unsigned *hcount;     // [max_bands] first-GEMM tiles finished per band
     unsigned *flags;      // [max_bands*n2] epoch of the call that finished the tile
     unsigned *fcount;     // [max_bands*n2] swapped-operand items: CTAs of the pair that have stored their half of the tile
-    // Unit stream of the movers when they also combine: ranks in the order in which their last segment comes up in
-    // the schedule; section i = the segments up to that one, then the combine units (COMBINE_TOKENS tokens each) of
-    // rank sec_rank[i].  sec_unit0[i] = first unit of section i, sec_unit0[R] = number of units.
-    int *rank_last;       // [R] 1 + index of the rank's last segment, 0 = none (cleared per call, built with atomicMax)
-    unsigned *rank_done;  // [R] units of the rank's segments that have landed (cleared per call)
-    int *rank_segs;       // [R] segments of the rank
-    int *sec_rank, *sec_seg_end, *sec_unit0;   // [R], [R], [R + 1]
     int *meta;            // [META_COUNT]
     // optional trace (null when off), raw %globaltimer values: one record per schedule item {claimed, first
     // operands landed, published by CTA 0 of the pair, published by CTA 1} plus trace_item_aux, and

@@ -30,13 +30,11 @@ inline size_t align_up(size_t v, size_t a = ALIGN) { return (v + a - 1) / a * a;
 struct Layout {
     // offsets into the workspace, in bytes
     size_t Xa, H, Y;
-    size_t zero_begin, bitmap, hcount, fcount, rank_last, rank_done, status, next_item, stamps, tok_slot, zero_end;   // cleared at the start of every call
+    size_t zero_begin, bitmap, hcount, fcount, status, next_item, stamps, tok_slot, zero_end;   // cleared at the start of every call
     size_t smid;
     size_t wordpfx, group_rows, group_start, group_slot, pos, slot, row_at, xready;
     size_t band_expert, band_dest, band_valid, band_slot0, sched_band, items, segs, seg_slot0;
     size_t tok_gate, flags, meta;
-    size_t rank_segs, sec_rank, sec_seg_end, sec_unit0;
-    long long max_units;
     size_t trace_items, trace_items2, trace_units, trace_item_aux, trace_bytes;   // MOE_OVL_FLAG_TRACE
     size_t sb[10];
     // host staging (MOE_OVL_FLAG_HOST_STAGING)
@@ -98,18 +96,12 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->bitmap = take((size_t)G * L->words * 4);
     L->hcount = take((size_t)L->max_bands * 4);
     L->fcount = take((size_t)L->max_bands * L->n2 * 4);
-    L->rank_last = take((size_t)c->num_src_ranks * 4);
-    L->rank_done = take((size_t)c->num_src_ranks * 4);
     L->status = take(ST_COUNT * 4);
     L->next_item = take(32);                 // next_item, plan_ticket, next_seg, assist_segs, next_gather
     L->stamps = take(STAMP_COUNT * 8);
     L->tok_slot = take(ntok * L->kmax * 4);
     L->zero_end = off;
     L->tok_gate = take(ntok * L->kmax * 4);
-    L->rank_segs = take((size_t)c->num_src_ranks * 4);
-    L->sec_rank = take((size_t)c->num_src_ranks * 4);
-    L->sec_seg_end = take((size_t)c->num_src_ranks * 4);
-    L->sec_unit0 = take((size_t)(c->num_src_ranks + 1) * 4);
     L->wordpfx = take((size_t)G * L->words * 4);
     L->group_rows = take((size_t)G * 4);
     L->group_start = take((size_t)G * 4);
@@ -132,14 +124,10 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     for (int i = 0; i < 10; ++i) L->sb[i] = take((size_t)L->max_bands * 4);
     L->st_ret_rows = (long long)c->tokens_per_rank * L->kmax;
     L->trace_bytes = 0;
-    // units of the movers: slices of segments (a segment per band at most) and the combine units of every rank
-    L->max_units = (long long)L->max_bands * MAX_SEG_CHUNKS +
-                   (long long)c->num_src_ranks * ((c->tokens_per_rank + COMBINE_TOKENS - 1) / COMBINE_TOKENS);
-    if (L->max_units > (1ll << 30)) return MOE_OVL_ERR_UNSUPPORTED;
     if (c->flags & MOE_OVL_FLAG_TRACE) {
         L->trace_items = take((size_t)L->max_items * sizeof(TraceRec));
         L->trace_items2 = take((size_t)L->max_items * sizeof(TraceRec));
-        L->trace_units = take((size_t)L->max_units * sizeof(TraceRec));
+        L->trace_units = take((size_t)L->max_bands * MAX_SEG_CHUNKS * sizeof(TraceRec));
         L->trace_item_aux = take((size_t)L->max_items * 8);
         L->trace_bytes = off - L->trace_items;
     }
@@ -241,9 +229,6 @@ Params make_params(moe_ovl_ctx *ctx)
     p.seg_slot0 = at<int>(ctx, L.seg_slot0); p.tok_slot = at<int>(ctx, L.tok_slot);
     p.tok_gate = at<float>(ctx, L.tok_gate); p.hcount = at<unsigned>(ctx, L.hcount);
     p.fcount = at<unsigned>(ctx, L.fcount);
-    p.rank_last = at<int>(ctx, L.rank_last); p.rank_done = at<unsigned>(ctx, L.rank_done);
-    p.rank_segs = at<int>(ctx, L.rank_segs); p.sec_rank = at<int>(ctx, L.sec_rank);
-    p.sec_seg_end = at<int>(ctx, L.sec_seg_end); p.sec_unit0 = at<int>(ctx, L.sec_unit0);
     p.swap_ok = (!(c.flags & MOE_OVL_FLAG_NO_SMALL_GROUP_TILES) && (L.single || c.d_ffn % (2 * H_TILE) == 0))
                     ? ((c.flags & MOE_OVL_FLAG_TEST_ALL_SMALL_GROUP_TILES) ? 2 : 1) : 0;
     p.next_item = at<int>(ctx, L.next_item);
@@ -516,9 +501,6 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     p.M = a->num_rows;
     p.lag_items = prod_ctas;                        // two rounds of the prod_ctas / 2 CTA pairs
     p.seg_chunks = in_kernel ? MAX_SEG_CHUNKS : 1;
-    // with movers at work (either kind) they also form the weighted sums, rank by rank; the comparison baseline
-    // keeps the reduction as a kernel of its own after the return
-    p.fuse_combine = mode != MOE_OVL_MODE_NON_OVERLAP && !(c.flags & MOE_OVL_FLAG_SEPARATE_COMBINE);
     p.ret_rows_per_rank = a->ret_rows_per_rank;
     p.x = static_cast<const uint16_t *>(a->x);
     p.expert_counts = a->expert_counts; p.src_rank = a->src_rank; p.src_token = a->src_token; p.gate = a->gate;
@@ -604,10 +586,8 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
         }
         TIME_POINT(ctx->t_m1, st);
     }
-    if (!p.fuse_combine) {
-        combine_kernel<<<ctx->combine_blocks_per_sm * ctx->num_sms, 256, 0, st>>>(p);
-        ++launches;
-    }
+    combine_kernel<<<ctx->combine_blocks_per_sm * ctx->num_sms, 256, 0, st>>>(p);
+    ++launches;
     CU_CHECK(ctx, cudaGetLastError());
     TIME_POINT(ctx->t_end, st);
 #undef TIME_POINT
@@ -742,7 +722,6 @@ int moe_ovl_get_report(moe_ovl_ctx *ctx, moe_ovl_report *r)
             r->us_first_flag = (float)((double)(first - t0) / 1e3);
             r->us_gemm_done = (float)((double)(st[STAMP_LAST_FLAG] - t0) / 1e3);
             r->us_return_done = (float)((double)(st[STAMP_LAST_SEG] - t0) / 1e3);
-            if (st[STAMP_LAST_COMBINE] != 0) r->us_combine_done = (float)((double)(st[STAMP_LAST_COMBINE] - t0) / 1e3);
             const double window = (double)r->us_return_done - r->us_first_flag;
             const double exposed = std::max(0.0, (double)r->us_return_done - r->us_gemm_done);
             r->overlap_ratio = window > 0 ? (float)(1.0 - exposed / window) : 1.0f;
@@ -854,7 +833,7 @@ int moe_ovl_get_trace(moe_ovl_ctx *ctx, void *host_buf, size_t bytes, size_t *wr
     CU_CHECK(ctx, cudaMemcpy(meta, ctx->ws + L.meta, sizeof(meta), cudaMemcpyDeviceToHost));
     CU_CHECK(ctx, cudaMemcpy(st, ctx->ws + L.stamps, sizeof(st), cudaMemcpyDeviceToHost));
     const size_t n_items = (size_t)meta[META_ITEMS];
-    const size_t n_units = ctx->last_mode == MOE_OVL_MODE_NON_OVERLAP ? 0 : (size_t)meta[META_UNITS];
+    const size_t n_units = ctx->last_mode == MOE_OVL_MODE_NON_OVERLAP ? 0 : (size_t)meta[META_SEGS] * ctx->last_chunks;
     const size_t need = (n_items + n_units) * sizeof(moe_ovl_trace_record);
     if (!host_buf) { *written = need; return MOE_OVL_OK; }
     if (bytes < need) return MOE_OVL_ERR_INVALID_ARG;
@@ -892,10 +871,8 @@ int moe_ovl_get_trace(moe_ovl_ctx *ctx, void *host_buf, size_t bytes, size_t *wr
         const TraceRec &t = items[n_items + u];
         moe_ovl_trace_record &r = out[n_items + u];
         std::memset(&r, 0, sizeof(r));
-        const int who_kind = (int32_t)(t.a >> 32);
-        r.kind = (who_kind >> 8) ? MOE_OVL_TRACE_COMBINE : MOE_OVL_TRACE_UNIT;
-        r.index = (int32_t)(t.d >> 32); r.cta = (int32_t)(t.a & 0xffffffffu);
-        r.who = who_kind & 0xff; r.rows = (int32_t)(t.d & 0xffffffffu); r.chunks = ctx->last_chunks;
+        r.kind = MOE_OVL_TRACE_UNIT; r.index = (int32_t)u; r.cta = (int32_t)(t.a & 0xffffffffu);
+        r.who = (int32_t)(t.a >> 32); r.rows = (int32_t)t.d; r.chunks = ctx->last_chunks;
         r.ns_claim = r.ns_ready = rel(t.b);
         r.ns_done0 = r.ns_done1 = rel(t.c);
     }

@@ -33,80 +33,11 @@ __device__ __forceinline__ void copy_rows_16B(const uint16_t *src, uint16_t *dst
     for (; v < nvec; v += nthr) __stcs(d + v, __ldcg(s + v));
 }
 
-// Weighted reduction of one token (Section 2.1 step 5): out[tok] = sum_j gate_j * ret[rank][slot_j], fp32, ascending
-// local expert, by a group of tpt threads (thread lt of the group handles 16-byte vectors lt, lt + tpt, ...).  cs / cg:
-// the token's first two list entries (slot + 1, 0 = none; gate).  kStrong: read the rows through L2 -- for callers
-// that run beside the kernel that writes them.
-template <bool kStrong>
-__device__ __forceinline__ void combine_token(const Params &p, int tok, const int (&cs)[2], const float (&cg)[2], int lt,
-                                              int tpt)
-{
-    constexpr int KFAST = 2;
-    const int nv = p.dout / 8;
-    const uint16_t *region = p.ret + (size_t)(tok / p.T) * p.ret_rows_per_rank * p.dout;
-    uint4 *o = reinterpret_cast<uint4 *>(p.out + (size_t)tok * p.dout);
-    auto ld = [](const uint4 *q) { return kStrong ? __ldcg(q) : __ldcs(q); };
-    // two 16-byte vectors per thread and iteration: all of their row loads are issued before any arithmetic
-    for (int v0 = lt; v0 < nv; v0 += 2 * tpt) {
-        const int v1 = v0 + tpt;
-        const bool has1 = v1 < nv;
-        uint4 row[2][KFAST];
-#pragma unroll
-        for (int j = 0; j < KFAST; ++j) {
-            const uint4 *src = reinterpret_cast<const uint4 *>(region + (size_t)(cs[j] > 0 ? cs[j] - 1 : 0) * p.dout);
-            row[0][j] = cs[j] > 0 ? ld(src + v0) : make_uint4(0, 0, 0, 0);
-            row[1][j] = (cs[j] > 0 && has1) ? ld(src + v1) : make_uint4(0, 0, 0, 0);
-        }
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int v = u == 0 ? v0 : v1;
-            if (u == 1 && !has1) break;
-            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            auto add = [&](const uint4 &q, float g) {
-                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    acc[2 * i] += g * __uint_as_float(w[i] << 16);
-                    acc[2 * i + 1] += g * __uint_as_float(w[i] & 0xffff0000u);
-                }
-            };
-            // ascending local expert; the list is dense, so the first empty entry (0) ends it
-            bool open = true;
-#pragma unroll
-            for (int j = 0; j < KFAST; ++j) {
-                open = open && cs[j] > 0;
-                if (open) add(row[u][j], cg[j]);
-            }
-            if (open) {
-                for (int j = KFAST; j < p.kmax; ++j) {        // tokens with more than two local rows
-                    const int s = p.tok_slot[(size_t)tok * p.kmax + j];
-                    if (s <= 0) break;
-                    add(ld(reinterpret_cast<const uint4 *>(region + (size_t)(s - 1) * p.dout) + v),
-                        p.tok_gate[(size_t)tok * p.kmax + j]);
-                }
-            }
-            uint32_t w[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(acc[2 * i + 1]), "f"(acc[2 * i]));
-            __stcs(o + v, make_uint4(w[0], w[1], w[2], w[3]));
-        }
-    }
-}
-
-// Threads per token: a power of two, about nv / 2 (two vectors per thread), between 32 and `limit`.
-__device__ __forceinline__ int combine_threads_per_token(int nv, int limit)
-{
-    int tpt = 256;
-    while (tpt > 32 && (tpt > nv / 2 || tpt > limit)) tpt >>= 1;
-    return tpt;
-}
-
 // A group of threads that moves segments: a whole CTA (barrier 0) or some warps of a GEMM CTA (their own
 // named barrier).  tid counts inside the group; the group's first warp claims and polls.
 struct MoverGroup {
     int tid, nthr, bar;
-    int *s_unit;          // eight ints of shared memory owned by the group
+    int *s_unit;          // two ints of shared memory owned by the group
     int who;              // TRACE_BY_* of the trace record
     __device__ __forceinline__ void sync() const
     {
@@ -114,25 +45,19 @@ struct MoverGroup {
     }
 };
 
-// Mover loop shared by the consumer CTAs, by GEMM CTAs that have run out of tiles and by the spare warps of GEMM
-// CTAs (in-kernel return): claim the next unit of the stream, wait (bounded, acquire) for what it depends on, do it.
-//   segment unit   one of p.seg_chunks equal row slices of a segment (1 = whole segments, the transfer unit of
-//                  Section 3.3.2): once every tile of every band of the segment is flagged, move the slice's valid
-//                  rows into the owner rank's receive buffer with one contiguous copy, then count it for the rank
-//   combine unit   (p.fuse_combine) COMBINE_TOKENS tokens of one rank: once every segment of that rank has landed,
-//                  form their gate-weighted sums (Section 2.1 step 5) -- the reduction the comparison baseline runs
-//                  as a kernel of its own after the return
-// Units are claimed in stream order: the segments in schedule order, each rank's combine units right behind the
-// rank's last segment.  A combine unit only waits for segment units that were claimed before it, a segment unit
-// only for the GEMM.  All threads of the group must call this together.
+// Segment mover shared by the consumer CTAs, by GEMM CTAs that have run out of tiles and by the spare warps of
+// GEMM CTAs (in-kernel return): claim the next unit in schedule order, wait (bounded, acquire) until every tile
+// of every band of its segment is flagged, then move the unit's valid rows into the owner rank's receive buffer
+// with one contiguous copy.  A unit is one of p.seg_chunks equal row slices of a segment (1 = whole segments,
+// the transfer unit of Section 3.3.2).  All threads of the group must call this together.
 __device__ __forceinline__ void move_segments(const Params &p, const MoverGroup &g)
 {
+    const int nseg = p.meta[META_SEGS];
     const int chunks = p.seg_chunks;
-    const int nunits = p.meta[META_UNITS];
+    const int nunits = nseg * chunks;
     const int lane = g.tid & 31;
     const unsigned epoch = *p.epoch;
     volatile int *s_unit = g.s_unit;
-    const int cu = (p.T + COMBINE_TOKENS - 1) / COMBINE_TOKENS;
     for (;;) {
         g.sync();
         if (g.tid < 32) {
@@ -140,95 +65,46 @@ __device__ __forceinline__ void move_segments(const Params &p, const MoverGroup 
             if (lane == 0) u = atomicAdd(p.next_seg, 1);
             u = __shfl_sync(0xffffffffu, u, 0);
             bool ok = true;
-            int kind = 0, a = 0, b = 0;          // segment unit: (segment, slice); combine unit: (rank, token block)
             if (u < nunits) {
-                int off = u, seg0 = 0;
-                if (p.fuse_combine) {
-                    // section = largest i with sec_unit0[i] <= u
-                    int lo = 0, hi = p.R;
-                    while (hi - lo > 1) {
-                        const int mid = (lo + hi) >> 1;
-                        if (p.sec_unit0[mid] <= u) lo = mid; else hi = mid;
-                    }
-                    seg0 = lo ? p.sec_seg_end[lo - 1] : 0;
-                    off = u - p.sec_unit0[lo];
-                    const int seg_units = (p.sec_seg_end[lo] - seg0) * chunks;
-                    if (off >= seg_units) { kind = 1; a = p.sec_rank[lo]; b = off - seg_units; }
-                }
-                if (kind == 0) {
-                    a = seg0 + off / chunks;
-                    b = off % chunks;
-                    const int4 seg = p.segs[a];          // {first band, bands, dest, rows}
-                    const int nflags = seg.y * p.n2;
-                    const unsigned *f = p.flags + (size_t)seg.x * p.n2;
-                    for (int i = lane; i < nflags && ok; i += 32)
-                        ok = wait_global(f + i, epoch, false, p, SITE_CONS_FLAG, (long long)seg.x * p.n2 + i, 2048);
-                } else if (lane == 0) {
-                    ok = wait_global(&p.rank_done[a], (unsigned)(p.rank_segs[a] * chunks), true, p, SITE_COMBINE_RANK, a,
-                                     2048);
-                }
+                const int4 seg = p.segs[u / chunks];          // {first band, bands, dest, rows}
+                const int nflags = seg.y * p.n2;
+                const unsigned *f = p.flags + (size_t)seg.x * p.n2;
+                for (int i = lane; i < nflags && ok; i += 32)
+                    ok = wait_global(f + i, epoch, false, p, SITE_CONS_FLAG, (long long)seg.x * p.n2 + i, 2048);
                 ok = __all_sync(0xffffffffu, ok);
             }
-            if (lane == 0) { s_unit[0] = u; s_unit[1] = ok ? 1 : 0; s_unit[2] = kind; s_unit[3] = a; s_unit[4] = b; }
+            if (lane == 0) { s_unit[0] = u; s_unit[1] = ok ? 1 : 0; }
         }
         g.sync();
         const int u = s_unit[0];
         if (u >= nunits || !s_unit[1]) return;
-        const int kind = s_unit[2], ua = s_unit[3], ub = s_unit[4];
-        const unsigned long long t_begin = globaltimer_ns();
-        int amount = 0;                                 // rows moved / tokens combined
-        if (kind == 0) {
-            const int4 seg = p.segs[ua];
-            const int per = (seg.w + chunks - 1) / chunks;         // rows per unit
-            const int r0 = ub * per, rows = min(per, seg.w - r0);
-            const long long slot0 = (long long)p.seg_slot0[ua] + r0;
-            amount = max(rows, 0);
-            // rows that would not fit into the rank's receive region (malformed routing, already reported) stay put
-            if (rows > 0 && slot0 + rows <= p.ret_rows_per_rank) {
-                const uint16_t *src = p.Y + ((size_t)seg.x * TB_M + r0) * p.dout;
-                uint16_t *dst = p.ret + ((size_t)seg.z * p.ret_rows_per_rank + slot0) * p.dout;
-                copy_rows_16B(src, dst, (size_t)rows * p.dout / 8, g.tid, g.nthr);
-            }
-            __threadfence();                            // the rows, before this unit is counted for its rank
-            g.sync();
-            if (g.tid == 0) {
-                red_release_add_u32(&p.rank_done[seg.z], 1u);
-                const unsigned long long now = globaltimer_ns();
-                stamp_max(&p.stamps[STAMP_LAST_SEG], now);
-                atomicAdd(&p.stamps[STAMP_COPY_NS], now - t_begin);                      // time one group spent copying
-                atomicAdd(&p.stamps[STAMP_COPY_BYTES], (unsigned long long)amount * p.dout * 2);
-                if (g.who != TRACE_BY_CONSUMER) atomicAdd(p.assist_segs, 1);
-            }
-        } else {
-            const int nv = p.dout / 8;
-            const int tpt = combine_threads_per_token(nv, 1 << (31 - __clz(g.nthr)));
-            const int sub = g.tid / tpt, lt = g.tid % tpt, per = g.nthr / tpt;
-            const int t0 = ub * COMBINE_TOKENS, t1 = min(p.T, t0 + COMBINE_TOKENS);
-            amount = t1 - t0;
-            if (sub < per) {
-                for (int t = t0 + sub; t < t1; t += per) {
-                    const int tok = ua * p.T + t;
-                    int cs[2];
-                    float cg[2];
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const bool use = j < p.kmax;
-                        cs[j] = use ? p.tok_slot[(size_t)tok * p.kmax + j] : 0;
-                        cg[j] = use ? p.tok_gate[(size_t)tok * p.kmax + j] : 0.f;
-                    }
-                    combine_token<true>(p, tok, cs, cg, lt, tpt);
-                }
-            }
-            g.sync();
-            if (g.tid == 0) stamp_max(&p.stamps[STAMP_LAST_COMBINE], globaltimer_ns());
+        const int s = u / chunks, c = u % chunks;
+        const int4 seg = p.segs[s];
+        const int per = (seg.w + chunks - 1) / chunks;         // rows per unit
+        const int r0 = c * per, rows = min(per, seg.w - r0);
+        const long long slot0 = (long long)p.seg_slot0[s] + r0;
+        const unsigned long long t_copy = globaltimer_ns();
+        // rows that would not fit into the rank's receive region (malformed routing, already reported) stay put
+        if (rows > 0 && slot0 + rows <= p.ret_rows_per_rank) {
+            const uint16_t *src = p.Y + ((size_t)seg.x * TB_M + r0) * p.dout;
+            uint16_t *dst = p.ret + ((size_t)seg.z * p.ret_rows_per_rank + slot0) * p.dout;
+            copy_rows_16B(src, dst, (size_t)rows * p.dout / 8, g.tid, g.nthr);
         }
-        if (g.tid == 0 && p.trace_units) {
-            TraceRec rec;
-            rec.a = ((unsigned long long)(unsigned)(g.who | (kind << 8)) << 32) | (unsigned)blockIdx.x;
-            rec.b = t_begin;                 // dependencies seen (every flag of the segment / every segment of the rank)
-            rec.c = globaltimer_ns();        // last row landed / last token written
-            rec.d = ((unsigned long long)(unsigned)(kind == 0 ? ua * chunks + ub : ua * cu + ub) << 32) | (unsigned)amount;
-            p.trace_units[u] = rec;
+        g.sync();
+        if (g.tid == 0) {
+            const unsigned long long now = globaltimer_ns();
+            stamp_max(&p.stamps[STAMP_LAST_SEG], now);
+            atomicAdd(&p.stamps[STAMP_COPY_NS], now - t_copy);                       // time one group spent copying
+            atomicAdd(&p.stamps[STAMP_COPY_BYTES], (unsigned long long)max(rows, 0) * p.dout * 2);
+            if (g.who != TRACE_BY_CONSUMER) atomicAdd(p.assist_segs, 1);
+            if (p.trace_units) {
+                TraceRec rec;
+                rec.a = ((unsigned long long)(unsigned)g.who << 32) | (unsigned)blockIdx.x;
+                rec.b = t_copy;                  // every flag of the segment seen
+                rec.c = now;                     // last row of the unit landed
+                rec.d = (unsigned long long)max(rows, 0);
+                p.trace_units[u] = rec;
+            }
         }
     }
 }
@@ -238,7 +114,7 @@ __device__ __forceinline__ void move_segments(const Params &p, const MoverGroup 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MOVER_THREADS, 1) consumer_kernel(const Params p)
 {
     extern __shared__ uint8_t unused_smem[];
-    __shared__ int s_unit[8];
+    __shared__ int s_unit[2];
     if (threadIdx.x == 0) p.smid_cons[blockIdx.x] = (int)smid();
     MoverGroup g{(int)threadIdx.x, (int)blockDim.x, 0, s_unit, TRACE_BY_CONSUMER};
     move_segments(p, g);
@@ -282,17 +158,65 @@ __global__ void __launch_bounds__(256) combine_kernel(const Params p)
             gate[j] = use ? __ldg(p.tok_gate + (size_t)tok * p.kmax + j) : 0.f;
         }
     };
-    const int tpt = combine_threads_per_token(nv, 256);
+    int tpt = 256;                                  // threads per token: power of two, about nv / 2
+    while (tpt > 32 && tpt > nv / 2) tpt >>= 1;
     const int sub = threadIdx.x / tpt, lt = threadIdx.x % tpt, per_block = blockDim.x / tpt;
     const int tok_stride = gridDim.x * per_block;
     fetch(blockIdx.x * per_block + sub);
     for (int tok = blockIdx.x * per_block + sub; tok < ntok; tok += tok_stride) {
+        const uint16_t *region = p.ret + (size_t)(tok / p.T) * p.ret_rows_per_rank * p.dout;
+        uint4 *o = reinterpret_cast<uint4 *>(p.out + (size_t)tok * p.dout);
         int cs[KFAST];
         float cg[KFAST];
 #pragma unroll
         for (int j = 0; j < KFAST; ++j) { cs[j] = slot[j]; cg[j] = gate[j]; }
         fetch(tok + tok_stride);
-        combine_token<false>(p, tok, cs, cg, lt, tpt);
+        // two 16-byte vectors per thread and iteration: all of their row loads are issued before any arithmetic
+        for (int v0 = lt; v0 < nv; v0 += 2 * tpt) {
+            const int v1 = v0 + tpt;
+            const bool has1 = v1 < nv;
+            uint4 row[2][KFAST];
+#pragma unroll
+            for (int j = 0; j < KFAST; ++j) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(region + (size_t)(cs[j] > 0 ? cs[j] - 1 : 0) * p.dout);
+                row[0][j] = cs[j] > 0 ? __ldcs(src + v0) : make_uint4(0, 0, 0, 0);
+                row[1][j] = (cs[j] > 0 && has1) ? __ldcs(src + v1) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int v = u == 0 ? v0 : v1;
+                if (u == 1 && !has1) break;
+                float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                auto add = [&](const uint4 &q, float g) {
+                    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        acc[2 * i] += g * __uint_as_float(w[i] << 16);
+                        acc[2 * i + 1] += g * __uint_as_float(w[i] & 0xffff0000u);
+                    }
+                };
+                // ascending local expert; the list is dense, so the first empty entry (0) ends it
+                bool open = true;
+#pragma unroll
+                for (int j = 0; j < KFAST; ++j) {
+                    open = open && cs[j] > 0;
+                    if (open) add(row[u][j], cg[j]);
+                }
+                if (open) {
+                    for (int j = KFAST; j < p.kmax; ++j) {        // tokens with more than two local rows
+                        const int s = p.tok_slot[(size_t)tok * p.kmax + j];
+                        if (s <= 0) break;
+                        add(__ldcs(reinterpret_cast<const uint4 *>(region + (size_t)(s - 1) * p.dout) + v),
+                            p.tok_gate[(size_t)tok * p.kmax + j]);
+                    }
+                }
+                uint32_t w[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(acc[2 * i + 1]), "f"(acc[2 * i]));
+                __stcs(o + v, make_uint4(w[0], w[1], w[2], w[3]));
+            }
+        }
     }
 }
 

@@ -299,7 +299,6 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
             const int rows = min(n[g] - first * TB_M, cnt * TB_M);
             p.segs[gsegoff[g] + q] = make_int4(gstart[g] / TB_M + first, cnt, r, rows);
             p.seg_slot0[gsegoff[g] + q] = gslot[g] + first * TB_M;
-            atomicMax(&p.rank_last[r], gsegoff[g] + q + 1);
         }
         if (lane == 0) p.group_rows[g] = n[g];
         if (lane == 1) p.group_start[g] = gstart[g];
@@ -352,34 +351,6 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
         }
     }
     __syncthreads();
-
-    // E2: unit stream of the movers when they also form the weighted sums (Section 2.1 step 5): a rank's tokens can
-    //     be combined as soon as its last segment has landed, so the combine units of every rank are placed right
-    //     after that segment in the order in which movers claim work.
-    {
-        const int chunks = p.seg_chunks, cu = (p.T + COMBINE_TOKENS - 1) / COMBINE_TOKENS;
-        for (int r = tid; r < R; r += blockDim.x) {
-            const int last = __ldcg(p.rank_last + r);     // built with atomics: read through L2
-            int order = 0;
-            for (int o = 0; o < R; ++o) {
-                const int lo = __ldcg(p.rank_last + o);
-                order += (lo < last) || (lo == last && o < r);
-            }
-            p.sec_rank[order] = r;
-            p.sec_seg_end[order] = last;
-            p.rank_segs[r] = segs_per_rank[r];
-        }
-        __threadfence_block();
-        __syncthreads();
-        for (int i = tid; i < R; i += blockDim.x)
-            p.sec_unit0[i] = (i ? p.sec_seg_end[i - 1] : 0) * chunks + i * cu;
-        if (tid == 0) {
-            const int nseg = p.meta[META_SEGS];
-            p.sec_unit0[R] = nseg * chunks + R * cu;
-            p.meta[META_UNITS] = p.fuse_combine ? nseg * chunks + R * cu : nseg * chunks;
-        }
-        __syncthreads();
-    }
 
     // F: issue order of tile blocks.  An item is a pair of bands times one tile.  Inside a super-band the tile
     //    index is the outer loop and the band pair the inner one, so that the CTA pairs working side by side

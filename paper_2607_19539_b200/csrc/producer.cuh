@@ -376,12 +376,12 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
     const uint32_t bar_go = tmem_slot + 8;                         // TMA thread -> scheduler: "started an item"
     const uint32_t bar_ring = bar_go + 8;                          // PROD_RING barriers: slot filled
     const uint32_t ring = bar_ring + 8 * PROD_RING;                // PROD_RING claimed item indices
-    const uint32_t mover_ints = ring + 4 * PROD_RING;              // eight ints of the in-kernel movers
+    const uint32_t mover_ints = ring + 4 * PROD_RING;              // two ints of the in-kernel movers
     // swapped-operand items: the load thread's band tables (this item and the next: band, rows per CTA) and the
     // epilogue's column -> buffer row maps (one per accumulator buffer, SWAP_MAX_N columns each)
-    const uint32_t swap_tab = mover_ints + 32;                     // [2][SWAP_MAX_BANDS] int2
+    const uint32_t swap_tab = mover_ints + 8;                      // [2][SWAP_MAX_BANDS] int2
     const uint32_t swap_rowmap = swap_tab + 2 * SWAP_MAX_BANDS * 8;   // [2][SWAP_MAX_N] int
-    static_assert(16 * PROD_STAGES + 16 + 16 + 8 + 8 + 8 + 8 * PROD_RING + 4 * PROD_RING + 32 + 2 * SWAP_MAX_BANDS * 8 +
+    static_assert(16 * PROD_STAGES + 16 + 16 + 8 + 8 + 8 + 8 * PROD_RING + 4 * PROD_RING + 8 + 2 * SWAP_MAX_BANDS * 8 +
                   2 * SWAP_MAX_N * 4 <= PROD_AUX_BYTES, "auxiliary shared memory");
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     volatile uint32_t *tmem_slot_gen = reinterpret_cast<volatile uint32_t *>(smem_gen + (tmem_slot - smem_base));
