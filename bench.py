@@ -591,7 +591,8 @@ def main():
             "rows": M, "padded_rows": rep.padded_rows, "tiles": rep.num_items, "segments": rep.num_segments,
             "producer_ctas": rep.producer_ctas, "consumer_ctas": rep.consumer_ctas, "mode_used": rep.mode_used,
             "overlap_ratio": statistics.mean(ovl_ratio) if ovl else None,
-            "segments_moved_by_gemm_ctas": statistics.mean(assist) if ovl else None,
+            "return_units": rep.return_units if ovl else None,
+            "return_units_moved_by_gemm_ctas": statistics.mean(assist) if ovl else None,
             "return_copy_gbs_per_cta": statistics.mean(copy_gbs) if ovl else None,
             "roofline": roofline, "burst": burst, "non_overlap": non_overlap, "consumer_sm_sweep": sweep,
             "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": rep.kernel_launches * args.steps,

@@ -159,8 +159,10 @@ typedef struct {
     int32_t producer_ctas;
     int32_t consumer_ctas;    /* 0 in NON_OVERLAP */
     int32_t kernel_launches;  /* kernels of this library launched by the call */
-    int32_t segments_by_gemm_ctas; /* segments (units) moved by GEMM CTAs: in OVERLAP those that had run out of
-                                      tiles, in IN_KERNEL all of them */
+    int32_t segments_by_gemm_ctas; /* units of the return (whole segments or slices, see return_units) moved by GEMM
+                                      CTAs: in OVERLAP by those that had run out of tiles, in IN_KERNEL all of them */
+    int32_t return_units;     /* units the return was moved in: a whole segment, or one of eight row slices of it (the
+                                 dedicated consumer slices the schedule's last 16 segments, the in-kernel movers all) */
     int32_t mode_used;        /* MOE_OVL_MODE_* the call ran in (differs from args->mode only for MODE_AUTO) */
     int32_t timing_valid;     /* 0 when the call was captured into a CUDA graph: the ms_* fields are then 0 (events
                                  recorded during capture carry no time); the us_* device stamps stay valid */
@@ -272,18 +274,19 @@ int moe_ovl_get_sm_map(moe_ovl_ctx *ctx, int32_t *producer_smid, int32_t *consum
 int moe_ovl_read_buffer(moe_ovl_ctx *ctx, int32_t which, size_t offset, size_t bytes, void *host_dst);
 
 /* Device trace of the last call (needs MOE_OVL_FLAG_TRACE).  One record per schedule item of the GEMM
- * kernel and one per moved unit of the return (a unit is a whole segment, or one of moe_ovl_report's
- * equal row slices of it when spare warps of the GEMM CTAs move the return); times are nanoseconds of the
+ * kernel and one per moved unit of the return (a unit is a whole segment or one of eight equal row slices of
+ * it, see `chunks` below); times are nanoseconds of the
  * GPU's global timer after the first GEMM CTA started.  It is what the overlap ratio of Section 4.2.2, the
  * tail after the last tile and the idle time of the consumer (Section 3.3.3) are read from. */
 enum { MOE_OVL_TRACE_ITEM = 0, MOE_OVL_TRACE_UNIT = 1 };
 typedef struct {
     int32_t kind;      /* MOE_OVL_TRACE_ITEM / MOE_OVL_TRACE_UNIT */
-    int32_t index;     /* item: position in issue order (moe_ovl_plan_view.item); unit: segment * chunks + chunk */
+    int32_t index;     /* item: position in issue order (moe_ovl_plan_view.item); unit: segment * 8 + slice */
     int32_t cta;       /* item: leader CTA of the pair that ran it; unit: CTA that moved it */
     int32_t who;       /* unit: 0 consumer CTA, 1 GEMM CTA that had run out of tiles, 2 spare warps of a GEMM CTA */
     int32_t rows;      /* unit: rows moved */
-    int32_t chunks;    /* unit: slices per segment in this call */
+    int32_t chunks;    /* unit: slices its segment is moved in: 1 (whole) or 8.  The dedicated consumer moves whole
+                          segments except the last 16 of the schedule; the spare warps of GEMM CTAs always slices */
     int64_t ns_claim;  /* item: claimed by the pair's scheduler; unit: every ready flag of the segment seen */
     int64_t ns_ready;  /* item: first operand stage landed, the MMAs can start; unit: same as ns_claim */
     int64_t ns_done0;  /* item: tile of the pair's first band published (flag or band counter), taken just

@@ -63,7 +63,8 @@ class HostArgs(C.Structure):
 class Report(C.Structure):
     _fields_ = [("padded_rows", C.c_int32), ("num_bands", C.c_int32), ("num_items", C.c_int32),
                 ("num_segments", C.c_int32), ("producer_ctas", C.c_int32), ("consumer_ctas", C.c_int32),
-                ("kernel_launches", C.c_int32), ("segments_by_gemm_ctas", C.c_int32), ("mode_used", C.c_int32),
+                ("kernel_launches", C.c_int32), ("segments_by_gemm_ctas", C.c_int32), ("return_units", C.c_int32),
+                ("mode_used", C.c_int32),
                 ("timing_valid", C.c_int32), ("ms_total", C.c_float),
                 ("ms_prep", C.c_float), ("ms_expert_return", C.c_float), ("ms_producer", C.c_float),
                 ("ms_mover", C.c_float), ("ms_combine", C.c_float), ("us_first_flag", C.c_float),
@@ -215,6 +216,7 @@ class ReportView:
     copy_gbs_per_cta: float = 0.0
     mode_used: int = 0
     timing_valid: int = 1
+    return_units: int = 0
 
 
 class MoeOvl:
@@ -278,7 +280,7 @@ class MoeOvl:
         return ReportView(r.padded_rows, r.num_bands, r.num_items, r.num_segments, r.producer_ctas, r.consumer_ctas,
                           r.kernel_launches, r.ms_total, r.ms_prep, r.ms_expert_return, r.ms_producer, r.ms_mover,
                           r.ms_combine, r.segments_by_gemm_ctas, r.us_first_flag, r.us_gemm_done, r.us_return_done,
-                          r.overlap_ratio, r.copy_gbs_per_cta, r.mode_used, r.timing_valid)
+                          r.overlap_ratio, r.copy_gbs_per_cta, r.mode_used, r.timing_valid, r.return_units)
 
     def moe_ovl_get_plan(self) -> Dict[str, np.ndarray]:
         rep = self.moe_ovl_get_report()

@@ -56,7 +56,8 @@ struct Params {
     int single;         // single-projection experts: no first GEMM, the output GEMM reads Xa
     int M;
     int mgb;            // bands per middle segment
-    int seg_chunks;     // units a segment is moved in: 1 (whole segments), more when spare warps of GEMM CTAs move them
+    int seg_chunks;     // equal row slices a sliced segment is moved in
+    int tail_segs;      // how many of the schedule's LAST segments are sliced (-1: all of them); the others are moved whole
     int group_bands;    // bands interleaved in one super-band
     int lag_items;      // schedule items between a band's last first-GEMM tile and its first second-GEMM tile
     int words;          // 32-bit words of one (expert, rank) token bitmap = ceil(T / 32)

@@ -167,7 +167,7 @@ struct moe_ovl_ctx {
     unsigned long long calls;
     cudaStream_t last_stream;
     bool ran;
-    int last_mode, last_prod_ctas, last_cons_ctas, last_launches, last_rows, last_chunks;
+    int last_mode, last_prod_ctas, last_cons_ctas, last_launches, last_rows, last_chunks, last_tail_segs;
     bool last_timed;                                  // false when the last call was captured into a graph
     bool hist_timed[MOE_OVL_TIMING_HISTORY];
     int last_cuda_error;
@@ -244,7 +244,8 @@ Params make_params(moe_ovl_ctx *ctx)
     p.flags = at<unsigned>(ctx, L.flags);
     p.epoch_rw = at<unsigned>(ctx, L.meta) + META_COUNT;     // the word after meta[], cleared at creation only
     p.epoch = p.epoch_rw; p.meta = at<int>(ctx, L.meta); p.status = at<int>(ctx, L.status);
-    p.seg_chunks = 1;
+    p.seg_chunks = MAX_SEG_CHUNKS;
+    p.tail_segs = 0;
     if (c.flags & MOE_OVL_FLAG_TRACE) {
         p.trace_items = at<TraceRec>(ctx, L.trace_items);
         p.trace_units = at<TraceRec>(ctx, L.trace_units);
@@ -500,7 +501,8 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     Params p = make_params(ctx);
     p.M = a->num_rows;
     p.lag_items = prod_ctas;                        // two rounds of the prod_ctas / 2 CTA pairs
-    p.seg_chunks = in_kernel ? MAX_SEG_CHUNKS : 1;
+    p.seg_chunks = MAX_SEG_CHUNKS;
+    p.tail_segs = in_kernel ? -1 : p.group_bands;       // dedicated consumer: whole segments but for the last super-band's
     p.ret_rows_per_rank = a->ret_rows_per_rank;
     p.x = static_cast<const uint16_t *>(a->x);
     p.expert_counts = a->expert_counts; p.src_rank = a->src_rank; p.src_token = a->src_token; p.gate = a->gate;
@@ -603,6 +605,7 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     ctx->last_launches = launches;
     ctx->last_rows = p.M;
     ctx->last_chunks = p.seg_chunks;
+    ctx->last_tail_segs = p.tail_segs;
     return MOE_OVL_OK;
 }
 
@@ -700,6 +703,11 @@ int moe_ovl_get_report(moe_ovl_ctx *ctx, moe_ovl_report *r)
     r->consumer_ctas = ctx->last_cons_ctas;
     r->kernel_launches = ctx->last_launches;
     r->mode_used = ctx->last_mode;
+    if (ctx->last_mode != MOE_OVL_MODE_NON_OVERLAP) {
+        const int nseg = meta[META_SEGS];
+        const int whole = ctx->last_tail_segs < 0 ? 0 : std::max(0, nseg - ctx->last_tail_segs);
+        r->return_units = whole + (nseg - whole) * ctx->last_chunks;
+    }
     r->timing_valid = ctx->last_timed ? 1 : 0;
     if (ctx->last_timed) {
         float prod_end = 0.f, mover_end = 0.f;
@@ -833,7 +841,9 @@ int moe_ovl_get_trace(moe_ovl_ctx *ctx, void *host_buf, size_t bytes, size_t *wr
     CU_CHECK(ctx, cudaMemcpy(meta, ctx->ws + L.meta, sizeof(meta), cudaMemcpyDeviceToHost));
     CU_CHECK(ctx, cudaMemcpy(st, ctx->ws + L.stamps, sizeof(st), cudaMemcpyDeviceToHost));
     const size_t n_items = (size_t)meta[META_ITEMS];
-    const size_t n_units = ctx->last_mode == MOE_OVL_MODE_NON_OVERLAP ? 0 : (size_t)meta[META_SEGS] * ctx->last_chunks;
+    const size_t nseg = (size_t)meta[META_SEGS];
+    const size_t whole = ctx->last_tail_segs < 0 ? 0 : (nseg > (size_t)ctx->last_tail_segs ? nseg - ctx->last_tail_segs : 0);
+    const size_t n_units = ctx->last_mode == MOE_OVL_MODE_NON_OVERLAP ? 0 : whole + (nseg - whole) * ctx->last_chunks;
     const size_t need = (n_items + n_units) * sizeof(moe_ovl_trace_record);
     if (!host_buf) { *written = need; return MOE_OVL_OK; }
     if (bytes < need) return MOE_OVL_ERR_INVALID_ARG;
@@ -871,8 +881,8 @@ int moe_ovl_get_trace(moe_ovl_ctx *ctx, void *host_buf, size_t bytes, size_t *wr
         const TraceRec &t = items[n_items + u];
         moe_ovl_trace_record &r = out[n_items + u];
         std::memset(&r, 0, sizeof(r));
-        r.kind = MOE_OVL_TRACE_UNIT; r.index = (int32_t)u; r.cta = (int32_t)(t.a & 0xffffffffu);
-        r.who = (int32_t)(t.a >> 32); r.rows = (int32_t)t.d; r.chunks = ctx->last_chunks;
+        r.kind = MOE_OVL_TRACE_UNIT; r.index = (int32_t)(t.d >> 32); r.cta = (int32_t)(t.a & 0xffffffffu);
+        r.who = (int32_t)(t.a >> 32); r.rows = (int32_t)(t.d & 0xffffffu); r.chunks = (int32_t)((t.d >> 24) & 0xff);
         r.ns_claim = r.ns_ready = rel(t.b);
         r.ns_done0 = r.ns_done1 = rel(t.c);
     }

@@ -48,13 +48,17 @@ struct MoverGroup {
 // Segment mover shared by the consumer CTAs, by GEMM CTAs that have run out of tiles and by the spare warps of
 // GEMM CTAs (in-kernel return): claim the next unit in schedule order, wait (bounded, acquire) until every tile
 // of every band of its segment is flagged, then move the unit's valid rows into the owner rank's receive buffer
-// with one contiguous copy.  A unit is one of p.seg_chunks equal row slices of a segment (1 = whole segments,
-// the transfer unit of Section 3.3.2).  All threads of the group must call this together.
+// with one contiguous copy.  A unit is a whole segment (the transfer unit of Section 3.3.2) or one of
+// p.seg_chunks equal row slices of it: the dedicated consumer moves whole segments, except the last p.tail_segs of
+// the schedule, whose tiles finish together at the very end of the GEMM -- sliced, they spread over every CTA
+// that is free by then instead of keeping p.tail_segs CTAs busy for a whole segment each; the spare warps of the
+// GEMM CTAs move slices throughout.  All threads of the group must call this together.
 __device__ __forceinline__ void move_segments(const Params &p, const MoverGroup &g)
 {
     const int nseg = p.meta[META_SEGS];
     const int chunks = p.seg_chunks;
-    const int nunits = nseg * chunks;
+    const int whole = p.tail_segs < 0 ? 0 : max(0, nseg - p.tail_segs);       // leading segments moved whole
+    const int nunits = whole + (nseg - whole) * chunks;
     const int lane = g.tid & 31;
     const unsigned epoch = *p.epoch;
     volatile int *s_unit = g.s_unit;
@@ -66,7 +70,7 @@ __device__ __forceinline__ void move_segments(const Params &p, const MoverGroup 
             u = __shfl_sync(0xffffffffu, u, 0);
             bool ok = true;
             if (u < nunits) {
-                const int4 seg = p.segs[u / chunks];          // {first band, bands, dest, rows}
+                const int4 seg = p.segs[u < whole ? u : whole + (u - whole) / chunks];   // {first band, bands, dest, rows}
                 const int nflags = seg.y * p.n2;
                 const unsigned *f = p.flags + (size_t)seg.x * p.n2;
                 for (int i = lane; i < nflags && ok; i += 32)
@@ -78,9 +82,10 @@ __device__ __forceinline__ void move_segments(const Params &p, const MoverGroup 
         g.sync();
         const int u = s_unit[0];
         if (u >= nunits || !s_unit[1]) return;
-        const int s = u / chunks, c = u % chunks;
+        const int s = u < whole ? u : whole + (u - whole) / chunks, c = u < whole ? 0 : (u - whole) % chunks;
+        const int my_chunks = u < whole ? 1 : chunks;
         const int4 seg = p.segs[s];
-        const int per = (seg.w + chunks - 1) / chunks;         // rows per unit
+        const int per = (seg.w + my_chunks - 1) / my_chunks;   // rows per unit
         const int r0 = c * per, rows = min(per, seg.w - r0);
         const long long slot0 = (long long)p.seg_slot0[s] + r0;
         const unsigned long long t_copy = globaltimer_ns();
@@ -102,7 +107,8 @@ __device__ __forceinline__ void move_segments(const Params &p, const MoverGroup 
                 rec.a = ((unsigned long long)(unsigned)g.who << 32) | (unsigned)blockIdx.x;
                 rec.b = t_copy;                  // every flag of the segment seen
                 rec.c = now;                     // last row of the unit landed
-                rec.d = (unsigned long long)max(rows, 0);
+                rec.d = ((unsigned long long)(unsigned)(s * chunks + c) << 32) | ((unsigned long long)my_chunks << 24) |
+                        (unsigned long long)max(rows, 0);
                 p.trace_units[u] = rec;
             }
         }

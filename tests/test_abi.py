@@ -29,7 +29,7 @@ def test_struct_sizes_match_header_layout():
     # field-by-field mirror of the header; sizes are what the library checks in struct_size
     assert ctypes.sizeof(B.Config) == 16 * 4
     assert ctypes.sizeof(B.Args) == 8 + 7 * 8 + 8 + 8 + 8 + 8 + 3 * 8 + 8
-    assert ctypes.sizeof(B.Report) == 10 * 4 + 11 * 4
+    assert ctypes.sizeof(B.Report) == 11 * 4 + 11 * 4
     assert ctypes.sizeof(B.TraceRecord) == 6 * 4 + 8 * 8 == B.TRACE_DTYPE.itemsize
 
 
