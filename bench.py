@@ -225,10 +225,14 @@ def run_reference(args, shape):
 
 def workload_config(shape, args):
     kind = f"one projection N={shape.N_out}" if shape.N_out else f"ffn={shape.F}"
+    wbytes = 2 * shape.El * shape.d * (shape.N_out if shape.N_out else 3 * shape.F)
+    abytes = 2 * shape.R * shape.T * (shape.d + shape.dout)
+    l2 = ("inputs larger than L2 (weights + activations >> 126 MB), no flush" if wbytes + abytes > 2 * 126e6 else
+          "working set fits in the 126 MB L2 and is not flushed: warm-cache, launch-bound numbers")
     return {"workload": f"{shape.name}: {shape.R} simulated ranks x {shape.T} tokens, {shape.Eg} experts "
                         f"top-{shape.k}, {shape.El} local, d={shape.d}, {kind}, {shape.router} router",
             "consumer_sms": args.consumer_sms, "mode": getattr(args, "mode", "overlap"), "seed": shape.seed,
-            "l2": "inputs larger than L2 (weights + activations >> 126 MB), no flush",
+            "l2": l2,
             "preheat_s": PREHEAT_S,
             "parallelism": f"replicas x{args.gpus}" if args.gpus > 1 else "single GPU"}
 
