@@ -3,6 +3,7 @@
 //                    order, polls its ready flags and moves its valid rows into the owner
 //                    rank's receive buffer with one contiguous copy (Section 3.3.2-3.3.3);
 //                    GEMM CTAs that run out of tiles join in, which removes the tail
+//   move_segments    that loop; also run by spare warps of the GEMM CTAs (in-kernel return)
 //   scatter_kernel   the non-overlap comparison: all bands, whole GPU, after the GEMM
 //   combine_kernel   out[r,t] = sum_j gate_j * ret[r][slot_j]  (Section 2.1 step 5)
 // All three are HBM/L2-bandwidth work: 16-byte coalesced loads and stores.

@@ -1,6 +1,6 @@
 // Plan kernels: remote-owner-aligned row layout and remote-first tile schedule
-// (Algorithm 1), combine plan (Section 3.2.3), segments (Section 3.3.2, Figure 3b),
-// and the gather of the dispatched rows into the aligned layout.
+// (Algorithm 1), combine plan (Section 3.2.3), segments (Section 3.3.2, Figure 3b), the
+// item list the GEMM kernel follows, and the maps its gather warps need.
 //
 // All integer work.  Rank-in-group is found without sorting: a routed copy is
 // identified by (expert, owner rank, token), so every (expert, rank) group gets a

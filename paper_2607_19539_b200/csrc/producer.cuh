@@ -7,15 +7,18 @@
 // as clusters of two that share every MMA (cta_group::2): the pair computes a 256 x 256 tile,
 // each CTA holding its own 128 rows of A and only HALF of the B tile, which cuts the operand
 // traffic from L2 per SM by a third against a single-CTA 128 x 256 tile.
-//   warp 0     TMA loads (cp.async.bulk.tensor, 128-byte swizzle) into a 7-stage ring; both
-//              CTAs' loads complete on the leader CTA's mbarrier
+//   warp 0     TMA loads (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a 7-stage ring;
+//              both CTAs' loads complete on the leader CTA's mbarrier.  It looks its next item up a few
+//              stages before the current item's last load.
 //   warp 1     in the leader CTA one thread issues tcgen05.mma (bf16 x bf16 -> fp32, M=256
 //              N=256 K=16); accumulators in tensor memory, double buffered (2 x 256 columns)
 //   warps 2-5  epilogue: tcgen05.ld -> fp32 math -> bf16 -> global, then publish
 //   warps 7-10 gather: move the dispatched rows into the aligned layout Xa (Section 3.2.1) band by band in
 //              schedule order while the tensor cores work, and count finished rows per band; the TMA warp
 //              waits for a band's count before its first load.  The layout pass therefore costs no time
-//              of its own except for the first few bands.
+//              of its own except for the first few bands.  With the in-kernel return (PROD_WARP_MOVERS)
+//              the same warps, once Xa is complete, take over the consumer's job on this SM: they claim
+//              finished segments and move them into the receive buffers, so that no SM is set aside.
 //   warp 6     scheduler (leader CTA): claims the next schedule item with an atomic counter, one
 //              item ahead of the TMA warp, and hands it to every role of both CTAs through a
 //              small ring in shared memory.  Items are claimed in schedule order, so the
@@ -27,6 +30,10 @@
 //                c+128: h = silu(g) * u, 128 columns of H; then hcount[band] += 1 (release)
 //   second GEMM  waits until hcount[band] == F/128, A = H[band], B = 256 rows of W2 (128 per
 //                rank), writes 256 columns of Y; then flag[band][tile] = epoch (release)
+// Runs of small (expert, rank) groups may come as items with the operands swapped (KIND_G1S / KIND_G2S):
+// 256 weight rows on the MMA's M side, the valid rows of a group of up to 8 small bands on its N side,
+// transposed epilogue (lane = output column); see common.cuh and the plan kernel's cost rule.
+// The kernel exists in two builds: kTrace = true adds the per-item bookkeeping of the device trace.
 // Every wait is bounded; on a give-up the CTA records a status, drains its copies,
 // frees its tensor memory and returns.
 #pragma once
