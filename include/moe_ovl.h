@@ -97,8 +97,9 @@ typedef struct {
                                          bounded wait runs out and the call ends with MOE_OVL_ERR_TIMEOUT */
 #define MOE_OVL_FLAG_TRACE 4u         /* reserve workspace for, and record, the per-item / per-unit device trace
                                          (moe_ovl_get_trace); off by default, costs nothing when off */
-#define MOE_OVL_FLAG_NO_SMALL_GROUP_TILES 16u /* never issue the swapped-operand items that runs of small (expert, rank)
-                                         groups otherwise get (see moe_ovl_plan_view.item); for comparisons */
+#define MOE_OVL_FLAG_NO_SMALL_GROUP_TILES 16u /* never issue the 64-row-high pair items and the swapped-operand items that
+                                         small (expert, rank) groups otherwise get (see moe_ovl_plan_view.item); for
+                                         comparisons */
 #define MOE_OVL_FLAG_TEST_ALL_SMALL_GROUP_TILES 32u /* test hook: every eligible run of small groups gets swapped-operand
                                          items, also where the plan's cost rule would keep band pairs */
 #define MOE_OVL_FLAG_TEST_SKIP_GATHER 8u /* test hook: the first band of the schedule is never gathered, so the GEMM's
@@ -196,7 +197,9 @@ typedef struct {
     int32_t *sched_band;      /* [bands] band ids in schedule order */
     int32_t *item;            /* [items][4] in issue order.  Kinds 0 (first GEMM) and 1 (second GEMM): {kind | expert << 8,
                                  band, second band of the pair or -1, tile}, a 256-row x 256-column tile of two bands
-                                 (128 hidden columns per band for kind 0).  Kinds 2 and 3, the same two GEMMs for a
+                                 (128 hidden columns per band for kind 0); kinds 4 and 5 are the same items for a pair
+                                 whose bands hold at most 64 valid rows each, computed 64 rows high (half the
+                                 tensor-pipe time).  Kinds 2 and 3, the same two GEMMs for a
                                  run whose (expert, rank) groups hold at most 64 rows each: {kind | expert << 8,
                                  position of the first band in sched_band, bands | rows << 8, tile} -- the valid rows
                                  of up to 8 consecutive bands (each rounded up to 16, at most 128 together) against a

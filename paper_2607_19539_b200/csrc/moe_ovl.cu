@@ -172,7 +172,7 @@ struct moe_ovl_ctx {
     bool hist_timed[MOE_OVL_TIMING_HISTORY];
     int last_cuda_error;
     EncodeTiledFn encode;
-    CUtensorMap map_xa, map_h, map_xa8, map_h8;
+    CUtensorMap map_xa, map_h, map_xa8, map_h8, map_xa64, map_h64;
 };
 
 namespace {
@@ -229,6 +229,7 @@ Params make_params(moe_ovl_ctx *ctx)
     p.seg_slot0 = at<int>(ctx, L.seg_slot0); p.tok_slot = at<int>(ctx, L.tok_slot);
     p.tok_gate = at<float>(ctx, L.tok_gate); p.hcount = at<unsigned>(ctx, L.hcount);
     p.fcount = at<unsigned>(ctx, L.fcount);
+    p.low_ok = !(c.flags & MOE_OVL_FLAG_NO_SMALL_GROUP_TILES);
     p.swap_ok = (!(c.flags & MOE_OVL_FLAG_NO_SMALL_GROUP_TILES) && (L.single || c.d_ffn % (2 * H_TILE) == 0))
                     ? ((c.flags & MOE_OVL_FLAG_TEST_ALL_SMALL_GROUP_TILES) ? 2 : 1) : 0;
     p.next_item = at<int>(ctx, L.next_item);
@@ -425,6 +426,9 @@ int moe_ovl_create(moe_ovl_ctx **out, const moe_ovl_config *cfg, void *workspace
     // the same buffers in boxes of 8 rows, for the token side of the swapped-operand items
     if (rc == MOE_OVL_OK) rc = encode_map(ctx, &ctx->map_xa8, ctx->ws + L.Xa, P, cfg->d_model, 8);
     if (rc == MOE_OVL_OK) rc = encode_map(ctx, &ctx->map_h8, ctx->ws + L.H, P, L.f_eff, 8);
+    // ... and in boxes of 64 rows, for band pairs that are computed 64 rows high
+    if (rc == MOE_OVL_OK) rc = encode_map(ctx, &ctx->map_xa64, ctx->ws + L.Xa, P, cfg->d_model, 64);
+    if (rc == MOE_OVL_OK) rc = encode_map(ctx, &ctx->map_h64, ctx->ws + L.H, P, L.f_eff, 64);
     if (rc != MOE_OVL_OK) return fail(rc);
     // flags hold the epoch of the call that finished the tile: clear them once, never again
     CREATE_CHECK(cudaMemset(ctx->ws + L.flags, 0, (size_t)L.max_bands * L.n2 * 4));
@@ -514,14 +518,19 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     maps.h = ctx->map_h;
     maps.xa8 = ctx->map_xa8;
     maps.h8 = ctx->map_h8;
+    maps.xa64 = ctx->map_xa64;
+    maps.h64 = ctx->map_h64;
     int rc;
     if (L.single) {
         // one projection per expert: W[El, N, d] is the B operand of the GEMM that writes Y
         rc = encode_map(ctx, &maps.w2, a->w1, (size_t)c.num_local_experts * L.dout, c.d_model);
         maps.w1 = maps.w2;
+        maps.w1h = maps.w2;          // no first GEMM
     } else {
         rc = encode_map(ctx, &maps.w1, a->w1, (size_t)c.num_local_experts * 2 * c.d_ffn, c.d_model);
         if (rc == MOE_OVL_OK) rc = encode_map(ctx, &maps.w2, a->w2, (size_t)c.num_local_experts * c.d_model, c.d_ffn);
+        if (rc == MOE_OVL_OK)
+            rc = encode_map(ctx, &maps.w1h, a->w1, (size_t)c.num_local_experts * 2 * c.d_ffn, c.d_model, 64);
     }
     if (rc != MOE_OVL_OK) return rc;
 

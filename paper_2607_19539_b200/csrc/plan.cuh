@@ -231,10 +231,12 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
         run_exp[run] = e;
         run_nb[run] = nbands;
         run_segs[run] = nsegs;
-        // Worth it only if the groups are fewer than the band pairs they replace: an MMA costs the same whether its
-        // 256 rows are two bands of tokens or 256 weight rows against one group of tokens.  (swap_ok == 2: a
-        // test hook that takes every eligible run.)
-        const bool fewer = sgroups < (nbands + 1) / 2 || p.swap_ok == 2;
+        // Worth it only if the groups cost less tensor-pipe time than the band pairs they replace: an MMA over 256
+        // weight rows against one group of tokens costs what an MMA over two full bands of tokens costs, and twice
+        // what a pair of small bands costs when those are issued 64 rows high (KIND_LOW).  (swap_ok == 2: a test
+        // hook that takes every eligible run.)
+        const int pairs_run = (nbands + 1) / 2;
+        const bool fewer = (p.low_ok ? 2 * sgroups < pairs_run : sgroups < pairs_run) || p.swap_ok == 2;
         run_nsb[run] = (small && nbands > 0 && fewer) ? sgroups : -1;
     }
     __syncthreads();
@@ -404,7 +406,10 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
             const int pair = k % np, tile = k / np;
             const int b0 = p.sched_band[start + 2 * pair];
             const int b1 = 2 * pair + 1 < cnt ? p.sched_band[start + 2 * pair + 1] : -1;
-            p.items[(g1 ? o1 : o2) + k] = make_int4((g1 ? KIND_G1 : KIND_G2) | (e << 8), b0, b1, tile);
+            const bool low = p.low_ok && p.band_valid[b0] <= SMALL_BAND_ROWS &&
+                             (b1 < 0 || p.band_valid[b1] <= SMALL_BAND_ROWS);
+            p.items[(g1 ? o1 : o2) + k] =
+                make_int4((g1 ? KIND_G1 : KIND_G2) | (low ? KIND_LOW : 0) | (e << 8), b0, b1, tile);
         }
     }
 }

@@ -313,7 +313,12 @@ __device__ __forceinline__ void gather_unit(const Params &p, int band, int r0, i
 struct ProducerMaps {
     CUtensorMap xa, h, w1, w2;   // all 2-D bf16 row-major, box 64 x 128, 128-byte swizzle
     CUtensorMap xa8, h8;         // Xa and H again in boxes of 64 x 8: token rows of the swapped-operand items
+    CUtensorMap xa64, h64, w1h;  // Xa, H and W1 in boxes of 64 x 64: operands of the 64-row-high pair items (KIND_LOW)
 };
+
+// Instruction descriptor of a KIND_LOW item: M = 128 over the CTA pair (64 rows per CTA), N = 256.
+constexpr uint32_t UMMA_IDESC_LOW = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TB_N >> 3) << 17) |
+                                    ((uint32_t)(TB_M >> 4) << 24);
 
 // Instruction descriptor of a swapped-operand MMA: 256 weight rows over the CTA pair, N = rows of the band group.
 __device__ __forceinline__ uint32_t umma_idesc_n(int n)
@@ -421,6 +426,9 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
         prefetch_tmap(&maps.w2);
         prefetch_tmap(&maps.xa8);
         prefetch_tmap(&maps.h8);
+        prefetch_tmap(&maps.xa64);
+        prefetch_tmap(&maps.h64);
+        prefetch_tmap(&maps.w1h);
     }
     if (warp == 1) tmem_alloc(tmem_slot, PROD_TMEM_COLS);
     tc_fence_before();
@@ -460,6 +468,8 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             // swapped-operand items: weight rows are the A side; nb bands of tokens the B side (table in
             // shared memory, slot tab); gate and up projection take separate stage fills (fills = 2 * ksteps)
             int swap, nb, tab, half_rows, w_row, w_row_up, tok_is_x;
+            // KIND_LOW: 64-row boxes for A; the first GEMM's B is two 64-row boxes (gate rows, up rows; b2_row >= 0)
+            int low, b2_row;
         };
         volatile int2 *tabs = reinterpret_cast<volatile int2 *>(smem_gen + (swap_tab - smem_base));
         // 1 = item n is in `j`, 0 = schedule exhausted, -1 = gave up.  Lane 0 only.
@@ -471,7 +481,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             const int4 item = p.items[it];       // {kind | expert << 8, band 0, band 1 or -1, tile}
             const int kind = item.x & 0xff, e = item.x >> 8, tile = item.w;
             j.it = it;
-            j.swap = kind >= KIND_G1S;
+            j.swap = kind == KIND_G1S || kind == KIND_G2S;
             if (j.swap) {
                 // {kind | expert << 8, first schedule position, bands | rows << 8, tile}
                 j.nb = item.z & 0xff;
@@ -504,7 +514,19 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             const int band = (rank == 0 || item.z < 0) ? item.y : item.z;
             j.a_row = band * TB_M;
             j.dep_index = band;
-            if (kind == KIND_G1) {
+            j.low = (kind & KIND_LOW) != 0;
+            j.b2_row = -1;
+            if ((kind & 3) == KIND_G1 && j.low) {
+                // 64 rows per CTA: the accumulator's columns 0..127 (from CTA 0's B rows) land in lanes 0..63 and
+                // columns 128..255 (CTA 1's) in lanes 64..127 of BOTH CTAs.  So that a lane holds the gate and the
+                // up value of the same hidden column, each CTA's B rows are 64 gate rows followed by the matching
+                // 64 up rows: rank 0 the tile's hidden columns 0..63, rank 1 columns 64..127.
+                j.amap = &maps.xa64; j.bmap = &maps.w1h;
+                j.b_row = e * 2 * p.F + tile * H_TILE + (int)rank * (H_TILE / 2);
+                j.b2_row = j.b_row + p.F;
+                j.ksteps = p.d / TB_K;
+                j.dep = &p.xready[band]; j.dep_want = (unsigned)TB_M; j.dep_site = SITE_TMA_XREADY;
+            } else if ((kind & 3) == KIND_G1) {
                 j.amap = &maps.xa; j.bmap = &maps.w1;
                 // rank 0 holds the gate-projection rows of the tile, rank 1 the matching up-projection rows
                 j.b_row = e * 2 * p.F + tile * H_TILE + (int)rank * p.F;
@@ -513,7 +535,8 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 j.dep = &p.xready[band]; j.dep_want = (unsigned)TB_M; j.dep_site = SITE_TMA_XREADY;
             } else {
                 // single-projection experts: the output GEMM reads the aligned input itself
-                j.amap = p.single ? &maps.xa : &maps.h; j.bmap = &maps.w2;
+                j.amap = j.low ? (p.single ? &maps.xa64 : &maps.h64) : (p.single ? &maps.xa : &maps.h);
+                j.bmap = &maps.w2;
                 j.b_row = e * p.dout + tile * TB_N + (int)rank * (TB_N / 2);
                 j.ksteps = p.k2 / TB_K;
                 if (p.n1 > 0) {   // every first-GEMM tile of this band must have landed in H
@@ -619,9 +642,11 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 // arrival; the phase still cannot complete early because the arrival itself is pending.
                 // The peer can only refill a stage after the leader's MMAs have consumed (hence completed)
                 // its previous phase, so bytes never leak into the wrong phase.
-                if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * PROD_STAGE_BYTES);
+                if (rank == 0)
+                    mbar_arrive_expect_tx(bar_full + 8 * stage, cur.low ? 2 * (PROD_A_BYTES / 2 + PROD_B_BYTES) : 2 * PROD_STAGE_BYTES);
                 tma_load_2d(sa, cur.amap, full, ks * TB_K, cur.a_row);
                 tma_load_2d(sb, cur.bmap, full, ks * TB_K, cur.b_row);
+                if (cur.b2_row >= 0) tma_load_2d(sb + PROD_B_BYTES / 2, cur.bmap, full, ks * TB_K, cur.b2_row);
                 ++fills;
                 if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
                 if (ks == look) {
@@ -654,11 +679,11 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 if (it < 0 || it >= n_items) break;
                 const int4 item = p.items[it];
                 const int kind = item.x & 0xff;
-                const bool swap = kind >= KIND_G1S;
-                const bool first_gemm = kind == KIND_G1 || kind == KIND_G1S;
+                const bool swap = kind == KIND_G1S || kind == KIND_G2S;
+                const bool first_gemm = (kind & 3) == KIND_G1 || kind == KIND_G1S;
                 const int ksteps = (first_gemm ? p.d : p.k2) / TB_K;
                 const int ntok = swap ? item.z >> 8 : 0;
-                const uint32_t idesc = swap ? umma_idesc_n(ntok) : UMMA_IDESC;
+                const uint32_t idesc = swap ? umma_idesc_n(ntok) : ((kind & KIND_LOW) ? UMMA_IDESC_LOW : UMMA_IDESC);
                 unsigned long long w_acc = 0, w_first = 0, stall_ns = 0;    // trace only
                 if (kTrace && !mbar_try_wait_cluster(bar_tempty + 8 * acc, acc_phase ^ 1u)) {
                     const unsigned long long w0 = globaltimer_ns();
@@ -764,8 +789,9 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             if (it >= n_items) break;
             const int4 item = p.items[it];
             const int kind = item.x & 0xff, tile = item.w;
-            const bool swap = kind >= KIND_G1S;
-            const bool first_gemm = kind == KIND_G1 || kind == KIND_G1S;
+            const bool swap = kind == KIND_G1S || kind == KIND_G2S;
+            const bool low = (kind & KIND_LOW) != 0;
+            const bool first_gemm = (kind & 3) == KIND_G1 || kind == KIND_G1S;
             const bool present = swap || (rank == 0) || item.z >= 0;     // the pair's second band may be absent
             const int band = rank == 0 ? item.y : item.z;
             ok = mbar_wait(bar_tfull + 8 * acc, acc_phase, p, SITE_EPI_TFULL, it);
@@ -817,6 +843,45 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 }
             } else if (!present) {
                 // nothing to store: the accumulator of an absent band is discarded
+            } else if (low) {
+                // 64 rows per CTA: lanes 0..63 hold the rows' accumulator columns 0..127, lanes 64..127 the same rows'
+                // columns 128..255 (in tensor-memory columns 0..127 both).  First GEMM: a lane's 128 columns are 64
+                // gate values followed by the 64 matching up values (see the load warp).
+                const int lrow = (q & 1) * 32 + lane, half = q >> 1;
+                const size_t lgrow = (size_t)band * TB_M + lrow;
+                if (first_gemm) {
+                    uint16_t *dst = p.H + lgrow * p.F + (size_t)tile * H_TILE + half * (H_TILE / 2);
+#pragma unroll 1
+                    for (int c = 0; c < H_TILE / 2; c += 32) {
+                        uint32_t g[32], u[32];
+                        tmem_ld32(taddr + c, g);
+                        tmem_ld32(taddr + H_TILE / 2 + c, u);
+                        tmem_ld_wait();
+                        uint32_t o[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            o[j] = pack_bf16x2(silu_mul(__uint_as_float(g[2 * j]), __uint_as_float(u[2 * j])),
+                                               silu_mul(__uint_as_float(g[2 * j + 1]), __uint_as_float(u[2 * j + 1])));
+                        uint4 *d4 = reinterpret_cast<uint4 *>(dst + c);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) d4[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                    }
+                } else {
+                    uint16_t *dst = p.Y + lgrow * p.dout + (size_t)tile * TB_N + half * (TB_N / 2);
+#pragma unroll 1
+                    for (int c = 0; c < TB_N / 2; c += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(taddr + c, v);
+                        tmem_ld_wait();
+                        uint32_t o[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            o[j] = pack_bf16x2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                        uint4 *d4 = reinterpret_cast<uint4 *>(dst + c);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) d4[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                    }
+                }
             } else if (kind == KIND_G1) {
                 uint16_t *dst = p.H + grow * p.F + (size_t)tile * H_TILE;
 #pragma unroll 1
@@ -883,7 +948,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     }
                 }
             } else if (leader && present) {
-                if (kind == KIND_G1) red_release_add_u32(&p.hcount[band], 1u);
+                if (first_gemm) red_release_add_u32(&p.hcount[band], 1u);
                 else if (raise_flags) {
                     st_release_u32(&p.flags[(size_t)band * p.n2 + tile], epoch);
                     const unsigned long long now = globaltimer_ns();

@@ -70,6 +70,10 @@ def check_indices(shape, dsp, plan, gpu_plan, slot_out, rows_per_rank, segs_per_
     valid = gpu_plan["band_valid"].tolist()
     for x, b0, b1, tile in raw.tolist():
         kind, e = x & 0xff, x >> 8
+        if kind & 4:                 # a band pair computed 64 rows high: both bands hold at most 64 valid rows
+            assert valid[b0] <= 64 and (b1 < 0 or valid[b1] <= 64)
+            kind &= 3
+            assert kind < 2
         if kind >= 2:
             group = sched[b0:b0 + (b1 & 0xff)]
             assert 1 <= len(group) <= 8 and all(valid[b] <= 64 for b in group)

@@ -605,3 +605,15 @@ def test_small_group_items_can_be_switched_off(name):
     assert kinds[B.FLAG_NO_SMALL_GROUP_TILES] <= {0, 1}
     # every one of these problems has at least one run of small groups
     assert kinds[B.FLAG_TEST_ALL_SMALL_GROUP_TILES] & {2, 3}
+    # left to itself the plan computes pairs of small bands 64 rows high (kinds 4, 5); these shapes hold too few
+    # items for swapped-operand groups to pay
+    ctx = Hn.make_context(shape, max_rows=dsp.M)
+    prob = Hn.upload(inp, dsp)
+    Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=4)
+    torch.cuda.synchronize()
+    assert ctx.moe_ovl_query_status()[0] == 0
+    gp = ctx.moe_ovl_get_plan()
+    U.check_indices(shape, dsp, plan, gp, prob.slot_out.cpu().numpy(), prob.rows_per_rank_out.cpu().numpy(),
+                    prob.segs_per_rank_out.cpu().numpy(), ctx.moe_ovl_get_report())
+    U.check_values(shape, dsp, plan, toks, *o, Hn.device_to_bits(prob.out), Hn.device_to_bits(prob.ret))
+    assert set((gp["item"][:, 0] & 0xff).tolist()) & {4, 5}
