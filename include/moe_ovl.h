@@ -100,6 +100,10 @@ typedef struct {
 #define MOE_OVL_FLAG_NO_SMALL_GROUP_TILES 16u /* never issue the 64-row-high pair items and the swapped-operand items that
                                          small (expert, rank) groups otherwise get (see moe_ovl_plan_view.item); for
                                          comparisons */
+#define MOE_OVL_FLAG_NO_STACKED_BANDS 64u /* never stack three or four small bands into one full-height item (kinds 8
+                                         and 9 of moe_ovl_plan_view.item); for comparisons */
+#define MOE_OVL_FLAG_NO_LOCAL_RIDERS 128u /* never let an expert's local band join the last item of its remote bands (see
+                                         moe_ovl_plan_view.item); for comparisons */
 #define MOE_OVL_FLAG_TEST_ALL_SMALL_GROUP_TILES 32u /* test hook: every eligible run of small groups gets swapped-operand
                                          items, also where the plan's cost rule would keep band pairs */
 #define MOE_OVL_FLAG_TEST_SKIP_GATHER 8u /* test hook: the first band of the schedule is never gathered, so the GEMM's
@@ -198,8 +202,15 @@ typedef struct {
     int32_t *item;            /* [items][4] in issue order.  Kinds 0 (first GEMM) and 1 (second GEMM): {kind | expert << 8,
                                  band, second band of the pair or -1, tile}, a 256-row x 256-column tile of two bands
                                  (128 hidden columns per band for kind 0); kinds 4 and 5 are the same items for a pair
-                                 whose bands hold at most 64 valid rows each, computed 64 rows high (half the
-                                 tensor-pipe time).  Kinds 2 and 3, the same two GEMMs for a
+                                 whose bands hold at most 64 valid rows each, computed 64 rows high (about 0.9 of
+                                 the tensor-pipe time).  Kinds 8 and 9: {kind | expert << 8, first band, bands,
+                                 tile} -- 3 or 4 bands with consecutive ids, at most 64 valid rows each, stacked
+                                 into one full-height item (rows 0..63 of two bands per CTA), i.e. two such pairs
+                                 for the time of one.  Where the last item of an expert's remote bands (kinds 4, 5,
+                                 8, 9) has rows to spare and the expert's local rows are one band of at most 64, that
+                                 band is issued in the same item (its id is the last remote band's + 1) and has no
+                                 items of its own: no remote tile is issued later for it, and the expert's weights
+                                 are read once instead of twice.  Kinds 2 and 3, the same two GEMMs for a
                                  run whose (expert, rank) groups hold at most 64 rows each: {kind | expert << 8,
                                  position of the first band in sched_band, bands | rows << 8, tile} -- the valid rows
                                  of up to 8 consecutive bands (each rounded up to 16, at most 128 together) against a

@@ -22,8 +22,13 @@ constexpr int KIND_G2 = 1;    // H . W2 -> Y, raises the consumer-visible flag
 constexpr int KIND_G1S = 2;
 constexpr int KIND_G2S = 3;
 // Bit of the item kind, on KIND_G1 / KIND_G2 only: both bands of the pair hold at most SMALL_BAND_ROWS valid rows,
-// so the pair is computed as an M = 128 MMA (64 rows per CTA), which takes half the tensor-pipe time of M = 256.
+// so the pair is computed as an M = 128 MMA (64 rows per CTA), which takes about 0.9 of the time of M = 256 (each MMA
+// still reads the whole 256-row B tile from shared memory).
 constexpr int KIND_LOW = 4;
+// Bit of the item kind, on KIND_G1 / KIND_G2 only: three or four consecutive bands of one run, each with at most
+// SMALL_BAND_ROWS valid rows, stacked into one full-height item: CTA c computes rows 0..63 of bands 2c and 2c + 1
+// in the upper and lower half of its 128 accumulator lanes.  Item = {kind | expert << 8, first band, bands, tile}.
+constexpr int KIND_STACK = 8;
 constexpr int SMALL_BAND_ROWS = 64;
 constexpr int SWAP_MAX_N = 128;
 constexpr int SWAP_MAX_BANDS = 8;          // SWAP_MAX_N / 16
@@ -65,7 +70,9 @@ struct Params {
     int lag_items;      // schedule items between a band's last first-GEMM tile and its first second-GEMM tile
     int words;          // 32-bit words of one (expert, rank) token bitmap = ceil(T / 32)
     int n1, n2;         // tiles per band: F / 128 (0 for single-projection experts) and dout / 256
-    int low_ok;         // band pairs whose bands hold at most SMALL_BAND_ROWS rows each are issued with KIND_LOW
+    int low_ok;         // band pairs whose bands hold at most SMALL_BAND_ROWS rows each are issued with KIND_LOW;
+                        // 2: and two such pairs side by side as one KIND_STACK item; 3: and an expert's small local band
+                        // may join the last item of its remote bands
     int swap_ok;        // runs of small groups may use the swapped-operand items (needs F % 256 == 0 for FFN experts):
                         // 0 never, 1 where the plan's cost rule says so, 2 every eligible run (test hook)
     int max_bands, max_items;

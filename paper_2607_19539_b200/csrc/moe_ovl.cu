@@ -36,7 +36,7 @@ struct Layout {
     size_t band_expert, band_dest, band_valid, band_slot0, sched_band, items, segs, seg_slot0;
     size_t tok_gate, flags, meta;
     size_t trace_items, trace_items2, trace_units, trace_item_aux, trace_bytes;   // MOE_OVL_FLAG_TRACE
-    size_t sb[10];
+    size_t sb[13];
     // host staging (MOE_OVL_FLAG_HOST_STAGING)
     size_t st_x[2], st_counts[2], st_rank[2], st_token[2], st_gate[2], st_out[2], st_ret;   // two staging slots
     size_t total;
@@ -121,7 +121,7 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->flags = take((size_t)L->max_bands * L->n2 * 4);
     L->meta = take(META_COUNT * 4 + 4);      // meta[] and the call counter
     L->smid = take(2 * 1024 * 4);            // SM of every GEMM CTA, then of every consumer CTA
-    for (int i = 0; i < 10; ++i) L->sb[i] = take((size_t)L->max_bands * 4);
+    for (int i = 0; i < 13; ++i) L->sb[i] = take((size_t)L->max_bands * 4);
     L->st_ret_rows = (long long)c->tokens_per_rank * L->kmax;
     L->trace_bytes = 0;
     if (c->flags & MOE_OVL_FLAG_TRACE) {
@@ -229,7 +229,9 @@ Params make_params(moe_ovl_ctx *ctx)
     p.seg_slot0 = at<int>(ctx, L.seg_slot0); p.tok_slot = at<int>(ctx, L.tok_slot);
     p.tok_gate = at<float>(ctx, L.tok_gate); p.hcount = at<unsigned>(ctx, L.hcount);
     p.fcount = at<unsigned>(ctx, L.fcount);
-    p.low_ok = !(c.flags & MOE_OVL_FLAG_NO_SMALL_GROUP_TILES);
+    p.low_ok = (c.flags & MOE_OVL_FLAG_NO_SMALL_GROUP_TILES) ? 0
+             : (c.flags & MOE_OVL_FLAG_NO_STACKED_BANDS)   ? 1
+             : (c.flags & MOE_OVL_FLAG_NO_LOCAL_RIDERS)    ? 2 : 3;
     p.swap_ok = (!(c.flags & MOE_OVL_FLAG_NO_SMALL_GROUP_TILES) && (L.single || c.d_ffn % (2 * H_TILE) == 0))
                     ? ((c.flags & MOE_OVL_FLAG_TEST_ALL_SMALL_GROUP_TILES) ? 2 : 1) : 0;
     p.next_item = at<int>(ctx, L.next_item);
@@ -539,6 +541,7 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     sc.sb_g1off = at<int>(ctx, L.sb[3]); sc.sb_g2off = at<int>(ctx, L.sb[4]); sc.sb_g1end = at<int>(ctx, L.sb[5]);
     sc.sb_kind = at<int>(ctx, L.sb[6]); sc.sb_ntok = at<int>(ctx, L.sb[7]);
     sc.sb_c1 = at<int>(ctx, L.sb[8]); sc.sb_c2 = at<int>(ctx, L.sb[9]);
+    sc.sb_units = at<int>(ctx, L.sb[10]); sc.unit_tab = at<int>(ctx, L.sb[11]); sc.sb_role = at<int>(ctx, L.sb[12]);
 
     int launches = 0;
     const int hist = (int)(ctx->calls % MOE_OVL_TIMING_HISTORY);

@@ -29,6 +29,10 @@ struct PlanScratch {
     int *sb_ntok;    // group of small bands: valid rows, each band rounded up to 16
     int *sb_c1;      // items of the super-band's first-GEMM block
     int *sb_c2;      // ... of its second-GEMM block
+    int *sb_units;   // super-band of band pairs: its units (a pair, or two pairs of small bands stacked)
+    int *unit_tab;   // [bands], a super-band's units at its first schedule position: first band's offset | bands << 8
+                     // | (1 << 16 if the unit's last band is the expert's local band riding with its remote ones)
+    int *sb_role;    // 1: last super-band of an expert's remote run, 2: super-band of a local run, else 0
 };
 
 __device__ __forceinline__ int ceil16(int v) { return (v + 15) & ~15; }
@@ -112,6 +116,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     __shared__ int segs_per_rank[PLAN_MAX_GROUPS];
     __shared__ int s_nsb;
     __shared__ int s_sb_c1[PLAN_SB_STAGE], s_sb_c2[PLAN_SB_STAGE], s_sb_end[PLAN_SB_STAGE];
+    __shared__ unsigned char erider[PLAN_MAX_EXPERTS];   // the expert's local band rides with its last remote bands
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
     const int G = p.El * p.R;
@@ -348,9 +353,56 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
             sc.sb_expert[sb] = run_exp[run];
             sc.sb_kind[sb] = 0;
             sc.sb_ntok[sb] = 0;
-            sc.sb_c1[sb] = ((sc.sb_nb[sb] + 1) / 2) * p.n1;
-            sc.sb_c2[sb] = ((sc.sb_nb[sb] + 1) / 2) * p.n2;
+            sc.sb_role[sb] = run >= El ? 2 : (q == nsb - 1 ? 1 : 0);
         }
+    }
+    for (int e = tid; e < El; e += blockDim.x) erider[e] = 0;
+    __syncthreads();
+
+    // E2: the units of every super-band of band pairs.  A unit is one schedule item per tile: a band pair, or --
+    //     where two neighbouring pairs hold only bands of at most SMALL_BAND_ROWS valid rows -- those three or four
+    //     bands stacked into one full-height item (KIND_STACK), which costs the tensor pipe what ONE pair costs.
+    //     Rider: where the LAST unit of an expert's remote run holds at most three bands, all small, and the expert's
+    //     local rows are one small band, that band joins the unit -- it takes rows of the item that would otherwise
+    //     be padding, so no remote tile is issued later than without it (the purpose of rule (i) of Section 3.2.2
+    //     holds), and the expert's weights are streamed once instead of twice.  The bands of an expert are
+    //     consecutive in the layout, remote ones first, so the unit's bands still have consecutive ids.
+    for (int sb = tid; sb < s_nsb; sb += blockDim.x) {
+        if (sc.sb_kind[sb]) continue;
+        const int start = sc.sb_start[sb], cnt = sc.sb_nb[sb], e = sc.sb_expert[sb];
+        auto small_band = [&](int o) { return p.band_valid[p.sched_band[start + o]] <= SMALL_BAND_ROWS; };
+        int units = 0, last_o = 0, last_take = 0;
+        for (int o = 0; o < cnt;) {
+            int take = min(2, cnt - o);
+            if (p.low_ok >= 2 && cnt - o >= 3) {
+                bool all_small = true;
+                const int four = min(4, cnt - o);
+                for (int q = 0; q < four; ++q) all_small = all_small && small_band(o + q);
+                if (all_small) take = four;
+            }
+            sc.unit_tab[start + units++] = o | (take << 8);
+            last_o = o;
+            last_take = take;
+            o += take;
+        }
+        const int n_local = n[e * R + self];
+        if (p.low_ok == 3 && sc.sb_role[sb] == 1 && units > 0 && last_take <= 3 && n_local > 0 &&
+            n_local <= SMALL_BAND_ROWS && run_nsb[El + e] < 0) {
+            bool all_small = true;
+            for (int q = 0; q < last_take; ++q) all_small = all_small && small_band(last_o + q);
+            if (all_small) {
+                sc.unit_tab[start + units - 1] = last_o | ((last_take + 1) << 8) | (1 << 16);
+                erider[e] = 1;
+            }
+        }
+        sc.sb_units[sb] = units;
+    }
+    __syncthreads();
+    for (int sb = tid; sb < s_nsb; sb += blockDim.x) {
+        if (sc.sb_kind[sb]) continue;
+        if (sc.sb_role[sb] == 2 && erider[sc.sb_expert[sb]]) sc.sb_units[sb] = 0;   // the band was issued with the remote ones
+        sc.sb_c1[sb] = sc.sb_units[sb] * p.n1;
+        sc.sb_c2[sb] = sc.sb_units[sb] * p.n2;
     }
     __syncthreads();
 
@@ -369,9 +421,16 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
         if (tid == 0) {
             int *c1v = staged ? s_sb_c1 : sc.sb_c1, *c2v = staged ? s_sb_c2 : sc.sb_c2;
             int *endv = staged ? s_sb_end : sc.sb_g1end;
+            // The schedule's last first-GEMM block must not be followed by its own second-GEMM block at once (every
+            // CTA pair that claims one of its tiles would wait for the block's stragglers, and with few tiles most
+            // pairs would idle meanwhile): the second-GEMM blocks of the last super-bands, as many whole blocks as
+            // stay within one item per CTA pair (lag_items is two), are held back until every first-GEMM block
+            // has been issued.  (More would only lengthen the run of long second-GEMM items at the very end.)
+            int hold_from = nsb - 1;
+            for (int acc = 0; hold_from > 0 && 2 * (acc + c2v[hold_from - 1]) <= p.lag_items;) acc += c2v[--hold_from];
             int ng1 = 0, off = 0;
             for (int ng2 = 0; ng2 < nsb; ++ng2) {
-                while (ng1 < nsb && (ng1 <= ng2 || off - endv[ng2] < p.lag_items)) {
+                while (ng1 < nsb && (ng1 <= ng2 || ng2 >= hold_from || off - endv[ng2] < p.lag_items)) {
                     sc.sb_g1off[ng1] = off;
                     off += c1v[ng1];
                     endv[ng1] = off;
@@ -388,7 +447,6 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     // G: the item list, one warp per super-band
     for (int sb = warp; sb < s_nsb; sb += nwarps) {
         const int start = sc.sb_start[sb], cnt = sc.sb_nb[sb], e = sc.sb_expert[sb];
-        const int np = (cnt + 1) / 2;
         const int o1 = sc.sb_g1off[sb], o2 = sc.sb_g2off[sb];
         if (sc.sb_kind[sb]) {
             // group of small bands: {kind | expert << 8, first schedule position, bands | rows << 8, tile}
@@ -400,12 +458,20 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
             }
             continue;
         }
-        for (int idx = lane; idx < np * (p.n1 + p.n2); idx += 32) {
-            const bool g1 = idx < np * p.n1;
-            const int k = g1 ? idx : idx - np * p.n1;
-            const int pair = k % np, tile = k / np;
-            const int b0 = p.sched_band[start + 2 * pair];
-            const int b1 = 2 * pair + 1 < cnt ? p.sched_band[start + 2 * pair + 1] : -1;
+        const int nu = sc.sb_units[sb];
+        for (int idx = lane; idx < nu * (p.n1 + p.n2); idx += 32) {
+            const bool g1 = idx < nu * p.n1;
+            const int k = g1 ? idx : idx - nu * p.n1;
+            const int unit = sc.unit_tab[start + k % nu], tile = k / nu;
+            const int o = unit & 0xff, take = (unit >> 8) & 0xff;
+            const bool rider = (unit >> 16) != 0;
+            const int b0 = p.sched_band[start + o];
+            if (take > 2) {
+                // the bands of a run are consecutive in the layout: b0, b0 + 1, ...
+                p.items[(g1 ? o1 : o2) + k] = make_int4((g1 ? KIND_G1 : KIND_G2) | KIND_STACK | (e << 8), b0, take, tile);
+                continue;
+            }
+            const int b1 = take == 2 ? (rider ? b0 + 1 : p.sched_band[start + o + 1]) : -1;
             const bool low = p.low_ok && p.band_valid[b0] <= SMALL_BAND_ROWS &&
                              (b1 < 0 || p.band_valid[b1] <= SMALL_BAND_ROWS);
             p.items[(g1 ? o1 : o2) + k] =

@@ -24,7 +24,8 @@
 //              small ring in shared memory.  Items are claimed in schedule order, so the
 //              remote-first order holds and every dependency still points to an earlier claim.
 // A schedule item is a pair of 128-row bands of one expert (the second may be absent) times
-// one tile; CTA rank r of the cluster owns band r of the pair:
+// one tile (or three or four bands of at most 64 valid rows each, two per CTA: KIND_STACK); CTA rank r of the
+// cluster owns band r of the pair:
 //   first GEMM   A = Xa[band]; B = 128 gate rows of W1 (held by rank 0) and the matching 128
 //                up rows (rank 1) -> one N=256 accumulator; the epilogue pairs column c with
 //                c+128: h = silu(g) * u, 128 columns of H; then hcount[band] += 1 (release)
@@ -470,6 +471,10 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             int swap, nb, tab, half_rows, w_row, w_row_up, tok_is_x;
             // KIND_LOW: 64-row boxes for A; the first GEMM's B is two 64-row boxes (gate rows, up rows; b2_row >= 0)
             int low, b2_row;
+            // KIND_STACK: A is two 64-row boxes, rows 0..63 of two bands (a2_row >= 0); the second band has a
+            // counter of its own to wait for (dep2, may be null)
+            int a2_row;
+            const unsigned *dep2;
         };
         volatile int2 *tabs = reinterpret_cast<volatile int2 *>(smem_gen + (swap_tab - smem_base));
         // 1 = item n is in `j`, 0 = schedule exhausted, -1 = gave up.  Lane 0 only.
@@ -511,8 +516,14 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 j.dep = on_x ? p.xready : p.hcount;
                 return 1;
             }
-            const int band = (rank == 0 || item.z < 0) ? item.y : item.z;
+            const bool stack = (kind & KIND_STACK) != 0;
+            // stacked bands: this CTA's are item.y + 2 * rank and, if the item has that many, the one after it
+            const int band = stack ? item.y + 2 * (int)rank : ((rank == 0 || item.z < 0) ? item.y : item.z);
+            const int band2 = (stack && 2 * (int)rank + 1 < item.z) ? band + 1 : -1;
             j.a_row = band * TB_M;
+            // no second band: the box is filled with the first band's rows 64..127, whose results are not stored
+            j.a2_row = stack ? (band2 >= 0 ? band2 * TB_M : j.a_row + TB_M / 2) : -1;
+            j.dep2 = nullptr;
             j.dep_index = band;
             j.low = (kind & KIND_LOW) != 0;
             j.b2_row = -1;
@@ -527,25 +538,29 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 j.ksteps = p.d / TB_K;
                 j.dep = &p.xready[band]; j.dep_want = (unsigned)TB_M; j.dep_site = SITE_TMA_XREADY;
             } else if ((kind & 3) == KIND_G1) {
-                j.amap = &maps.xa; j.bmap = &maps.w1;
+                j.amap = stack ? &maps.xa64 : &maps.xa; j.bmap = &maps.w1;
                 // rank 0 holds the gate-projection rows of the tile, rank 1 the matching up-projection rows
                 j.b_row = e * 2 * p.F + tile * H_TILE + (int)rank * p.F;
                 j.ksteps = p.d / TB_K;
                 // all 128 rows of the band (padding included) must have been gathered into Xa
                 j.dep = &p.xready[band]; j.dep_want = (unsigned)TB_M; j.dep_site = SITE_TMA_XREADY;
+                if (band2 >= 0) j.dep2 = &p.xready[band2];
             } else {
                 // single-projection experts: the output GEMM reads the aligned input itself
-                j.amap = j.low ? (p.single ? &maps.xa64 : &maps.h64) : (p.single ? &maps.xa : &maps.h);
+                j.amap = (j.low || stack) ? (p.single ? &maps.xa64 : &maps.h64) : (p.single ? &maps.xa : &maps.h);
                 j.bmap = &maps.w2;
                 j.b_row = e * p.dout + tile * TB_N + (int)rank * (TB_N / 2);
                 j.ksteps = p.k2 / TB_K;
                 if (p.n1 > 0) {   // every first-GEMM tile of this band must have landed in H
                     j.dep = &p.hcount[band]; j.dep_want = (unsigned)p.n1; j.dep_site = SITE_TMA_HCOUNT;
+                    if (band2 >= 0) j.dep2 = &p.hcount[band2];
                 } else {
                     j.dep = &p.xready[band]; j.dep_want = (unsigned)TB_M; j.dep_site = SITE_TMA_XREADY;
+                    if (band2 >= 0) j.dep2 = &p.xready[band2];
                 }
             }
-            j.dep_ok = ld_acquire_u32(j.dep) >= j.dep_want;      // the counters only grow
+            j.dep_ok = ld_acquire_u32(j.dep) >= j.dep_want &&      // the counters only grow
+                       (j.dep2 == nullptr || ld_acquire_u32(j.dep2) >= j.dep_want);
             return 1;
         };
         Job cur, nxt;
@@ -628,6 +643,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             // ---- band-pair item, lane 0
             if (!cur.dep_ok) {
                 ok = wait_global(cur.dep, cur.dep_want, true, p, cur.dep_site, cur.dep_index);
+                if (ok && cur.dep2) ok = wait_global(cur.dep2, cur.dep_want, true, p, cur.dep_site, cur.dep_index + 1);
                 if (!ok) continue;
             }
             asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
@@ -645,6 +661,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 if (rank == 0)
                     mbar_arrive_expect_tx(bar_full + 8 * stage, cur.low ? 2 * (PROD_A_BYTES / 2 + PROD_B_BYTES) : 2 * PROD_STAGE_BYTES);
                 tma_load_2d(sa, cur.amap, full, ks * TB_K, cur.a_row);
+                if (cur.a2_row >= 0) tma_load_2d(sa + PROD_A_BYTES / 2, cur.amap, full, ks * TB_K, cur.a2_row);
                 tma_load_2d(sb, cur.bmap, full, ks * TB_K, cur.b_row);
                 if (cur.b2_row >= 0) tma_load_2d(sb + PROD_B_BYTES / 2, cur.bmap, full, ks * TB_K, cur.b2_row);
                 ++fills;
@@ -792,15 +809,20 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             const bool swap = kind == KIND_G1S || kind == KIND_G2S;
             const bool low = (kind & KIND_LOW) != 0;
             const bool first_gemm = (kind & 3) == KIND_G1 || kind == KIND_G1S;
-            const bool present = swap || (rank == 0) || item.z >= 0;     // the pair's second band may be absent
-            const int band = rank == 0 ? item.y : item.z;
+            const bool stack = (kind & KIND_STACK) != 0;
+            // stacked bands: lanes 0..63 hold rows 0..63 of band item.y + 2 * rank, lanes 64..127 those of the next
+            // band, if the item has that many (item.z = its bands)
+            const int sband = item.y + 2 * (int)rank + (q >> 1);
+            const bool present = stack ? 2 * (int)rank + (q >> 1) < item.z
+                                       : (swap || (rank == 0) || item.z >= 0);     // the pair's second band may be absent
+            const int band = stack ? sband : (rank == 0 ? item.y : item.z);
             ok = mbar_wait(bar_tfull + 8 * acc, acc_phase, p, SITE_EPI_TFULL, it);
             ok = epilogue_all(ok);
             if (!ok) break;
             tc_fence_after();
             if (kTrace && leader && rank == 0) p.trace_items2[it].a = globaltimer_ns();
             const uint32_t taddr = tmem_base + (uint32_t)acc * TB_N + ((uint32_t)(q * 32) << 16);
-            const size_t grow = (size_t)(present ? band : 0) * TB_M + row;
+            const size_t grow = (size_t)(present ? band : 0) * TB_M + (stack ? (q & 1) * 32 + lane : row);
             if (swap) {
                 // Swapped operands: lane = one of this CTA's 128 weight rows, i.e. one hidden / output column;
                 // accumulator column n = row n of the band group (first halves of all bands from CTA 0's token
@@ -882,7 +904,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                         for (int j = 0; j < 4; ++j) d4[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
                     }
                 }
-            } else if (kind == KIND_G1) {
+            } else if ((kind & 3) == KIND_G1) {
                 uint16_t *dst = p.H + grow * p.F + (size_t)tile * H_TILE;
 #pragma unroll 1
                 for (int c = 0; c < H_TILE; c += 32) {
@@ -926,7 +948,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             __threadfence();
             if (first_gemm) asm volatile("fence.proxy.async;" ::: "memory");   // H is re-read through TMA
             bar_sync_epilogue();
-            if (kTrace && leader && present) {
+            if (kTrace && leader && (present || stack)) {
                 // taken before the release below, so that no observer of the flag can carry an earlier time
                 const unsigned long long now = globaltimer_ns();
                 if (rank == 0) p.trace_items[it].c = now; else p.trace_items[it].d = now;
@@ -941,6 +963,18 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     if (first_gemm) {
                         red_release_add_u32(&p.hcount[b], 1u);
                     } else if (raise_flags && atom_add_acq_rel_u32(&p.fcount[(size_t)b * p.n2 + tile], 1u) == 1u) {
+                        st_release_u32(&p.flags[(size_t)b * p.n2 + tile], epoch);
+                        const unsigned long long now = globaltimer_ns();
+                        stamp_max(&p.stamps[STAMP_FIRST_FLAG_INV], ~now);
+                        stamp_max(&p.stamps[STAMP_LAST_FLAG], now);
+                    }
+                }
+            } else if (leader && stack) {
+                // this CTA's one or two bands of the stack
+                for (int b = item.y + 2 * (int)rank; b < item.y + min(2 * (int)rank + 2, item.z); ++b) {
+                    if (first_gemm) {
+                        red_release_add_u32(&p.hcount[b], 1u);
+                    } else if (raise_flags) {
                         st_release_u32(&p.flags[(size_t)b * p.n2 + tile], epoch);
                         const unsigned long long now = globaltimer_ns();
                         stamp_max(&p.stamps[STAMP_FIRST_FLAG_INV], ~now);

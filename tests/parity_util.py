@@ -63,9 +63,22 @@ def check_indices(shape, dsp, plan, gpu_plan, slot_out, rows_per_rank, segs_per_
     # an item is {kind | expert << 8, band, second band of the pair or -1, tile}: expand pairs to single bands
     # (kinds 2 and 3 -- a group of small bands against 256 weight rows, operands swapped -- expand to the same
     # per-band tiles: {kind | expert << 8, first schedule position, bands | rows << 8, tile}, where a first-GEMM
-    # tile of 256 hidden columns stands for two of 128)
+    # tile of 256 hidden columns stands for two of 128; kinds 8 and 9 -- {kind | expert << 8, first band, bands,
+    # tile} -- expand to their 3 or 4 consecutive bands)
     raw = gpu_plan["item"]
     rows = []
+    band = {b.band: b for b in plan.bands}
+    riders = set()
+
+    def note_rider(group):
+        # An expert's local band may ride in rows of its last remote item that would otherwise be padding: one local
+        # band, the last of the item, all of the item's bands small and consecutive in the layout.
+        if band[group[-1]].local and not band[group[0]].local:
+            assert not any(band[b].local for b in group[:-1]) and group == list(range(group[0], group[0] + len(group)))
+            assert all(valid[b] <= 64 for b in group) and len({band[b].expert for b in group}) == 1
+            riders.add(group[-1])
+        else:
+            assert len({band[b].local for b in group}) == 1
     sched = gpu_plan["sched_band"].tolist()
     valid = gpu_plan["band_valid"].tolist()
     for x, b0, b1, tile in raw.tolist():
@@ -74,6 +87,15 @@ def check_indices(shape, dsp, plan, gpu_plan, slot_out, rows_per_rank, segs_per_
             assert valid[b0] <= 64 and (b1 < 0 or valid[b1] <= 64)
             kind &= 3
             assert kind < 2
+        if kind & 8:                 # three or four bands of at most 64 valid rows, stacked into one full-height item
+            group = list(range(b0, b0 + b1))
+            note_rider(group)
+            at, own = sched.index(b0), b1 - (group[-1] in riders)
+            assert b1 in (3, 4) and sched[at:at + own] == group[:own] and all(valid[b] <= 64 for b in group)
+            kind &= 3
+            assert kind < 2
+            rows += [(kind, b, tile, e) for b in group]
+            continue
         if kind >= 2:
             group = sched[b0:b0 + (b1 & 0xff)]
             assert 1 <= len(group) <= 8 and all(valid[b] <= 64 for b in group)
@@ -83,6 +105,7 @@ def check_indices(shape, dsp, plan, gpu_plan, slot_out, rows_per_rank, segs_per_
             continue
         rows.append((kind, b0, tile, e))
         if b1 >= 0:
+            note_rider([b0, b1])
             rows.append((kind, b1, tile, e))
     items = np.asarray(rows, np.int64).reshape(-1, 4)
     n1, n2 = (0 if shape.N_out else shape.F // 128), shape.dout // 256
@@ -91,14 +114,13 @@ def check_indices(shape, dsp, plan, gpu_plan, slot_out, rows_per_rank, segs_per_
     expect = sorted((b.band, j) for b in plan.bands for j in range(n2))
     assert sorted(map(tuple, g2[:, 1:3].tolist())) == expect                       # every output tile once
     assert sorted(map(tuple, g1[:, 1:3].tolist())) == sorted((b.band, j) for b in plan.bands for j in range(n1))
-    band = {b.band: b for b in plan.bands}
     assert all(band[b].expert == e for _, b, _, e in items.tolist())
-    first_seen = list(dict.fromkeys(g2[:, 1].tolist()))
-    assert first_seen == plan.band_order                                           # bands start in schedule order
-    local = [band[b].local for b in g2[:, 1].tolist()]
+    first_seen = [b for b in dict.fromkeys(g2[:, 1].tolist()) if b not in riders]
+    assert first_seen == [b for b in plan.band_order if b not in riders]           # bands start in schedule order
+    local = [band[b].local for b in g2[:, 1].tolist() if b not in riders]
     k = local.index(True) if True in local else len(local)
     assert not any(local[:k]) and all(local[k:])                                   # rule (i): remote tiles first
-    ex = [e for e in g2[:k, 3].tolist()]
+    ex = [e for b, e in zip(g2[:, 1].tolist(), g2[:, 3].tolist()) if b not in riders][:k]
     runs = [e for i, e in enumerate(ex) if i == 0 or ex[i - 1] != e]
     assert runs == [e for e in plan.expert_order if any(b.expert == e and not b.local for b in plan.bands)]
     # a second-GEMM tile is issued after every first-GEMM tile of its band

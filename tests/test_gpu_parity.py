@@ -432,7 +432,7 @@ def test_trace_records_every_item_and_unit(mode, csm):
     assert len(items) == rep.num_items and items["index"].tolist() == list(range(rep.num_items))
     assert (items["ns_claim"] >= 0).all()
     assert (items["ns_claim"] <= items["ns_ready"]).all() and (items["ns_ready"] <= items["ns_done0"]).all()
-    second = plan["item"][:, 2] >= 0                     # the pair's second band exists
+    second = plan["item"][:, 2] >= 0                     # the pair's second band exists (a stack always has one)
     assert (items["ns_done1"][second] >= items["ns_ready"][second]).all() and (items["ns_done1"][~second] == -1).all()
     assert (items["cta"] % 2 == 0).all() and items["cta"].max() < rep.producer_ctas
     # claims are handed out in issue order (each pair stamps its own claim, hence the slack)
@@ -455,8 +455,16 @@ def test_trace_records_every_item_and_unit(mode, csm):
     # latest publication time of any output tile of each band (second-GEMM items only)
     n_bands = rep.num_bands
     band_done = np.zeros(n_bands, np.int64)
+    sched = plan["sched_band"].tolist()
     for (x, b0, b1, _tile), rec in zip(plan["item"].tolist(), items):
-        if x & 0xff == 1:
+        kind = x & 0xff
+        if kind == 3:                 # swapped operands: both CTAs hold columns of every band of the group
+            for b in sched[b0:b0 + (b1 & 0xff)]:
+                band_done[b] = max(band_done[b], rec["ns_done0"], rec["ns_done1"])
+        elif kind & 8 and kind & 1:   # stacked bands: the first two are the leader CTA's, the rest its peer's
+            for i in range(b1):
+                band_done[b0 + i] = max(band_done[b0 + i], rec["ns_done0"] if i < 2 else rec["ns_done1"])
+        elif kind & 3 == 1:
             band_done[b0] = max(band_done[b0], rec["ns_done0"])
             if b1 >= 0:
                 band_done[b1] = max(band_done[b1], rec["ns_done1"])
@@ -605,8 +613,8 @@ def test_small_group_items_can_be_switched_off(name):
     assert kinds[B.FLAG_NO_SMALL_GROUP_TILES] <= {0, 1}
     # every one of these problems has at least one run of small groups
     assert kinds[B.FLAG_TEST_ALL_SMALL_GROUP_TILES] & {2, 3}
-    # left to itself the plan computes pairs of small bands 64 rows high (kinds 4, 5); these shapes hold too few
-    # items for swapped-operand groups to pay
+    # left to itself the plan computes pairs of small bands 64 rows high (kinds 4, 5) or stacks them (8, 9); these
+    # shapes hold too few items for swapped-operand groups to pay
     ctx = Hn.make_context(shape, max_rows=dsp.M)
     prob = Hn.upload(inp, dsp)
     Hn.run(ctx, prob, mode=B.MODE_OVERLAP, consumer_sm_count=4)
@@ -616,4 +624,19 @@ def test_small_group_items_can_be_switched_off(name):
     U.check_indices(shape, dsp, plan, gp, prob.slot_out.cpu().numpy(), prob.rows_per_rank_out.cpu().numpy(),
                     prob.segs_per_rank_out.cpu().numpy(), ctx.moe_ovl_get_report())
     U.check_values(shape, dsp, plan, toks, *o, Hn.device_to_bits(prob.out), Hn.device_to_bits(prob.ret))
-    assert set((gp["item"][:, 0] & 0xff).tolist()) & {4, 5}
+    default_kinds = set((gp["item"][:, 0] & 0xff).tolist())
+    assert default_kinds & {4, 5, 8, 9} and not default_kinds & {2, 3}
+    if name != "tiny":
+        # three remote groups per expert, all small: stacked into one full-height item per tile (kinds 8, 9) unless
+        # the flag forbids it
+        assert default_kinds & {8, 9}
+        ctx = Hn.make_context(shape, max_rows=dsp.M, flags=B.FLAG_NO_STACKED_BANDS)
+        prob = Hn.upload(inp, dsp)
+        Hn.run(ctx, prob, mode=B.MODE_IN_KERNEL)
+        torch.cuda.synchronize()
+        assert ctx.moe_ovl_query_status()[0] == 0
+        gp = ctx.moe_ovl_get_plan()
+        U.check_indices(shape, dsp, plan, gp, prob.slot_out.cpu().numpy(), prob.rows_per_rank_out.cpu().numpy(),
+                        prob.segs_per_rank_out.cpu().numpy(), ctx.moe_ovl_get_report())
+        U.check_values(shape, dsp, plan, toks, *o, Hn.device_to_bits(prob.out), Hn.device_to_bits(prob.ret))
+        assert set((gp["item"][:, 0] & 0xff).tolist()) <= {0, 1, 4, 5}
