@@ -313,6 +313,10 @@ typedef struct {
                                       (the bubble between two items, or the kernel's start-up) */
     int64_t ns_accumulator_wait;   /* item: time it waited for a free accumulator buffer, i.e. for the epilogue of
                                       the item before the previous one: non-zero means the epilogue is the bound */
+    int64_t ns_inputs_ready;       /* item: the load thread of the pair's first CTA saw the rows the item reads
+                                      complete (gathered into the layout, or every hidden tile of the band written)
+                                      and issued its first copies; ns_ready - ns_inputs_ready is the latency of
+                                      those copies; unit: 0 */
 } moe_ovl_trace_record;
 /* Waits for the last call, then writes its records to HOST memory: items in issue order, then units in
  * claim order.  *written = bytes written.  host_buf == NULL: only reports the bytes needed.

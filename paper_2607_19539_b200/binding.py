@@ -79,14 +79,14 @@ class TraceRecord(C.Structure):
                 ("rows", C.c_int32), ("chunks", C.c_int32), ("ns_claim", C.c_int64), ("ns_ready", C.c_int64),
                 ("ns_done0", C.c_int64), ("ns_done1", C.c_int64), ("ns_operand_wait", C.c_int64),
                 ("ns_epilogue_start", C.c_int64), ("ns_first_operand_wait", C.c_int64),
-                ("ns_accumulator_wait", C.c_int64)]
+                ("ns_accumulator_wait", C.c_int64), ("ns_inputs_ready", C.c_int64)]
 
 
 TRACE_DTYPE = np.dtype([("kind", np.int32), ("index", np.int32), ("cta", np.int32), ("who", np.int32),
                         ("rows", np.int32), ("chunks", np.int32), ("ns_claim", np.int64), ("ns_ready", np.int64),
                         ("ns_done0", np.int64), ("ns_done1", np.int64), ("ns_operand_wait", np.int64),
                         ("ns_epilogue_start", np.int64), ("ns_first_operand_wait", np.int64),
-                        ("ns_accumulator_wait", np.int64)])
+                        ("ns_accumulator_wait", np.int64), ("ns_inputs_ready", np.int64)])
 
 
 class PlanView(C.Structure):

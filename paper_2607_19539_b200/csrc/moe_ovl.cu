@@ -888,6 +888,7 @@ int moe_ovl_get_trace(moe_ovl_ctx *ctx, void *host_buf, size_t bytes, size_t *wr
         r.ns_epilogue_start = rel(items2[i].a);
         r.ns_first_operand_wait = (int64_t)items2[i].b;
         r.ns_accumulator_wait = (int64_t)items2[i].c;
+        r.ns_inputs_ready = rel(items2[i].d);
     }
     for (size_t u = 0; u < n_units; ++u) {
         const TraceRec &t = items[n_items + u];

@@ -311,6 +311,38 @@ __device__ __forceinline__ void gather_unit(const Params &p, int band, int r0, i
     if (lane == 0) red_release_add_u32(&p.xready[band], (unsigned)ROWS);
 }
 
+// Gather loop of one warp: Xa[band * 128 + r] = x[row_at[...]] for units of rows claimed in schedule order from a
+// global counter; padding rows are zero-filled (Section 3.2.1).  It never waits, so the row counts the load warps
+// poll always make progress.  The first super-band is gathered in small units (2 rows: done after two memory
+// round trips at d = 4096) so that the first tiles can start a few microseconds after the kernel does; the rest in
+// units of GATHER_ROWS rows, which cost fewer claims.
+__device__ __forceinline__ void gather_units(const Params &p, int kflags, int lane)
+{
+    const int nbands = p.meta[META_BANDS];
+    const int head_bands = min(nbands, p.group_bands);
+    const int head_units = head_bands * (TB_M / GATHER_HEAD_ROWS);
+    const int nunits = head_units + (nbands - head_bands) * (TB_M / GATHER_ROWS);
+    int unit = 0;
+    if (lane == 0) unit = atomicAdd(p.next_gather, 1);
+    unit = __shfl_sync(0xffffffffu, unit, 0);
+    while (unit < nunits) {
+        int next = 0;
+        if (lane == 0) next = atomicAdd(p.next_gather, 1);      // claimed while this unit's rows are moving
+        if ((kflags & PROD_SKIP_FIRST_BAND) && unit < TB_M / GATHER_HEAD_ROWS) {
+            // test hook: leave band 0 of the schedule ungathered, so that the wait for it runs out
+        } else if (unit < head_units) {
+            const int per = TB_M / GATHER_HEAD_ROWS;
+            gather_unit<GATHER_HEAD_ROWS, 16 / GATHER_HEAD_ROWS>(p, p.sched_band[unit / per],
+                                                                 (unit % per) * GATHER_HEAD_ROWS, lane);
+        } else {
+            const int u = unit - head_units, per = TB_M / GATHER_ROWS;
+            gather_unit<GATHER_ROWS, 16 / GATHER_ROWS>(p, p.sched_band[head_bands + u / per],
+                                                       (u % per) * GATHER_ROWS, lane);
+        }
+        unit = __shfl_sync(0xffffffffu, next, 0);
+    }
+}
+
 struct ProducerMaps {
     CUtensorMap xa, h, w1, w2;   // all 2-D bf16 row-major, box 64 x 128, 128-byte swizzle
     CUtensorMap xa8, h8;         // Xa and H again in boxes of 64 x 8: token rows of the swapped-operand items
@@ -586,6 +618,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     }
                 }
                 asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
+                if (kTrace && lane == 0 && rank == 0 && ok) p.trace_items2[cur.it].d = globaltimer_ns();
                 __syncwarp();
                 ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
                 if (!ok) break;
@@ -647,6 +680,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 if (!ok) continue;
             }
             asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
+            if (kTrace && rank == 0) p.trace_items2[cur.it].d = globaltimer_ns();
             int have_next = 0;
             const int look = cur.ksteps > PROD_LOOKAHEAD ? cur.ksteps - PROD_LOOKAHEAD : 0;
             for (int ks = 0; ks < cur.ksteps; ++ks) {
@@ -755,35 +789,8 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             }
         }
     } else if (warp >= 7) {
-        // ---------------- gather warps: Xa[band * 128 + r] = x[row_at[...]] for units of GATHER_ROWS rows, claimed in
-        // schedule order; padding rows are zero-filled (Section 3.2.1).  These warps never wait, so the row
-        // counts the TMA warps poll always make progress.
-        // The first super-band is gathered in small units (2 rows: done after two memory round trips at d = 4096)
-        // so that the first tiles can start a few microseconds after the kernel does; the rest in units of
-        // GATHER_ROWS rows, which cost fewer claims.
-        const int nbands = p.meta[META_BANDS];
-        const int head_bands = min(nbands, p.group_bands);
-        const int head_units = head_bands * (TB_M / GATHER_HEAD_ROWS);
-        const int nunits = head_units + (nbands - head_bands) * (TB_M / GATHER_ROWS);
-        int unit = 0;
-        if (lane == 0) unit = atomicAdd(p.next_gather, 1);
-        unit = __shfl_sync(0xffffffffu, unit, 0);
-        while (unit < nunits) {
-            int next = 0;
-            if (lane == 0) next = atomicAdd(p.next_gather, 1);      // claimed while this unit's rows are moving
-            if ((kflags & PROD_SKIP_FIRST_BAND) && unit < TB_M / GATHER_HEAD_ROWS) {
-                // test hook: leave band 0 of the schedule ungathered, so that the wait for it runs out
-            } else if (unit < head_units) {
-                const int per = TB_M / GATHER_HEAD_ROWS;
-                gather_unit<GATHER_HEAD_ROWS, 16 / GATHER_HEAD_ROWS>(p, p.sched_band[unit / per],
-                                                                     (unit % per) * GATHER_HEAD_ROWS, lane);
-            } else {
-                const int u = unit - head_units, per = TB_M / GATHER_ROWS;
-                gather_unit<GATHER_ROWS, 16 / GATHER_ROWS>(p, p.sched_band[head_bands + u / per],
-                                                           (u % per) * GATHER_ROWS, lane);
-            }
-            unit = __shfl_sync(0xffffffffu, next, 0);
-        }
+        // ---------------- gather warps: move the dispatched rows into the aligned layout
+        gather_units(p, kflags, lane);
         // In-kernel return: with Xa complete these warps have nothing left to do, so they take over the
         // consumer's job on this SM -- no SM is taken from the GEMM.  They only ever wait on tile flags, which
         // the epilogue warps raise without waiting on anybody.

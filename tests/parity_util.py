@@ -10,6 +10,15 @@ TOL_REL = 2e-2    # max relative error on values (bf16 output, fp32 accumulate),
 TOL_NORM = 5e-3   # per-token 2-norm distance: what the rounding model supports (both sides round H, Y and out to
                   # bf16 at the same points; they differ where fp32 summation order flips a rounding, one bf16
                   # ulp = 2^-8..2^-7 relative on a fraction of the elements)
+TOL_NORM_NARROW = 1e-2   # the same for FFN experts with fewer than 256 hidden columns (only seeded random shapes
+                  # have them): an output element is then a sum of so few terms that ONE flipped rounding of a
+                  # dominant hidden value (2^-8 of a term that can be a third of the sum) moves every element of the
+                  # row by a fraction of an ulp, and most of them then round the other way: measured up to 5.6e-3
+                  # on one row in 3500, every element within one ulp
+
+
+def tol_norm(shape):
+    return TOL_NORM if (shape.N_out or shape.F >= 256) else TOL_NORM_NARROW
 
 
 def elem_err(a, b):
@@ -143,7 +152,7 @@ def oracle_values(inp, tokens):
 
 def check_values(shape, dsp, plan, tokens, o_out, o_y, o_yexp, gpu_out_bits, gpu_ret_bits):
     """out and the returned rows of the given tokens against the oracle: every element within TOL_REL of
-    (|b| + rms of its row), every row within TOL_NORM in the 2-norm."""
+    (|b| + rms of its row), every row within tol_norm(shape) in the 2-norm."""
     tokens = np.asarray(tokens)
     got = I.bf16_bits_to_f32(gpu_out_bits[tokens])
     ref = I.bf16_bits_to_f32(o_out)
@@ -153,7 +162,7 @@ def check_values(shape, dsp, plan, tokens, o_out, o_y, o_yexp, gpu_out_bits, gpu
     if (~none).any():
         worst = float(rel_dist(got[~none], ref[~none]).max())
         worst_el = float(elem_err(got[~none], ref[~none]).max())
-    assert worst <= TOL_NORM, worst
+    assert worst <= tol_norm(shape), worst
     assert worst_el <= TOL_REL, worst_el
     # returned rows: ret[r][slot] holds the unscaled expert output of that (token, expert)
     kmax = o_yexp.shape[1]
@@ -171,7 +180,7 @@ def check_values(shape, dsp, plan, tokens, o_out, o_y, o_yexp, gpu_out_bits, gpu
         b = I.bf16_bits_to_f32(o_y[s_, j_])
         worst_y = max(worst_y, float(rel_dist(a, b).max()))
         worst_y_el = max(worst_y_el, float(elem_err(a, b).max()))
-    assert worst_y <= TOL_NORM, worst_y
+    assert worst_y <= tol_norm(shape), worst_y
     assert worst_y_el <= TOL_REL, worst_y_el
     return worst, worst_y, worst_el, worst_y_el
 

@@ -30,7 +30,7 @@ def test_struct_sizes_match_header_layout():
     assert ctypes.sizeof(B.Config) == 16 * 4
     assert ctypes.sizeof(B.Args) == 8 + 7 * 8 + 8 + 8 + 8 + 8 + 3 * 8 + 8
     assert ctypes.sizeof(B.Report) == 11 * 4 + 11 * 4
-    assert ctypes.sizeof(B.TraceRecord) == 6 * 4 + 8 * 8 == B.TRACE_DTYPE.itemsize
+    assert ctypes.sizeof(B.TraceRecord) == 6 * 4 + 9 * 8 == B.TRACE_DTYPE.itemsize
 
 
 def _cfg(**kw):
