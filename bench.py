@@ -267,7 +267,7 @@ def dry_run(args, shape):
     D.finalize()
 
 
-def interleaved_medians(torch, run_variant, names, rounds):
+def interleaved_medians(torch, run_variant, names, rounds, return_all=False):
     """Variants measured call by call, interleaved (the GPU is power-limited under this load, so a block
     of steps measured later runs slower than one measured earlier); returns the median ms of each."""
     evs = {n: [] for n in names}
@@ -283,7 +283,10 @@ def interleaved_medians(torch, run_variant, names, rounds):
             if r >= 2:
                 evs[name].append((a, b))
     torch.cuda.synchronize()
-    return {n: statistics.median(a.elapsed_time(b) for a, b in v) for n, v in evs.items()}
+    times = {n: [a.elapsed_time(b) for a, b in v] for n, v in evs.items()}
+    if return_all:
+        return times
+    return {n: statistics.median(v) for n, v in times.items()}
 
 
 def run_sweep(args):
@@ -346,7 +349,20 @@ def run_sweep(args):
         code, detail = ctx.moe_ovl_query_status()
         if code != 0:
             raise SystemExit(f"device status {code} detail {detail:#x} at {shape.name}")
-        med = interleaved_medians(torch, run_variant, names, args.rounds)
+        # short layers get more rounds (at least 15 ms of the baseline per variant): their medians are noisier
+        for _ in range(3):
+            run_variant("non_overlap")
+        torch.cuda.synchronize()
+        est_ms = ctx.moe_ovl_get_report().ms_total
+        rounds = int(min(8 * args.rounds, max(args.rounds, 15.0 / max(est_ms, 1e-3))))
+        times = interleaved_medians(torch, run_variant, names, rounds, return_all=True)
+        med = {n: statistics.median(v) for n, v in times.items()}
+        # auto against the best fixed variant without selection bias: the best is picked on the even rounds and
+        # both are compared on the odd ones (the minimum of several noisy medians is biased low)
+        fixed = [n for n in names if n != "auto"]
+        even = {n: statistics.median(times[n][0::2]) for n in fixed}
+        pick = min(even, key=even.get)
+        heldout = statistics.median(times["auto"][1::2]) / statistics.median(times[pick][1::2])
         run_variant("non_overlap")
         rep = ctx.moe_ovl_get_report()
         run_variant("auto")
@@ -359,7 +375,8 @@ def run_sweep(args):
                "gemm_us": round(rep.ms_producer * 1e3, 1),
                "ratio": {k: round(v / nov, 4) for k, v in med.items() if k != "non_overlap"},
                "best": best, "auto_choice": {"mode": rep_auto.mode_used, "consumer_ctas": rep_auto.consumer_ctas},
-               "auto_vs_best": round(med["auto"] / med[best], 4), "rounds": args.rounds}
+               "auto_vs_best": round(med["auto"] / med[best], 4),
+               "auto_vs_best_heldout": round(heldout, 4), "heldout_pick": pick, "rounds": rounds}
         print(json.dumps(row), flush=True)
         del ctx, prob
         torch.cuda.empty_cache()

@@ -61,7 +61,8 @@ constexpr int PROD_TMEM_COLS = 512;
 constexpr int PROD_RAISE_FLAGS = 1;    // publish a ready flag per finished output tile; idle CTAs help drain segments
 constexpr int PROD_WARP_MOVERS = 2;    // in-kernel return: the gather warps move finished segments once Xa is complete
 constexpr int PROD_SKIP_FIRST_BAND = 4; // test hook: the first band of the schedule is never gathered
-constexpr int PROD_AUX_BYTES = 1792;   // barriers, claim ring, mover ints, tables of the swapped-operand items
+constexpr int PROD_AUX_BYTES = 2048;   // barriers, claim ring (index, item record, inputs-complete mark), mover ints,
+                                       // tables of the swapped-operand items
 constexpr int PROD_SMEM_BYTES = PROD_STAGES * PROD_STAGE_BYTES + 1024 /*alignment slack*/ + PROD_AUX_BYTES;
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -426,11 +427,26 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
     // epilogue's column -> buffer row maps (one per accumulator buffer, SWAP_MAX_N columns each)
     const uint32_t swap_tab = mover_ints + 8;                      // [2][SWAP_MAX_BANDS] int2
     const uint32_t swap_rowmap = swap_tab + 2 * SWAP_MAX_BANDS * 8;   // [2][SWAP_MAX_N] int
+    // the scheduler also hands out the item's record and whether its inputs were already complete at the claim, so
+    // that no role has to fetch them from global memory at an item boundary
+    const uint32_t ring_item = swap_rowmap + 2 * SWAP_MAX_N * 4;   // PROD_RING int4 (16-byte aligned: see the assert)
+    const uint32_t ring_dep = ring_item + 16 * PROD_RING;          // PROD_RING ints
+    static_assert((16 * PROD_STAGES + 16 + 16 + 8 + 8 + 8 + 8 * PROD_RING + 4 * PROD_RING + 8 + 2 * SWAP_MAX_BANDS * 8 +
+                   2 * SWAP_MAX_N * 4) % 16 == 0, "item records must be 16-byte aligned");
     static_assert(16 * PROD_STAGES + 16 + 16 + 8 + 8 + 8 + 8 * PROD_RING + 4 * PROD_RING + 8 + 2 * SWAP_MAX_BANDS * 8 +
-                  2 * SWAP_MAX_N * 4 <= PROD_AUX_BYTES, "auxiliary shared memory");
+                  2 * SWAP_MAX_N * 4 + 16 * PROD_RING + 4 * PROD_RING <= PROD_AUX_BYTES, "auxiliary shared memory");
+    static_assert(PROD_SMEM_BYTES <= 232448, "dynamic shared memory of one CTA");
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     volatile uint32_t *tmem_slot_gen = reinterpret_cast<volatile uint32_t *>(smem_gen + (tmem_slot - smem_base));
     volatile int *ring_gen = reinterpret_cast<volatile int *>(smem_gen + (ring - smem_base));
+    volatile int *ring_item_gen = reinterpret_cast<volatile int *>(smem_gen + (ring_item - smem_base));
+    volatile int *ring_dep_gen = reinterpret_cast<volatile int *>(smem_gen + (ring_dep - smem_base));
+    // record of the n-th item of this cluster (valid once claimed(n) has returned it)
+    auto claimed_item = [&](int n) -> int4 {
+        const int slot = n % PROD_RING;
+        return make_int4(ring_item_gen[4 * slot], ring_item_gen[4 * slot + 1], ring_item_gen[4 * slot + 2],
+                         ring_item_gen[4 * slot + 3]);
+    };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();          // 0 = leader: owns the barriers the pair synchronises on
@@ -515,7 +531,8 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             if (it < 0) return -1;
             if (it >= n_items) return 0;
             if (rank == 0) mbar_arrive(bar_go);  // lets the scheduler claim the item after this one
-            const int4 item = p.items[it];       // {kind | expert << 8, band 0, band 1 or -1, tile}
+            const int4 item = claimed_item(n);   // {kind | expert << 8, band 0, band 1 or -1, tile}
+            const bool pre_ok = ring_dep_gen[n % PROD_RING] != 0;   // inputs were complete when the item was claimed
             const int kind = item.x & 0xff, e = item.x >> 8, tile = item.w;
             j.it = it;
             j.swap = kind == KIND_G1S || kind == KIND_G2S;
@@ -591,8 +608,8 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     if (band2 >= 0) j.dep2 = &p.xready[band2];
                 }
             }
-            j.dep_ok = ld_acquire_u32(j.dep) >= j.dep_want &&      // the counters only grow
-                       (j.dep2 == nullptr || ld_acquire_u32(j.dep2) >= j.dep_want);
+            j.dep_ok = pre_ok || (ld_acquire_u32(j.dep) >= j.dep_want &&      // the counters only grow
+                                  (j.dep2 == nullptr || ld_acquire_u32(j.dep2) >= j.dep_want));
             return 1;
         };
         Job cur, nxt;
@@ -728,7 +745,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             for (int n = 0; ok; ++n) {
                 const int it = claimed(n);
                 if (it < 0 || it >= n_items) break;
-                const int4 item = p.items[it];
+                const int4 item = claimed_item(n);
                 const int kind = item.x & 0xff;
                 const bool swap = kind == KIND_G1S || kind == KIND_G2S;
                 const bool first_gemm = (kind & 3) == KIND_G1 || kind == KIND_G1S;
@@ -771,6 +788,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
         // ---------------- scheduler (leader CTA): claim items in schedule order, one ahead of the TMA warp
         if (lane == 0 && rank == 0) {
             const uint32_t peer_ring = map_to_cta(ring, 1), peer_bar = map_to_cta(bar_ring, 1);
+            const uint32_t peer_item = map_to_cta(ring_item, 1), peer_dep = map_to_cta(ring_dep, 1);
             for (int n = 0;; ++n) {
                 // claim n is taken when the TMA thread starts item n-1: exactly one item ahead, so the claim's
                 // latency is hidden and no role can fall a whole ring behind
@@ -780,9 +798,34 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                     p.trace_items[it].a = globaltimer_ns();
                     p.trace_item_aux[it].x = (int)blockIdx.x;
                 }
+                // The item's record, and whether the rows it reads are complete already (they usually are: the gather
+                // runs far ahead, and a band's second-GEMM tiles are issued well after its first-GEMM tiles), travel
+                // with the claim.  This thread is a whole item ahead of the loads, so its round trips cost nothing.
+                int4 item = make_int4(0, 0, 0, 0);
+                int pre_ok = 0;
+                if (it < n_items) {
+                    item = p.items[it];
+                    const int kind = item.x & 0xff;
+                    if (kind != KIND_G1S && kind != KIND_G2S) {
+                        const bool on_x = (kind & 3) == KIND_G1 || p.n1 == 0;
+                        const unsigned *cnt = on_x ? p.xready : p.hcount;
+                        const unsigned want = on_x ? (unsigned)TB_M : (unsigned)p.n1;
+                        const int b0 = item.y, nb = (kind & KIND_STACK) ? item.z : 1;
+                        unsigned lo = ld_acquire_u32(cnt + b0);
+                        for (int i = 1; i < nb; ++i) lo = min(lo, ld_acquire_u32(cnt + b0 + i));
+                        if (!(kind & KIND_STACK) && item.z >= 0) lo = min(lo, ld_acquire_u32(cnt + item.z));
+                        pre_ok = lo >= want;
+                    }
+                }
                 const int slot = n % PROD_RING;
                 ring_gen[slot] = it;
+                ring_item_gen[4 * slot] = item.x; ring_item_gen[4 * slot + 1] = item.y;
+                ring_item_gen[4 * slot + 2] = item.z; ring_item_gen[4 * slot + 3] = item.w;
+                ring_dep_gen[slot] = pre_ok;
                 asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_ring + 4 * slot), "r"(it) : "memory");
+                asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(peer_item + 16 * slot), "r"(item.x),
+                             "r"(item.y), "r"(item.z), "r"(item.w) : "memory");
+                asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_dep + 4 * slot), "r"(pre_ok) : "memory");
                 mbar_arrive(bar_ring + 8 * slot);
                 mbar_arrive_cluster(peer_bar + 8 * slot);        // release at cluster scope: orders the store above
                 if (it >= n_items) break;
@@ -811,7 +854,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             const int it = claimed(n);
             if (!epilogue_all(it >= 0)) break;            // leave together if any thread gave up
             if (it >= n_items) break;
-            const int4 item = p.items[it];
+            const int4 item = claimed_item(n);
             const int kind = item.x & 0xff, tile = item.w;
             const bool swap = kind == KIND_G1S || kind == KIND_G2S;
             const bool low = (kind & KIND_LOW) != 0;
