@@ -55,7 +55,7 @@ constexpr int PROD_THREADS = 224 + 32 * PROD_GATHER_WARPS;   // TMA, MMA, 4 epil
 constexpr int GATHER_ROWS = 8;                         // rows per gather unit
 constexpr int GATHER_HEAD_ROWS = 2;                    // ... in the first super-band of the schedule
 constexpr int PROD_RING = 16;                          // claimed-item ring; roles are never more than 6 items apart
-constexpr int PROD_LOOKAHEAD = 5;                      // stages before an item's last load at which the next item is looked up
+constexpr int PROD_LOOKAHEAD = 3;                      // stages before an item's last load at which the next item is looked up
 constexpr int PROD_TMEM_COLS = 512;
 // kernel flags
 constexpr int PROD_RAISE_FLAGS = 1;    // publish a ready flag per finished output tile; idle CTAs help drain segments
@@ -634,7 +634,11 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                         ok = wait_global(cur.dep + b, cur.dep_want, true, p, cur.dep_site, b);
                     }
                 }
-                asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
+                // (No proxy fence here: every thread that writes rows the copies below read -- the gather warps, the
+                // epilogue warps of first-GEMM tiles -- issues fence.proxy.async after its stores and before the
+                // release this thread has acquired, which is what orders those generic-proxy writes before the
+                // async-proxy reads.  A second fence on this side stalled the load thread at every item: 2 % of the
+                // kernel where items are short.)
                 if (kTrace && lane == 0 && rank == 0 && ok) p.trace_items2[cur.it].d = globaltimer_ns();
                 __syncwarp();
                 ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -696,7 +700,7 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
                 if (ok && cur.dep2) ok = wait_global(cur.dep2, cur.dep_want, true, p, cur.dep_site, cur.dep_index + 1);
                 if (!ok) continue;
             }
-            asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy reads
+            // (no proxy fence on this side: the writers of the rows issue it before their release, see above)
             if (kTrace && rank == 0) p.trace_items2[cur.it].d = globaltimer_ns();
             int have_next = 0;
             const int look = cur.ksteps > PROD_LOOKAHEAD ? cur.ksteps - PROD_LOOKAHEAD : 0;
