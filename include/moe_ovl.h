@@ -82,7 +82,7 @@ typedef struct {
     int32_t mid_seg_bands;      /* bands per middle segment (x of Figure 3b); 0 = chosen by the library: 1, because
                                    with HBM as the link a transfer has no fixed cost to amortise (larger middle
                                    segments were never faster in the measured grids) */
-    int32_t group_bands;        /* bands whose tiles are interleaved so that they share weight tiles in L2; 0 = default (16) */
+    int32_t group_bands;        /* bands whose tiles are interleaved so that they share weight tiles in L2; 0 = default (16), at most 64 */
     int32_t wait_timeout_us;    /* bound on every device-side wait; 0 = default (2 s) */
     int32_t producer_sm_limit;  /* NON_OVERLAP only: cap on GEMM CTAs (diagnostic baseline); 0 = all SMs */
     int32_t single_gemm_out;    /* 0: SwiGLU FFN experts.  N > 0: the operator the paper evaluates (Table 2) -- each

@@ -216,7 +216,7 @@ Params make_params(moe_ovl_ctx *ctx)
     p.kmax = L.kmax; p.d = c.d_model; p.F = L.f_eff;
     p.dout = L.dout; p.k2 = L.k2; p.single = L.single;
     p.mgb = std::max(1, c.mid_seg_bands);
-    p.group_bands = c.group_bands > 0 ? c.group_bands : 16;
+    p.group_bands = c.group_bands > 0 ? (c.group_bands < 64 ? c.group_bands : 64) : 16;
     p.words = L.words; p.n1 = L.n1; p.n2 = L.n2; p.max_bands = L.max_bands; p.max_items = L.max_items;
     p.timeout_ns = (unsigned long long)(c.wait_timeout_us > 0 ? c.wait_timeout_us : 2000000) * 1000ull;
     p.Xa = at<uint16_t>(ctx, L.Xa); p.H = at<uint16_t>(ctx, L.H); p.Y = at<uint16_t>(ctx, L.Y);

@@ -32,7 +32,8 @@ struct PlanScratch {
     int *sb_units;   // super-band of band pairs: its units (a pair, or two pairs of small bands stacked)
     int *unit_tab;   // [bands], a super-band's units at its first schedule position: first band's offset | bands << 8
                      // | (1 << 16 if the unit's last band is the expert's local band riding with its remote ones)
-    int *sb_role;    // 1: last super-band of an expert's remote run, 2: super-band of a local run, else 0
+    int *sb_role;    // bits 0-1: 1 last super-band of an expert's remote run, 2 super-band of a local run, else 0;
+                     // bit 2: the run may hold stacks of small bands or take a rider (its units are in unit_tab)
 };
 
 __device__ __forceinline__ int ceil16(int v) { return (v + 15) & ~15; }
@@ -243,6 +244,22 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
         const int pairs_run = (nbands + 1) / 2;
         const bool fewer = (p.low_ok ? 2 * sgroups < pairs_run : sgroups < pairs_run) || p.swap_ok == 2;
         run_nsb[run] = (small && nbands > 0 && fewer) ? sgroups : -1;
+        // Can the run hold a stack of small bands or take a rider?  Only the last band of a group can be small, so a
+        // stack needs three single-band groups in a row, and a rider the run's last band small.  (Decided exactly,
+        // band by band, in phase E2; runs that cannot are skipped there.)
+        int chain = 0, best = 0;
+        bool last_small = false;
+        for (int q = remote ? 0 : R - 1; q < (remote ? R - 1 : R); ++q) {
+            const int r = q < R - 1 ? (q < self ? q : q + 1) : self;
+            const int g = e * R + r;
+            if (nb[g] == 0) continue;
+            last_small = n[g] - (nb[g] - 1) * TB_M <= SMALL_BAND_ROWS;
+            chain = (nb[g] == 1 && last_small) ? chain + 1 : 0;
+            best = max(best, chain);
+        }
+        const int n_local = n[e * R + self];
+        const bool may_ride = remote && last_small && n_local > 0 && n_local <= SMALL_BAND_ROWS;
+        if (run_nsb[run] < 0 && !(p.low_ok >= 2 && (best >= 3 || may_ride))) run_nsb[run] = -2;
     }
     __syncthreads();
     if (tid == 0) {
@@ -252,7 +269,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
         for (int run = 0; run < 2 * El; ++run)
             if (run_nsb[run] >= 0) group_items += run_nsb[run] * (p.n1 / 2 + p.n2);
         if (group_items < p.lag_items && p.swap_ok != 2)
-            for (int run = 0; run < 2 * El; ++run) run_nsb[run] = -1;
+            for (int run = 0; run < 2 * El; ++run)
+                if (run_nsb[run] >= 0) run_nsb[run] = p.low_ok >= 2 ? -1 : -2;
         int spos = 0, segoff = 0, sbcount = 0;
         for (int run = 0; run < 2 * El; ++run) {
             run_start[run] = spos;
@@ -353,7 +371,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
             sc.sb_expert[sb] = run_exp[run];
             sc.sb_kind[sb] = 0;
             sc.sb_ntok[sb] = 0;
-            sc.sb_role[sb] = run >= El ? 2 : (q == nsb - 1 ? 1 : 0);
+            sc.sb_role[sb] = (run >= El ? 2 : (q == nsb - 1 ? 1 : 0)) | (run_nsb[run] == -1 ? 4 : 0);
+            sc.sb_units[sb] = (sc.sb_nb[sb] + 1) / 2;      // band pairs, unless phase E2 finds stacks or a rider
         }
     }
     for (int e = tid; e < El; e += blockDim.x) erider[e] = 0;
@@ -367,42 +386,38 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     //     be padding, so no remote tile is issued later than without it (the purpose of rule (i) of Section 3.2.2
     //     holds), and the expert's weights are streamed once instead of twice.  The bands of an expert are
     //     consecutive in the layout, remote ones first, so the unit's bands still have consecutive ids.
-    for (int sb = tid; sb < s_nsb; sb += blockDim.x) {
-        if (sc.sb_kind[sb]) continue;
+    //     One warp per super-band of a run that can hold such units (the others keep plain pairs): the lanes look the
+    //     bands' row counts up together, lane 0 then forms the units from a bit mask.
+    for (int sb = warp; sb < s_nsb; sb += nwarps) {
+        const int role = sc.sb_role[sb];
+        if (sc.sb_kind[sb] || !(role & 4)) continue;
         const int start = sc.sb_start[sb], cnt = sc.sb_nb[sb], e = sc.sb_expert[sb];
-        auto small_band = [&](int o) { return p.band_valid[p.sched_band[start + o]] <= SMALL_BAND_ROWS; };
+        unsigned long long small_mask = 0;      // bit o: band o of the super-band holds at most SMALL_BAND_ROWS rows
+        for (int base = 0; base < min(cnt, 64); base += 32) {
+            const int o = base + lane;
+            const bool sm = o < cnt && p.band_valid[p.sched_band[start + o]] <= SMALL_BAND_ROWS;
+            small_mask |= (unsigned long long)__ballot_sync(0xffffffffu, sm) << base;
+        }
+        if (lane != 0) continue;
+        auto all_small = [&](int o, int k) {    // bands o .. o + k - 1 (beyond 64 bands per super-band: never stacked)
+            return o + k <= 64 && ((small_mask >> o) & ((1ull << k) - 1)) == (1ull << k) - 1;
+        };
         int units = 0, last_o = 0, last_take = 0;
         for (int o = 0; o < cnt;) {
             int take = min(2, cnt - o);
-            if (p.low_ok >= 2 && cnt - o >= 3) {
-                bool all_small = true;
-                const int four = min(4, cnt - o);
-                for (int q = 0; q < four; ++q) all_small = all_small && small_band(o + q);
-                if (all_small) take = four;
-            }
+            if (p.low_ok >= 2 && cnt - o >= 3 && all_small(o, min(4, cnt - o))) take = min(4, cnt - o);
             sc.unit_tab[start + units++] = o | (take << 8);
             last_o = o;
             last_take = take;
             o += take;
         }
         const int n_local = n[e * R + self];
-        if (p.low_ok == 3 && sc.sb_role[sb] == 1 && units > 0 && last_take <= 3 && n_local > 0 &&
-            n_local <= SMALL_BAND_ROWS && run_nsb[El + e] < 0) {
-            bool all_small = true;
-            for (int q = 0; q < last_take; ++q) all_small = all_small && small_band(last_o + q);
-            if (all_small) {
-                sc.unit_tab[start + units - 1] = last_o | ((last_take + 1) << 8) | (1 << 16);
-                erider[e] = 1;
-            }
+        if (p.low_ok == 3 && (role & 3) == 1 && units > 0 && last_take <= 3 && n_local > 0 &&
+            n_local <= SMALL_BAND_ROWS && run_nsb[El + e] < 0 && all_small(last_o, last_take)) {
+            sc.unit_tab[start + units - 1] = last_o | ((last_take + 1) << 8) | (1 << 16);
+            erider[e] = 1;
         }
         sc.sb_units[sb] = units;
-    }
-    __syncthreads();
-    for (int sb = tid; sb < s_nsb; sb += blockDim.x) {
-        if (sc.sb_kind[sb]) continue;
-        if (sc.sb_role[sb] == 2 && erider[sc.sb_expert[sb]]) sc.sb_units[sb] = 0;   // the band was issued with the remote ones
-        sc.sb_c1[sb] = sc.sb_units[sb] * p.n1;
-        sc.sb_c2[sb] = sc.sb_units[sb] * p.n2;
     }
     __syncthreads();
 
@@ -415,8 +430,18 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     {
         const int nsb = s_nsb;
         const bool staged = nsb <= PLAN_SB_STAGE;
-        if (staged)
-            for (int i = tid; i < nsb; i += blockDim.x) { s_sb_c1[i] = sc.sb_c1[i]; s_sb_c2[i] = sc.sb_c2[i]; }
+        for (int i = tid; i < nsb; i += blockDim.x) {
+            int c1 = sc.sb_c1[i], c2 = sc.sb_c2[i];
+            const int kind = sc.sb_kind[i], role = sc.sb_role[i], e = sc.sb_expert[i];
+            int units = sc.sb_units[i];
+            if (!kind) {
+                if ((role & 3) == 2 && erider[e]) units = 0;   // the band was issued with the remote ones
+                sc.sb_units[i] = units;
+                sc.sb_c1[i] = c1 = units * p.n1;
+                sc.sb_c2[i] = c2 = units * p.n2;
+            }
+            if (staged) { s_sb_c1[i] = c1; s_sb_c2[i] = c2; }
+        }
         __syncthreads();
         if (tid == 0) {
             int *c1v = staged ? s_sb_c1 : sc.sb_c1, *c2v = staged ? s_sb_c2 : sc.sb_c2;
@@ -444,38 +469,51 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     }
     __syncthreads();
 
-    // G: the item list, one warp per super-band
-    for (int sb = warp; sb < s_nsb; sb += nwarps) {
+    // G: the item list.  A team of warps per super-band; the first lanes of every warp work out the super-band's
+    //    units once (bands, height: a few dependent look-ups), every item is then a unit's record with a tile number.
+    const int wps = max(1, min(8, nwarps / max(s_nsb, 1))), teams = nwarps / wps;
+    for (int sb = warp / wps; sb < s_nsb && warp < teams * wps; sb += teams) {
+        const int sub = warp % wps;
         const int start = sc.sb_start[sb], cnt = sc.sb_nb[sb], e = sc.sb_expert[sb];
         const int o1 = sc.sb_g1off[sb], o2 = sc.sb_g2off[sb];
         if (sc.sb_kind[sb]) {
             // group of small bands: {kind | expert << 8, first schedule position, bands | rows << 8, tile}
             const int c1 = sc.sb_c1[sb], desc = cnt | (sc.sb_ntok[sb] << 8);
-            for (int idx = lane; idx < c1 + p.n2; idx += 32) {
+            for (int idx = sub * 32 + lane; idx < c1 + p.n2; idx += 32 * wps) {
                 const bool g1 = idx < c1;
                 p.items[g1 ? o1 + idx : o2 + idx - c1] =
                     make_int4((g1 ? KIND_G1S : KIND_G2S) | (e << 8), start, desc, g1 ? idx : idx - c1);
             }
             continue;
         }
-        const int nu = sc.sb_units[sb];
-        for (int idx = lane; idx < nu * (p.n1 + p.n2); idx += 32) {
-            const bool g1 = idx < nu * p.n1;
-            const int k = g1 ? idx : idx - nu * p.n1;
-            const int unit = sc.unit_tab[start + k % nu], tile = k / nu;
+        const int nu = sc.sb_units[sb];                // at most 32: a super-band holds at most 64 bands
+        const bool plain = !(sc.sb_role[sb] & 4);      // band pairs only: no table of units
+        int ux = 0, uy = 0, uz = 0;                    // lane u: kind bits, first band, second band or band count of unit u
+        if (lane < nu) {
+            const int unit = plain ? (2 * lane) | (min(2, cnt - 2 * lane) << 8) : sc.unit_tab[start + lane];
             const int o = unit & 0xff, take = (unit >> 8) & 0xff;
             const bool rider = (unit >> 16) != 0;
-            const int b0 = p.sched_band[start + o];
+            uy = p.sched_band[start + o];
             if (take > 2) {
-                // the bands of a run are consecutive in the layout: b0, b0 + 1, ...
-                p.items[(g1 ? o1 : o2) + k] = make_int4((g1 ? KIND_G1 : KIND_G2) | KIND_STACK | (e << 8), b0, take, tile);
-                continue;
+                ux = KIND_STACK;                       // the bands of a run are consecutive in the layout: b0, b0 + 1, ...
+                uz = take;
+            } else {
+                uz = take == 2 ? (rider ? uy + 1 : p.sched_band[start + o + 1]) : -1;
+                const bool low = p.low_ok && p.band_valid[uy] <= SMALL_BAND_ROWS &&
+                                 (uz < 0 || p.band_valid[uz] <= SMALL_BAND_ROWS);
+                ux = low ? KIND_LOW : 0;
             }
-            const int b1 = take == 2 ? (rider ? b0 + 1 : p.sched_band[start + o + 1]) : -1;
-            const bool low = p.low_ok && p.band_valid[b0] <= SMALL_BAND_ROWS &&
-                             (b1 < 0 || p.band_valid[b1] <= SMALL_BAND_ROWS);
-            p.items[(g1 ? o1 : o2) + k] =
-                make_int4((g1 ? KIND_G1 : KIND_G2) | (low ? KIND_LOW : 0) | (e << 8), b0, b1, tile);
+        }
+        const int total = nu * (p.n1 + p.n2);
+        for (int base = sub * 32; base < total; base += 32 * wps) {
+            const int idx = base + lane;
+            const bool active = idx < total;
+            const bool g1 = idx < nu * p.n1;
+            const int k = g1 ? idx : idx - nu * p.n1;
+            const int u = active ? k % nu : 0, tile = active ? k / nu : 0;
+            const int x = __shfl_sync(0xffffffffu, ux, u), y = __shfl_sync(0xffffffffu, uy, u);
+            const int z = __shfl_sync(0xffffffffu, uz, u);
+            if (active) p.items[(g1 ? o1 : o2) + k] = make_int4((g1 ? KIND_G1 : KIND_G2) | x | (e << 8), y, z, tile);
         }
     }
 }
