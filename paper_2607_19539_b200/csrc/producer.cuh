@@ -344,6 +344,9 @@ __device__ __forceinline__ void gather_units(const Params &p, int kflags, int la
     }
 }
 
+struct TrueT { static constexpr bool value = true; };
+struct FalseT { static constexpr bool value = false; };
+
 struct ProducerMaps {
     CUtensorMap xa, h, w1, w2;   // all 2-D bf16 row-major, box 64 x 128, 128-byte swizzle
     CUtensorMap xa8, h8;         // Xa and H again in boxes of 64 x 8: token rows of the swapped-operand items
@@ -702,30 +705,51 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
             }
             // (no proxy fence on this side: the writers of the rows issue it before their release, see above)
             if (kTrace && rank == 0) p.trace_items2[cur.it].d = globaltimer_ns();
+            // The leader announces the bytes of both CTAs.  The peer's bytes may land before this arrival; the
+            // phase still cannot complete early because the arrival itself is pending.  The peer can only refill a
+            // stage after the leader's MMAs have consumed (hence completed) its previous phase, so bytes never leak
+            // into the wrong phase.
+            // This loop sets the pace at which freed stages are refilled: one untaken branch more in it costs percents
+            // of the kernel, so the copies per stage are compile-time variants and the look-up of the next item
+            // sits between two runs of the loop.
+            const uint32_t tx = cur.low ? 2 * (PROD_A_BYTES / 2 + PROD_B_BYTES) : 2 * PROD_STAGE_BYTES;
+            const CUtensorMap *amap = cur.amap, *bmap = cur.bmap;
+            const int a_row = cur.a_row, a2_row = cur.a2_row, b_row = cur.b_row, b2_row = cur.b2_row, it_now = cur.it;
+            auto fill = [&](auto second_a, auto second_b, int ks0, int ks1) -> bool {
+                uint32_t sa = smem_base + stage * PROD_STAGE_BYTES, off = 8 * stage;   // running addresses
+                int x = ks0 * TB_K;
+                for (int ks = ks0; ks < ks1; ++ks) {
+                    if (!mbar_wait(bar_empty + off, phase ^ 1u, p, SITE_TMA_EMPTY, it_now)) {
+                        fills += ks - ks0;      // the give-up path waits for the copies issued so far
+                        return false;
+                    }
+                    const uint32_t full = lead_full + off;
+                    if (rank == 0) mbar_arrive_expect_tx(bar_full + off, tx);
+                    tma_load_2d(sa, amap, full, x, a_row);
+                    if (decltype(second_a)::value) tma_load_2d(sa + PROD_A_BYTES / 2, amap, full, x, a2_row);
+                    tma_load_2d(sa + PROD_A_BYTES, bmap, full, x, b_row);
+                    if (decltype(second_b)::value) tma_load_2d(sa + PROD_A_BYTES + PROD_B_BYTES / 2, bmap, full, x, b2_row);
+                    x += TB_K;
+                    sa += PROD_STAGE_BYTES;
+                    off += 8;
+                    if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; sa = smem_base; off = 0; }
+                }
+                fills += ks1 - ks0;
+                return true;
+            };
+            auto fill_any = [&](int ks0, int ks1) -> bool {
+                if (cur.a2_row >= 0) return fill(TrueT{}, FalseT{}, ks0, ks1);      // stacked bands
+                if (cur.b2_row >= 0) return fill(FalseT{}, TrueT{}, ks0, ks1);      // 64-row-high first GEMM
+                return fill(FalseT{}, FalseT{}, ks0, ks1);
+            };
             int have_next = 0;
             const int look = cur.ksteps > PROD_LOOKAHEAD ? cur.ksteps - PROD_LOOKAHEAD : 0;
-            for (int ks = 0; ks < cur.ksteps; ++ks) {
-                ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, p, SITE_TMA_EMPTY, cur.it);
-                if (!ok) break;
-                const uint32_t sa = smem_base + stage * PROD_STAGE_BYTES, sb = sa + PROD_A_BYTES;
-                const uint32_t full = lead_full + 8 * stage;
-                // The leader announces the bytes of both CTAs.  The peer's bytes may land before this
-                // arrival; the phase still cannot complete early because the arrival itself is pending.
-                // The peer can only refill a stage after the leader's MMAs have consumed (hence completed)
-                // its previous phase, so bytes never leak into the wrong phase.
-                if (rank == 0)
-                    mbar_arrive_expect_tx(bar_full + 8 * stage, cur.low ? 2 * (PROD_A_BYTES / 2 + PROD_B_BYTES) : 2 * PROD_STAGE_BYTES);
-                tma_load_2d(sa, cur.amap, full, ks * TB_K, cur.a_row);
-                if (cur.a2_row >= 0) tma_load_2d(sa + PROD_A_BYTES / 2, cur.amap, full, ks * TB_K, cur.a2_row);
-                tma_load_2d(sb, cur.bmap, full, ks * TB_K, cur.b_row);
-                if (cur.b2_row >= 0) tma_load_2d(sb + PROD_B_BYTES / 2, cur.bmap, full, ks * TB_K, cur.b2_row);
-                ++fills;
-                if (++stage == PROD_STAGES) { stage = 0; phase ^= 1u; }
-                if (ks == look) {
-                    have_next = fetch(n + 1, nxt);
-                    if (have_next < 0) { ok = false; break; }
-                }
-            }
+            ok = fill_any(0, look + 1);
+            if (!ok) continue;
+            have_next = fetch(n + 1, nxt);
+            if (have_next < 0) { ok = false; continue; }
+            ok = fill_any(look + 1, cur.ksteps);
+            if (!ok) continue;
             cur = nxt;
             have = have_next;
         }
