@@ -34,7 +34,7 @@ constexpr int SWAP_MAX_N = 128;
 constexpr int SWAP_MAX_BANDS = 8;          // SWAP_MAX_N / 16
 
 // meta[] slots written by the plan kernel
-enum { META_P = 0, META_BANDS, META_ITEMS, META_SEGS, META_SUPERBANDS, META_COUNT = 8 };
+enum { META_P = 0, META_BANDS, META_ITEMS, META_SEGS, META_SUPERBANDS, META_GATHER_ORDER, META_COUNT = 8 };
 // stamps[] slots.  "first" stamps hold ~t so that the cleared state (0) is neutral under atomicMax.
 enum { STAMP_START_INV = 0, STAMP_FIRST_FLAG_INV, STAMP_LAST_FLAG, STAMP_LAST_SEG, STAMP_COPY_NS, STAMP_COPY_BYTES,
        STAMP_COUNT };
@@ -98,6 +98,7 @@ struct Params {
     int *slot;            // [M]
     int *band_expert, *band_dest, *band_valid, *band_slot0;   // [max_bands]
     int *sched_band;      // [max_bands]
+    int *gather_band;     // [max_bands] bands in the order they are gathered, when meta[META_GATHER_ORDER] is set
     int4 *items;          // [max_items] {kind | expert << 8, band 0, band 1 or -1, tile}
     int4 *segs;           // [max_bands] {first band, bands, dest, rows}
     int *seg_slot0;       // [max_bands]

@@ -33,7 +33,7 @@ struct Layout {
     size_t zero_begin, bitmap, hcount, fcount, status, next_item, stamps, tok_slot, zero_end;   // cleared at the start of every call
     size_t smid;
     size_t wordpfx, group_rows, group_start, group_slot, pos, slot, row_at, xready;
-    size_t band_expert, band_dest, band_valid, band_slot0, sched_band, items, segs, seg_slot0;
+    size_t band_expert, band_dest, band_valid, band_slot0, sched_band, gather_band, items, segs, seg_slot0;
     size_t tok_gate, flags, meta;
     size_t trace_items, trace_items2, trace_units, trace_item_aux, trace_bytes;   // MOE_OVL_FLAG_TRACE
     size_t sb[13];
@@ -115,6 +115,7 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->band_valid = take((size_t)L->max_bands * 4);
     L->band_slot0 = take((size_t)L->max_bands * 4);
     L->sched_band = take((size_t)L->max_bands * 4);
+    L->gather_band = take((size_t)L->max_bands * 4);
     L->items = take((size_t)L->max_items * 16);
     L->segs = take((size_t)L->max_bands * 16);
     L->seg_slot0 = take((size_t)L->max_bands * 4);
@@ -225,6 +226,7 @@ Params make_params(moe_ovl_ctx *ctx)
     p.group_slot = at<int>(ctx, L.group_slot); p.pos = at<int>(ctx, L.pos); p.slot = at<int>(ctx, L.slot);
     p.band_expert = at<int>(ctx, L.band_expert); p.band_dest = at<int>(ctx, L.band_dest);
     p.band_valid = at<int>(ctx, L.band_valid); p.band_slot0 = at<int>(ctx, L.band_slot0);
+    p.gather_band = at<int>(ctx, L.gather_band);
     p.sched_band = at<int>(ctx, L.sched_band); p.items = at<int4>(ctx, L.items); p.segs = at<int4>(ctx, L.segs);
     p.seg_slot0 = at<int>(ctx, L.seg_slot0); p.tok_slot = at<int>(ctx, L.tok_slot);
     p.tok_gate = at<float>(ctx, L.tok_gate); p.hcount = at<unsigned>(ctx, L.hcount);

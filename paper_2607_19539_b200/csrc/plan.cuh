@@ -116,6 +116,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     __shared__ int s_total;
     __shared__ int segs_per_rank[PLAN_MAX_GROUPS];
     __shared__ int s_nsb;
+    __shared__ int s_any_rider, s_riders;
     __shared__ int s_sb_c1[PLAN_SB_STAGE], s_sb_c2[PLAN_SB_STAGE], s_sb_end[PLAN_SB_STAGE];
     __shared__ unsigned char erider[PLAN_MAX_EXPERTS];   // the expert's local band rides with its last remote bands
 
@@ -156,7 +157,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     //    every group rounded up to a multiple of tb_M; receive-buffer slots expert-major and dense.
     //    One thread per expert lays out its own groups relative to the expert's start; a short prefix over
     //    the experts then places the experts.
-    if (tid == 0) s_total = 0;
+    if (tid == 0) { s_total = 0; s_any_rider = 0; }
     __syncthreads();
     for (int e = tid; e < El; e += blockDim.x) {
         int cur = 0, remote_bands = 0, rows = 0;
@@ -207,6 +208,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
         eorder[rank] = e;
     }
     __syncthreads();
+    // key[] is free now: it becomes the inverse of eorder (position of an expert among the remote runs)
+    for (int i = tid; i < El; i += blockDim.x) key[eorder[i]] = i;
 
     // D: schedule positions of groups.  Runs: the remote bands of each expert in sorted order (rule (i):
     //    all remote tiles first), then the local bands of each expert in natural order.  One thread per run
@@ -416,6 +419,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
             n_local <= SMALL_BAND_ROWS && run_nsb[El + e] < 0 && all_small(last_o, last_take)) {
             sc.unit_tab[start + units - 1] = last_o | ((last_take + 1) << 8) | (1 << 16);
             erider[e] = 1;
+            s_any_rider = 1;
         }
         sc.sb_units[sb] = units;
     }
@@ -443,6 +447,16 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
             if (staged) { s_sb_c1[i] = c1; s_sb_c2[i] = c2; }
         }
         __syncthreads();
+        if (tid == 32 && s_any_rider) {
+            // Riders change the order in which the GEMM needs the bands, so the gather follows them (below): how many
+            // riders come before the i-th remote run, and before the local run of expert e.  (esize[] and eorder[]
+            // are free by now; this thread works while thread 0 is in the serial loop.)
+            int before = 0;
+            for (int i = 0; i < El; ++i) { esize[i] = before; before += erider[run_exp[i]]; }
+            s_riders = before;
+            before = 0;
+            for (int e = 0; e < El; ++e) { eorder[e] = before; before += erider[e]; }
+        }
         if (tid == 0) {
             int *c1v = staged ? s_sb_c1 : sc.sb_c1, *c2v = staged ? s_sb_c2 : sc.sb_c2;
             int *endv = staged ? s_sb_end : sc.sb_g1end;
@@ -514,6 +528,24 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
             const int x = __shfl_sync(0xffffffffu, ux, u), y = __shfl_sync(0xffffffffu, uy, u);
             const int z = __shfl_sync(0xffffffffu, uz, u);
             if (active) p.items[(g1 ? o1 : o2) + k] = make_int4((g1 ? KIND_G1 : KIND_G2) | x | (e << 8), y, z, tile);
+        }
+    }
+
+    // H: the order in which the GEMM kernel's gather warps fill the layout.  It is the schedule order of the bands,
+    //    except that a riding local band is needed with its expert's remote bands, long before its place in the
+    //    schedule: it is gathered right after them.
+    if (tid == 0) p.meta[META_GATHER_ORDER] = s_any_rider;
+    if (s_any_rider) {
+        for (int g = warp; g < G; g += nwarps) {
+            const int e = g / R, r = g % R;
+            for (int b = lane; b < nb[g]; b += 32) {
+                const int spos = gsched[g] + b;
+                int at;
+                if (r != self) at = spos + esize[key[e]];
+                else if (erider[e]) at = run_start[key[e]] + run_nb[key[e]] + esize[key[e]];
+                else at = spos + s_riders - eorder[e];
+                p.gather_band[at] = gstart[g] / TB_M + b;
+            }
         }
     }
 }

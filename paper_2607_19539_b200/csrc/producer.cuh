@@ -320,6 +320,7 @@ __device__ __forceinline__ void gather_unit(const Params &p, int band, int r0, i
 __device__ __forceinline__ void gather_units(const Params &p, int kflags, int lane)
 {
     const int nbands = p.meta[META_BANDS];
+    const int *order = p.meta[META_GATHER_ORDER] ? p.gather_band : p.sched_band;   // see the plan kernel, phase H
     const int head_bands = min(nbands, p.group_bands);
     const int head_units = head_bands * (TB_M / GATHER_HEAD_ROWS);
     const int nunits = head_units + (nbands - head_bands) * (TB_M / GATHER_ROWS);
@@ -333,11 +334,11 @@ __device__ __forceinline__ void gather_units(const Params &p, int kflags, int la
             // test hook: leave band 0 of the schedule ungathered, so that the wait for it runs out
         } else if (unit < head_units) {
             const int per = TB_M / GATHER_HEAD_ROWS;
-            gather_unit<GATHER_HEAD_ROWS, 16 / GATHER_HEAD_ROWS>(p, p.sched_band[unit / per],
+            gather_unit<GATHER_HEAD_ROWS, 16 / GATHER_HEAD_ROWS>(p, order[unit / per],
                                                                  (unit % per) * GATHER_HEAD_ROWS, lane);
         } else {
             const int u = unit - head_units, per = TB_M / GATHER_ROWS;
-            gather_unit<GATHER_ROWS, 16 / GATHER_ROWS>(p, p.sched_band[head_bands + u / per],
+            gather_unit<GATHER_ROWS, 16 / GATHER_ROWS>(p, order[head_bands + u / per],
                                                        (u % per) * GATHER_ROWS, lane);
         }
         unit = __shfl_sync(0xffffffffu, next, 0);
