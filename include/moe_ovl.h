@@ -175,7 +175,7 @@ typedef struct {
     float ms_prep;            /* plan + gather into the aligned layout */
     float ms_expert_return;   /* start of the GEMM to the last row landed in ret */
     float ms_producer;        /* the GEMM kernel alone */
-    float ms_mover;           /* consumer (OVERLAP: concurrent with the GEMM) or scatter kernel */
+    float ms_mover;           /* consumer (OVERLAP: concurrent with the GEMM) or scatter kernel; 0 for the in-kernel return */
     float ms_combine;
     /* device timestamps (%globaltimer), microseconds after the first GEMM CTA started; OVERLAP mode */
     float us_first_flag;      /* first output tile flagged: the consumer's window opens */

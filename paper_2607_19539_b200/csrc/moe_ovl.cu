@@ -161,7 +161,9 @@ struct moe_ovl_ctx {
     unsigned long long host_calls;
     cudaEvent_t ev_fork, ev_prod_done, ev_cons_done;
     // timing: call start, after prep, GEMM start/end, mover start/end, call end
-    cudaEvent_t t_begin, t_prep, t_p0, t_p1, t_m0, t_m1, t_end;
+    cudaEvent_t t_begin, t_m0, t_m1, t_end;   // GEMM start / end: h_p0 / h_p1 of the call's history slot
+    int last_hist;
+    bool last_dedicated;
     // GEMM start/end of the last HISTORY calls, so that a caller can average the kernel's duration over a run
     // of back-to-back calls without synchronising between them
     cudaEvent_t h_p0[MOE_OVL_TIMING_HISTORY], h_p1[MOE_OVL_TIMING_HISTORY];
@@ -403,7 +405,7 @@ int moe_ovl_create(moe_ovl_ctx **out, const moe_ovl_config *cfg, void *workspace
     }
     cudaEvent_t *plain[] = {&ctx->ev_fork, &ctx->ev_prod_done, &ctx->ev_cons_done};
     for (auto e : plain) CREATE_CHECK(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
-    cudaEvent_t *timed[] = {&ctx->t_begin, &ctx->t_prep, &ctx->t_p0, &ctx->t_p1, &ctx->t_m0, &ctx->t_m1, &ctx->t_end};
+    cudaEvent_t *timed[] = {&ctx->t_begin, &ctx->t_m0, &ctx->t_m1, &ctx->t_end};
     for (auto e : timed) CREATE_CHECK(cudaEventCreate(e));
     for (int i = 0; i < MOE_OVL_TIMING_HISTORY; ++i) {
         CREATE_CHECK(cudaEventCreate(&ctx->h_p0[i]));
@@ -454,8 +456,8 @@ int moe_ovl_destroy(moe_ovl_ctx *ctx)
     for (int s = 0; s < 2; ++s)
         for (cudaEvent_t e : {ctx->ev_h2d[s], ctx->ev_comp[s], ctx->ev_d2h[s]})
             if (e) cudaEventDestroy(e);
-    cudaEvent_t evs[] = {ctx->ev_fork, ctx->ev_prod_done, ctx->ev_cons_done, ctx->t_begin, ctx->t_prep, ctx->t_p0,
-                         ctx->t_p1, ctx->t_m0, ctx->t_m1, ctx->t_end};
+    cudaEvent_t evs[] = {ctx->ev_fork, ctx->ev_prod_done, ctx->ev_cons_done, ctx->t_begin, ctx->t_m0, ctx->t_m1,
+                         ctx->t_end};
     for (auto e : evs)
         if (e) cudaEventDestroy(e);
     for (int i = 0; i < MOE_OVL_TIMING_HISTORY; ++i) {
@@ -561,7 +563,7 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
         ++launches;
     }
     CU_CHECK(ctx, cudaGetLastError());
-    TIME_POINT(ctx->t_prep, st);
+    // (the end of the plan is the start of the GEMM: one event, recorded below)
 
     if (dedicated) {
         // ---- two persistent kernels on two streams, disjoint SM sets (Section 3.3.3)
@@ -572,10 +574,8 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
         // GPU whose free SMs do not hold both grids), the GEMM runs to completion, its own CTAs drain every
         // segment at the end, and the consumer then finds nothing left -- instead of a consumer that waits for
         // flags nobody can raise.  With both grids resident the order makes no difference.
-        TIME_POINT(ctx->t_p0, ctx->s_prod);
         TIME_POINT(ctx->h_p0[hist], ctx->s_prod);
         launch_producer(prod_ctas, ctx->s_prod, maps, p, kflags);
-        TIME_POINT(ctx->t_p1, ctx->s_prod);
         TIME_POINT(ctx->h_p1[hist], ctx->s_prod);
         CU_CHECK(ctx, cudaEventRecord(ctx->ev_prod_done, ctx->s_prod));
         TIME_POINT(ctx->t_m0, ctx->s_cons);
@@ -589,18 +589,16 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
         // ---- one GEMM kernel on every SM.  IN_KERNEL: its spare warps move the finished segments while the
         //      tensor cores work.  NON_OVERLAP (the comparison baseline): it runs to completion, then a separate
         //      scatter kernel moves all rows.
-        TIME_POINT(ctx->t_p0, st);
+        // Few events: each costs host time on the enqueuing thread, which is what bounds small layers.
         TIME_POINT(ctx->h_p0[hist], st);
         launch_producer(prod_ctas, st, maps, p, kflags);
         ++launches;
-        TIME_POINT(ctx->t_p1, st);
-        TIME_POINT(ctx->h_p1[hist], st);
-        TIME_POINT(ctx->t_m0, st);
+        TIME_POINT(ctx->h_p1[hist], st);          // also the start of the scatter kernel, if any
         if (!in_kernel) {
             scatter_kernel<<<ctx->scatter_blocks_per_sm * ctx->num_sms, 256, 0, st>>>(p);
             ++launches;
+            TIME_POINT(ctx->t_m1, st);
         }
-        TIME_POINT(ctx->t_m1, st);
     }
     combine_kernel<<<ctx->combine_blocks_per_sm * ctx->num_sms, 256, 0, st>>>(p);
     ++launches;
@@ -613,6 +611,8 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     ctx->hist_timed[hist] = timed;
     ++ctx->calls;
     ctx->last_timed = timed;
+    ctx->last_hist = hist;
+    ctx->last_dedicated = dedicated;
     ctx->last_mode = mode;
     ctx->last_prod_ctas = prod_ctas;
     ctx->last_cons_ctas = cons_ctas;
@@ -726,11 +726,17 @@ int moe_ovl_get_report(moe_ovl_ctx *ctx, moe_ovl_report *r)
     if (ctx->last_timed) {
         float prod_end = 0.f, mover_end = 0.f;
         CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_total, ctx->t_begin, ctx->t_end));
-        CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_prep, ctx->t_begin, ctx->t_prep));
-        CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_producer, ctx->t_p0, ctx->t_p1));
-        CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_mover, ctx->t_m0, ctx->t_m1));
-        CU_CHECK(ctx, cudaEventElapsedTime(&prod_end, ctx->t_prep, ctx->t_p1));
-        CU_CHECK(ctx, cudaEventElapsedTime(&mover_end, ctx->t_prep, ctx->t_m1));
+        const cudaEvent_t p0 = ctx->h_p0[ctx->last_hist], p1 = ctx->h_p1[ctx->last_hist];
+        CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_prep, ctx->t_begin, p0));
+        CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_producer, p0, p1));
+        prod_end = r->ms_producer;
+        if (!ctx->last_dedicated && ctx->last_mode == MOE_OVL_MODE_IN_KERNEL) {
+            r->ms_mover = 0.f;                  // the return is inside the GEMM kernel: no phase of its own
+            mover_end = prod_end;
+        } else {
+            CU_CHECK(ctx, cudaEventElapsedTime(&r->ms_mover, ctx->last_dedicated ? ctx->t_m0 : p1, ctx->t_m1));
+            CU_CHECK(ctx, cudaEventElapsedTime(&mover_end, p0, ctx->t_m1));
+        }
         r->ms_expert_return = std::max(prod_end, mover_end);
         r->ms_combine = r->ms_total - r->ms_prep - r->ms_expert_return;
     }
