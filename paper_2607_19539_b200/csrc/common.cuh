@@ -70,6 +70,8 @@ struct Params {
     int lag_items;      // schedule items between a band's last first-GEMM tile and its first second-GEMM tile
     int words;          // 32-bit words of one (expert, rank) token bitmap = ceil(T / 32)
     int n1, n2;         // tiles per band: F / 128 (0 for single-projection experts) and dout / 256
+    int zero_early;     // overlapped return: the movers write the rows of `out` whose token selected no local expert
+                        // while they have nothing to move yet; the combine kernel then skips those rows
     int low_ok;         // band pairs whose bands hold at most SMALL_BAND_ROWS rows each are issued with KIND_LOW;
                         // 2: and two such pairs side by side as one KIND_STACK item; 3: and an expert's small local band
                         // may join the last item of its remote bands
@@ -111,6 +113,7 @@ struct Params {
     int *next_seg;        // segments claimed so far (consumer CTAs, and GEMM CTAs once they are out of tiles)
     int *next_item;       // schedule items claimed so far (GEMM CTA pairs take them in order)
     int *next_gather;     // gather units claimed so far (GEMM CTAs' gather warps)
+    int *next_zero;       // chunks of tokens claimed so far by the movers that write the all-zero rows of `out`
     int *row_at;          // [P] input row held by every aligned position (valid positions only)
     unsigned *xready;     // [max_bands] rows of the band gathered into Xa (128 = ready)
     unsigned *hcount;     // [max_bands] first-GEMM tiles finished per band

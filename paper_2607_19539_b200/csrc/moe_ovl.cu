@@ -97,7 +97,7 @@ int make_layout(const moe_ovl_config *c, Layout *L)
     L->hcount = take((size_t)L->max_bands * 4);
     L->fcount = take((size_t)L->max_bands * L->n2 * 4);
     L->status = take(ST_COUNT * 4);
-    L->next_item = take(32);                 // next_item, plan_ticket, next_seg, assist_segs, next_gather
+    L->next_item = take(32);                 // next_item, plan_ticket, next_seg, assist_segs, next_gather, next_zero
     L->stamps = take(STAMP_COUNT * 8);
     L->tok_slot = take(ntok * L->kmax * 4);
     L->zero_end = off;
@@ -243,6 +243,7 @@ Params make_params(moe_ovl_ctx *ctx)
     p.next_seg = at<int>(ctx, L.next_item) + 2;
     p.assist_segs = at<int>(ctx, L.next_item) + 3;
     p.next_gather = at<int>(ctx, L.next_item) + 4;
+    p.next_zero = at<int>(ctx, L.next_item) + 5;
     p.row_at = at<int>(ctx, L.row_at);
     p.xready = at<unsigned>(ctx, L.xready);
     p.stamps = at<unsigned long long>(ctx, L.stamps);
@@ -512,6 +513,7 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     p.M = a->num_rows;
     p.lag_items = prod_ctas;                        // two rounds of the prod_ctas / 2 CTA pairs
     p.seg_chunks = MAX_SEG_CHUNKS;
+    p.zero_early = mode != MOE_OVL_MODE_NON_OVERLAP;
     p.tail_segs = in_kernel ? -1 : p.group_bands;       // dedicated consumer: whole segments but for the last super-band's
     p.ret_rows_per_rank = a->ret_rows_per_rank;
     p.x = static_cast<const uint16_t *>(a->x);

@@ -46,6 +46,31 @@ struct MoverGroup {
     }
 };
 
+// A token that selected no local expert gets a row of zeros in `out` (the empty sum of Section 2.1, step 5): half of
+// the tokens at top-2 of 8 experts with 2 local ones.  With an overlapped return the spare warps of the GEMM CTAs
+// write those rows once the layout is gathered, so that this part of the reduction's memory traffic is hidden behind
+// the GEMM as well; the combine kernel then only writes the tokens that have rows.  (Which tokens those are is known
+// before the GEMM starts: the plan kernels have filled the per-token slot lists.)  All threads of the group call this.
+constexpr int ZERO_CHUNK_TOKENS = 64;
+__device__ __forceinline__ void zero_fill_rows(const Params &p, const MoverGroup &g)
+{
+    const int ntok = p.R * p.T, nv = p.dout / 8;
+    volatile int *s_unit = g.s_unit;
+    for (;;) {
+        g.sync();
+        if (g.tid == 0) s_unit[0] = atomicAdd(p.next_zero, 1);
+        g.sync();
+        const int t0 = s_unit[0] * ZERO_CHUNK_TOKENS;
+        if (t0 >= ntok) return;
+        const int t1 = min(ntok, t0 + ZERO_CHUNK_TOKENS);
+        for (int tok = t0 + (g.tid >> 5); tok < t1; tok += g.nthr >> 5) {       // a warp per token
+            if (p.tok_slot[(size_t)tok * p.kmax] != 0) continue;              // has a row: the combine kernel's
+            uint4 *o = reinterpret_cast<uint4 *>(p.out + (size_t)tok * p.dout);
+            for (int v = g.tid & 31; v < nv; v += 32) __stcs(o + v, make_uint4(0, 0, 0, 0));
+        }
+    }
+}
+
 // Segment mover shared by the consumer CTAs, by GEMM CTAs that have run out of tiles and by the spare warps of
 // GEMM CTAs (in-kernel return): claim the next unit in schedule order, wait (bounded, acquire) until every tile
 // of every band of its segment is flagged, then move the unit's valid rows into the owner rank's receive buffer
@@ -178,6 +203,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const Params p)
 #pragma unroll
         for (int j = 0; j < KFAST; ++j) { cs[j] = slot[j]; cg[j] = gate[j]; }
         fetch(tok + tok_stride);
+        if (p.zero_early && cs[0] <= 0) continue;     // no local row: its zeros were written during the GEMM
         // two 16-byte vectors per thread and iteration: all of their row loads are issued before any arithmetic
         for (int v0 = lt; v0 < nv; v0 += 2 * tpt) {
             const int v1 = v0 + tpt;

@@ -866,10 +866,11 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
         // In-kernel return: with Xa complete these warps have nothing left to do, so they take over the
         // consumer's job on this SM -- no SM is taken from the GEMM.  They only ever wait on tile flags, which
         // the epilogue warps raise without waiting on anybody.
-        if (warp_movers) {
+        if (warp_movers || p.zero_early) {
             MoverGroup g{(int)threadIdx.x - 224, 32 * PROD_GATHER_WARPS, 3,
                          reinterpret_cast<int *>(smem_gen + (mover_ints - smem_base)), TRACE_BY_GEMM_WARPS};
-            move_segments(p, g);
+            if (p.zero_early) zero_fill_rows(p, g);     // also with a dedicated consumer, whose few CTAs are too slow for it
+            if (warp_movers) move_segments(p, g);
         }
     } else {
         // ---------------- epilogue: warps 2..5 own tensor-memory lanes 32*(warp % 4) .. +31
