@@ -311,6 +311,23 @@ void choose_mode(const moe_ovl_ctx *ctx, int num_rows, int *mode, int *consumer_
     if (t_ded < best) { best = t_ded; *mode = MOE_OVL_MODE_OVERLAP; }
 }
 
+// Should the all-zero rows of `out` be written behind the GEMM (see zero_fill_rows)?  Their writes share HBM with
+// the GEMM's own traffic: worth it where the GEMM is long against them (0.990 against 0.999 of the baseline at the
+// Mixtral shape), a loss where the layer is already traffic-heavy (the paper's single-projection operator with
+// K = 2048: the GEMM kernel grew by 12 %).  Taken when the estimated GEMM time is at least sixteen times the time
+// the zero rows take alone (half of the tokens assumed to have none, 3.3 TB/s of writes).
+bool zero_rows_behind_gemm(const moe_ovl_ctx *ctx, int num_rows)
+{
+    const moe_ovl_config &c = ctx->cfg;
+    const Layout &L = ctx->L;
+    const double groups = (double)c.num_local_experts * c.num_src_ranks;
+    const double padded = num_rows + 0.5 * TB_M * groups;
+    const double flop_row = L.single ? 2.0 * c.d_model * L.dout : 6.0 * (double)c.d_model * c.d_ffn;
+    const double gemm = padded * flop_row / (8.6e12 * ctx->num_sms);
+    const double zeros = 0.5 * (double)c.num_src_ranks * c.tokens_per_rank * L.dout * 2.0 / 3.3e12;
+    return gemm >= 16.0 * zeros;
+}
+
 // Two builds of the GEMM kernel: the one with the trace bookkeeping compiled in runs only for contexts that asked
 // for a trace, so that the bookkeeping costs nothing otherwise.
 void launch_producer(int ctas, cudaStream_t st, const ProducerMaps &maps, const Params &p, int kflags)
@@ -513,7 +530,7 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     p.M = a->num_rows;
     p.lag_items = prod_ctas;                        // two rounds of the prod_ctas / 2 CTA pairs
     p.seg_chunks = MAX_SEG_CHUNKS;
-    p.zero_early = mode != MOE_OVL_MODE_NON_OVERLAP;
+    p.zero_early = mode != MOE_OVL_MODE_NON_OVERLAP && zero_rows_behind_gemm(ctx, a->num_rows);
     p.tail_segs = in_kernel ? -1 : p.group_bands;       // dedicated consumer: whole segments but for the last super-band's
     p.ret_rows_per_rank = a->ret_rows_per_rank;
     p.x = static_cast<const uint16_t *>(a->x);

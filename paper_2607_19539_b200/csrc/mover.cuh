@@ -52,16 +52,17 @@ struct MoverGroup {
 // the GEMM as well; the combine kernel then only writes the tokens that have rows.  (Which tokens those are is known
 // before the GEMM starts: the plan kernels have filled the per-token slot lists.)  All threads of the group call this.
 constexpr int ZERO_CHUNK_TOKENS = 64;
-__device__ __forceinline__ void zero_fill_rows(const Params &p, const MoverGroup &g)
+// Writes at most max_chunks chunks; false when there are none left.
+__device__ __forceinline__ bool zero_fill_rows(const Params &p, const MoverGroup &g, int max_chunks = 0x7fffffff)
 {
     const int ntok = p.R * p.T, nv = p.dout / 8;
     volatile int *s_unit = g.s_unit;
-    for (;;) {
+    for (int done = 0; done < max_chunks; ++done) {
         g.sync();
         if (g.tid == 0) s_unit[0] = atomicAdd(p.next_zero, 1);
         g.sync();
         const int t0 = s_unit[0] * ZERO_CHUNK_TOKENS;
-        if (t0 >= ntok) return;
+        if (t0 >= ntok) return false;
         const int t1 = min(ntok, t0 + ZERO_CHUNK_TOKENS);
         for (int tok = t0 + (g.tid >> 5); tok < t1; tok += g.nthr >> 5) {       // a warp per token
             if (p.tok_slot[(size_t)tok * p.kmax] != 0) continue;              // has a row: the combine kernel's
@@ -69,6 +70,7 @@ __device__ __forceinline__ void zero_fill_rows(const Params &p, const MoverGroup
             for (int v = g.tid & 31; v < nv; v += 32) __stcs(o + v, make_uint4(0, 0, 0, 0));
         }
     }
+    return true;
 }
 
 // Segment mover shared by the consumer CTAs, by GEMM CTAs that have run out of tiles and by the spare warps of
@@ -79,7 +81,9 @@ __device__ __forceinline__ void zero_fill_rows(const Params &p, const MoverGroup
 // the schedule, whose tiles finish together at the very end of the GEMM -- sliced, they spread over every CTA
 // that is free by then instead of keeping p.tail_segs CTAs busy for a whole segment each; the spare warps of the
 // GEMM CTAs move slices throughout.  All threads of the group must call this together.
-__device__ __forceinline__ void move_segments(const Params &p, const MoverGroup &g)
+// with_zero_rows: the group also writes the all-zero rows of `out`, a few chunks before every unit it moves, so that
+// those writes are spread over the whole GEMM (as one burst at its start they held the GEMM's own loads up).
+__device__ __forceinline__ void move_segments(const Params &p, const MoverGroup &g, bool with_zero_rows = false)
 {
     const int nseg = p.meta[META_SEGS];
     const int chunks = p.seg_chunks;
@@ -88,7 +92,11 @@ __device__ __forceinline__ void move_segments(const Params &p, const MoverGroup 
     const int lane = g.tid & 31;
     const unsigned epoch = *p.epoch;
     volatile int *s_unit = g.s_unit;
+    const int zero_chunks = (p.R * p.T + ZERO_CHUNK_TOKENS - 1) / ZERO_CHUNK_TOKENS;
+    const int zero_per_unit = zero_chunks / max(nunits, 1) + 1;
+    bool zero_left = with_zero_rows;
     for (;;) {
+        if (zero_left) zero_left = zero_fill_rows(p, g, zero_per_unit);
         g.sync();
         if (g.tid < 32) {
             int u = 0;
@@ -107,7 +115,10 @@ __device__ __forceinline__ void move_segments(const Params &p, const MoverGroup 
         }
         g.sync();
         const int u = s_unit[0];
-        if (u >= nunits || !s_unit[1]) return;
+        if (u >= nunits || !s_unit[1]) {
+            if (zero_left && s_unit[1]) zero_fill_rows(p, g);      // whatever is left of the zero rows
+            return;
+        }
         const int s = u < whole ? u : whole + (u - whole) / chunks, c = u < whole ? 0 : (u - whole) % chunks;
         const int my_chunks = u < whole ? 1 : chunks;
         const int4 seg = p.segs[s];

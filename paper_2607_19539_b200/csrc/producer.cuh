@@ -869,8 +869,9 @@ producer_kernel(const __grid_constant__ ProducerMaps maps, const Params p, const
         if (warp_movers || p.zero_early) {
             MoverGroup g{(int)threadIdx.x - 224, 32 * PROD_GATHER_WARPS, 3,
                          reinterpret_cast<int *>(smem_gen + (mover_ints - smem_base)), TRACE_BY_GEMM_WARPS};
-            if (p.zero_early) zero_fill_rows(p, g);     // also with a dedicated consumer, whose few CTAs are too slow for it
-            if (warp_movers) move_segments(p, g);
+            // (the zero rows also with a dedicated consumer, whose few CTAs are too slow for them)
+            if (warp_movers) move_segments(p, g, p.zero_early != 0);
+            else zero_fill_rows(p, g);
         }
     } else {
         // ---------------- epilogue: warps 2..5 own tensor-memory lanes 32*(warp % 4) .. +31
