@@ -281,7 +281,7 @@ int choose_consumer_sms(const moe_ovl_ctx *ctx)
 // the trade-off and leaves the choice to future work).  A three-line cost model over what the host knows --
 // the shape and the number of rows -- with coefficients measured on a B200 at its power cap:
 //   GEMM      padded flop / (8.6 TFLOP/s per GEMM CTA): 148 CTAs reach about 1270 TFLOP/s sustained
-//   scatter   non-overlap only: a launch boundary (about 6 us) + 4*dout bytes per row at 5.5 TB/s
+//   scatter   non-overlap only: a launch boundary and its timing event (about 10 us) + 4*dout bytes per row at 5.5 TB/s
 //   tail      what is left to move after the last tile is flagged: one segment per mover.  A consumer CTA
 //             moves about 35 GB/s of payload, the four spare warps of a GEMM CTA about 15 GB/s of a unit that
 //             is an eighth of a segment
@@ -301,7 +301,7 @@ void choose_mode(const moe_ovl_ctx *ctx, int num_rows, int *mode, int *consumer_
     const double gemm_all = padded * flop_row / (8.6e12 * sms);            // seconds on every SM
     const double row_bytes = 2.0 * L.dout;
     const double seg_bytes = (double)std::max(1, c.mid_seg_bands) * TB_M * row_bytes;
-    const double t_non = gemm_all + 6e-6 + 2.0 * row_bytes * num_rows / 5.5e12;
+    const double t_non = gemm_all + 10e-6 + 2.0 * row_bytes * num_rows / 5.5e12;
     const double t_in = gemm_all * 1.004 + (seg_bytes / MAX_SEG_CHUNKS) / 15e9;
     const double cs = *consumer_sms;
     const double t_ded = gemm_all * sms / (sms - cs) + seg_bytes / 35e9 / std::max(1.0, cs / 4.0);
