@@ -104,6 +104,9 @@ typedef struct {
                                          and 9 of moe_ovl_plan_view.item); for comparisons */
 #define MOE_OVL_FLAG_NO_LOCAL_RIDERS 128u /* never let an expert's local band join the last item of its remote bands (see
                                          moe_ovl_plan_view.item); for comparisons */
+#define MOE_OVL_FLAG_TEST_ZERO_ROWS_EARLY 256u /* test hook: in the overlapped modes the all-zero rows of `out` (tokens
+                                         with no local expert) are written behind the GEMM also where the host's cost
+                                         rule would leave them to the combine kernel (small layers) */
 #define MOE_OVL_FLAG_TEST_ALL_SMALL_GROUP_TILES 32u /* test hook: every eligible run of small groups gets swapped-operand
                                          items, also where the plan's cost rule would keep band pairs */
 #define MOE_OVL_FLAG_TEST_SKIP_GATHER 8u /* test hook: the first band of the schedule is never gathered, so the GEMM's

@@ -26,6 +26,7 @@ FLAG_NO_SMALL_GROUP_TILES = 16
 FLAG_TEST_ALL_SMALL_GROUP_TILES = 32
 FLAG_NO_STACKED_BANDS = 64
 FLAG_NO_LOCAL_RIDERS = 128
+FLAG_TEST_ZERO_ROWS_EARLY = 256
 TRACE_ITEM, TRACE_UNIT = 0, 1
 BUF_XA, BUF_H, BUF_Y = 0, 1, 2
 TB_M, TB_N, H_TILE = 128, 256, 128

@@ -530,7 +530,8 @@ int moe_ovl_expert_return(moe_ovl_ctx *ctx, const moe_ovl_args *a)
     p.M = a->num_rows;
     p.lag_items = prod_ctas;                        // two rounds of the prod_ctas / 2 CTA pairs
     p.seg_chunks = MAX_SEG_CHUNKS;
-    p.zero_early = mode != MOE_OVL_MODE_NON_OVERLAP && zero_rows_behind_gemm(ctx, a->num_rows);
+    p.zero_early = mode != MOE_OVL_MODE_NON_OVERLAP &&
+                   (zero_rows_behind_gemm(ctx, a->num_rows) || (c.flags & MOE_OVL_FLAG_TEST_ZERO_ROWS_EARLY));
     p.tail_segs = in_kernel ? -1 : p.group_bands;       // dedicated consumer: whole segments but for the last super-band's
     p.ret_rows_per_rank = a->ret_rows_per_rank;
     p.x = static_cast<const uint16_t *>(a->x);

@@ -86,7 +86,8 @@ def test_overlap_equals_non_overlap_bitwise(name):
         inp = I.make_inputs(I.with_seed(shape, seed))
         dsp = I.dispatch(inp)
         probs.append((inp, dsp))
-    ctx = Hn.make_context(shape, max_rows=max(d.M for _, d in probs), flags=B.FLAG_TEST_ALL_SMALL_GROUP_TILES)
+    ctx = Hn.make_context(shape, max_rows=max(d.M for _, d in probs),
+                          flags=B.FLAG_TEST_ALL_SMALL_GROUP_TILES | B.FLAG_TEST_ZERO_ROWS_EARLY)
     refs = []
     for inp, dsp in probs:
         base = Hn.upload(inp, dsp)
@@ -353,7 +354,8 @@ def test_random_shapes_full_parity(seed):
     inp = I.make_inputs(shape)
     dsp = I.dispatch(inp, shuffle_seed=int(rng.integers(0, 99)) if seed % 2 else None)
     ctx = Hn.make_context(shape, max_rows=max(dsp.M, 1) + int(rng.integers(0, 300)), mid_seg_bands=mgb, group_bands=gb,
-                          flags=B.FLAG_TEST_ALL_SMALL_GROUP_TILES if seed % 3 else 0)
+                          flags=(B.FLAG_TEST_ALL_SMALL_GROUP_TILES if seed % 3 else 0) |
+                                (B.FLAG_TEST_ZERO_ROWS_EARLY if seed % 2 == 0 else 0))
     prob = Hn.upload(inp, dsp)
     Hn.run(ctx, prob, mode=mode, consumer_sm_count=csm)
     torch.cuda.synchronize()
@@ -392,6 +394,7 @@ def test_random_small_group_shapes_full_parity(seed):
     csm = int(rng.choice([0, 2, 6]))
     gb = int(rng.choice([0, 2, 4, 64]))
     flags = (0, 0, B.FLAG_NO_LOCAL_RIDERS, B.FLAG_TEST_ALL_SMALL_GROUP_TILES, B.FLAG_NO_STACKED_BANDS, 0)[seed % 6]
+    flags |= B.FLAG_TEST_ZERO_ROWS_EARLY if seed % 2 else 0      # zero rows of `out` written behind the GEMM
     inp = I.make_inputs(shape)
     dsp = I.dispatch(inp, shuffle_seed=int(rng.integers(0, 99)) if seed % 2 else None)
     plan = U.oracle_plan(shape, dsp)
