@@ -128,22 +128,32 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_mark_build_kernel(Params
     //    at a time so that their (independent) loads are in flight together.
     for (int g0 = warp * 4; g0 < G; g0 += nwarps * 4) {
         int run[4] = {0, 0, 0, 0};
-        for (int w0 = 0; w0 < p.words; w0 += 32) {
-            const int w = w0 + lane;
-            int c[4];
+        // four steps of 32 words per round, all sixteen loads issued before the first scan: one trip to L2 per
+        // round instead of one per step
+        for (int w0 = 0; w0 < p.words; w0 += 128) {
+            int c[4][4];
 #pragma unroll
-            for (int k = 0; k < 4; ++k)     // written by other blocks' atomics: read through L2
-                c[k] = (g0 + k < G && w < p.words) ? __popc(__ldcg(p.bitmap + (size_t)(g0 + k) * p.words + w)) : 0;
+            for (int s = 0; s < 4; ++s) {
+                const int w = w0 + 32 * s + lane;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                int inc = c[k];
+                for (int k = 0; k < 4; ++k)     // written by other blocks' atomics: read through L2
+                    c[s][k] = (g0 + k < G && w < p.words) ? __popc(__ldcg(p.bitmap + (size_t)(g0 + k) * p.words + w)) : 0;
+            }
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int v = __shfl_up_sync(0xffffffffu, inc, o);
-                    if (lane >= o) inc += v;
+            for (int s = 0; s < 4; ++s) {
+                const int w = w0 + 32 * s + lane;
+                if (w0 + 32 * s >= p.words) break;          // uniform
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    int inc = c[s][k];
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const int v = __shfl_up_sync(0xffffffffu, inc, o);
+                        if (lane >= o) inc += v;
+                    }
+                    if (g0 + k < G && w < p.words) p.wordpfx[(size_t)(g0 + k) * p.words + w] = run[k] + inc - c[s][k];
+                    run[k] += __shfl_sync(0xffffffffu, inc, 31);
                 }
-                if (g0 + k < G && w < p.words) p.wordpfx[(size_t)(g0 + k) * p.words + w] = run[k] + inc - c[k];
-                run[k] += __shfl_sync(0xffffffffu, inc, 31);
             }
         }
 #pragma unroll
